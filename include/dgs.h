@@ -1,0 +1,177 @@
+/*
+ * dgs.h -- C ABI of the DGS push / apply / pull loop on one GPU.
+ *
+ * DGS (dual-way gradient sparsification with sparsification-aware momentum,
+ * arXiv 1910.10929) lets N asynchronous workers exchange sparse updates with a
+ * parameter server in both directions.  This library keeps the N workers and the
+ * server on ONE device and runs, per arrival ("event") of a worker k:
+ *
+ *   push   worker side, Algorithm 3:  t = m*u_k + eta*grad;  per layer keep the
+ *          k_j entries of largest |t| (the packet g);  u_k <- t on the sent
+ *          entries and t*(1/m) on the others (Eq. 11a, Eq. 12).
+ *   apply  server side, Algorithm 2:  M <- M - decode(g)  (Eq. 1).  The model is
+ *          stored as theta = theta_0 + M (Eq. 2) and every worker's model
+ *          difference D_q = M - v_q (Eq. 3) moves with M.
+ *   pull   server side, Algorithm 2 with secondary compression (Eq. 6a/6b):
+ *          per layer keep the k_j entries of largest |D_k| (the packet G), clear
+ *          them in D_k (v_k <- v_k + G), leave the rest as the server's residual;
+ *          optionally the worker installs theta_k <- theta_k + G (Eq. 5).
+ *
+ * Conventions
+ *   - All numbers are IEEE binary32; every arithmetic step is one rounded
+ *     operation (no fused multiply-add, no flush-to-zero), so results do not
+ *     depend on launch shapes.  Inputs must be finite.
+ *   - "Largest |x|" compares the bit pattern of x with the sign bit cleared.
+ *     Exactly k_j entries are kept per layer; among equal magnitudes the lowest
+ *     index wins.  Packets list (index, value) pairs in ascending index order.
+ *   - DEVICE pointers are marked DEVICE, everything else is host memory.
+ *   - The caller owns all device memory (the arena) and the stream; the library
+ *     allocates no device memory.  Calls only enqueue work on the stream given at
+ *     dgs_init and return; results are ready when the stream reaches them.
+ *     One host thread per context.
+ *   - Every function returns DGS_OK (0) or a negative dgs_error.  Nothing aborts,
+ *     throws or waits without bound.
+ */
+#ifndef DGS_H_
+#define DGS_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DGS_OK = 0,
+  DGS_EINVAL = -1,   /* null pointer, worker out of range, bad segment table, m not in (0,1], n >= 2^32, misaligned pointer */
+  DGS_ENOMEM = -2,   /* arena too small */
+  DGS_ECUDA = -3,    /* a CUDA runtime call or launch failed; see dgs_last_cuda_error */
+  DGS_ETIMEOUT = -4, /* a bounded device-side wait gave up (reported by dgs_status) */
+  DGS_ESTATE = -5    /* context already freed or unusable after an earlier error */
+} dgs_error;
+
+typedef struct dgs_ctx dgs_ctx; /* opaque, host side */
+
+/* One layer j of the per-layer loops of Algorithm 3 / Algorithm 2: a contiguous
+ * slice [offset, offset+len) of the flat parameter vector that is sparsified on
+ * its own.  Segments must be listed in ascending order and tile [0, n) exactly.
+ * 1 <= k_push <= len and 1 <= k_pull <= len. */
+typedef struct {
+  uint64_t offset;
+  uint64_t len;
+  uint32_t k_push; /* entries the worker sends per push from this layer   */
+  uint32_t k_pull; /* entries the server sends per pull from this layer   */
+} dgs_segment;
+
+/* A sparse update in coordinate format (the paper's encode()): count pairs,
+ * idx ascending.  Packets returned by the library point into the context's own
+ * packet slots (DEVICE) and stay valid until the next call that produces a packet
+ * of the same kind (push or pull). */
+typedef struct {
+  const uint32_t* idx; /* DEVICE u32[count], flat parameter index */
+  const float* val;    /* DEVICE f32[count]                        */
+  uint32_t count;      /* = sum of k_push (push) or k_pull (pull)  */
+} dgs_packet;
+
+enum {
+  DGS_KEEP_LOCAL_MODEL = 1u << 0, /* keep theta_k per worker and add every pulled G to it (Eq. 5) */
+  DGS_RESIDUAL_MODE = 1u << 1,    /* worker rule of Algorithm 1 instead of Algorithm 3: v <- v + eta*grad,
+                                     sent entries leave v, the rest stay (no momentum, no 1/m rescale) */
+  DGS_HOST_IO = 1u << 2,          /* reserve staging buffers for dgs_event_host */
+  DGS_NO_SPECULATION = 1u << 3    /* always take the two-pass selection (histogram pass, then stream pass) */
+};
+
+typedef struct {
+  uint64_t n;                  /* number of parameters, 1 <= n < 2^32                                  */
+  uint32_t num_workers;        /* N >= 1                                                               */
+  float lr;                    /* eta, finite                                                          */
+  float momentum;              /* m, 0 < m <= 1 (1/m is taken once, by IEEE division)                  */
+  uint32_t num_segments;       /* S >= 1, S < 65536                                                    */
+  const dgs_segment* segments; /* HOST array [S], copied                                               */
+  const float* theta0;         /* DEVICE f32[n], initial model (Algorithm 3, first line), copied       */
+  void* arena;                 /* DEVICE memory owned by the caller, 256-byte aligned                  */
+  uint64_t arena_bytes;        /* >= what dgs_arena_bytes reports for this configuration               */
+  void* stream;                /* cudaStream_t on which all work is enqueued (NULL = default stream)   */
+  uint32_t flags;              /* DGS_* flags above                                                    */
+} dgs_config;
+
+enum { DGS_THETA = 0, DGS_U = 1, DGS_D = 2, DGS_THETA_LOCAL = 3 };
+
+/* Bytes of device memory a context for this configuration carves from the arena
+ * (model, N velocities + one spare, N differences, packet slots, selection
+ * scratch).  No GPU work.  arena/arena_bytes/theta0/stream are ignored. */
+int dgs_arena_bytes(const dgs_config* cfg, uint64_t* out_bytes);
+
+/* Creates the context: u_k = 0 and D_k = 0 for every worker (Algorithm 3 and
+ * Algorithm 2, initialisation), theta = theta0, theta_k = theta0 if kept.
+ * Enqueues the clears and copies on cfg->stream.  The arena must stay alive and
+ * untouched by others until dgs_free. */
+int dgs_init(const dgs_config* cfg, dgs_ctx** out);
+
+/* Worker push (Algorithm 3, velocity update through encode(); Eq. 11a, Eq. 12).
+ * grad: DEVICE f32[n], 16-byte aligned, read only, must stay valid until the
+ * stream has run this call.  On return *out describes the push packet slot. */
+int dgs_worker_push(dgs_ctx* ctx, uint32_t worker, const float* grad, dgs_packet* out);
+
+/* Server apply (Algorithm 2, "M <- M - decode(g)"; Eq. 1-3): theta[i] -= val and
+ * D_q[i] -= val for every worker q, the sender included, for each (i, val) of the
+ * packet.  pkt may be the library's own push packet or any DEVICE packet with
+ * strictly ascending indices < n.  Also advances the server timestamp t. */
+int dgs_server_apply(dgs_ctx* ctx, uint32_t worker, const dgs_packet* pkt);
+
+/* Worker pull with secondary compression (Algorithm 2, per-layer top-k of
+ * G = M - v_k; Eq. 6a, 6b): builds the pull packet from D_worker, clears the sent
+ * entries there, adds them to theta_worker when DGS_KEEP_LOCAL_MODEL is set
+ * (Eq. 5), and records prev(worker) = t. */
+int dgs_worker_pull(dgs_ctx* ctx, uint32_t worker, dgs_packet* out);
+
+/* One whole event for `worker`: push, apply of that packet, pull.  Either packet
+ * pointer may be NULL. */
+int dgs_event(dgs_ctx* ctx, uint32_t worker, const float* grad, dgs_packet* push_out, dgs_packet* pull_out);
+
+/* The same event with HOST buffers (needs DGS_HOST_IO): copies grad (HOST f32[n],
+ * ideally pinned) to the device, runs the event, copies the pull packet back into
+ * out_idx / out_val (HOST, sum(k_pull) entries each, may be NULL to skip) and
+ * waits for the stream.  This is the end-to-end path: what a worker process
+ * without its own device buffers would call. */
+int dgs_event_host(dgs_ctx* ctx, uint32_t worker, const float* grad_host, uint32_t* out_idx, float* out_val);
+
+/* Pointer to a state vector, DEVICE f32[n]: which = DGS_THETA (worker ignored),
+ * DGS_U, DGS_D or DGS_THETA_LOCAL.  Waits for the stream (velocity buffers are
+ * exchanged with a spare on the device, so their address is only known then).
+ * The pointer is valid until the next push of that worker (DGS_U) or dgs_free. */
+int dgs_state_ptr(dgs_ctx* ctx, int which, uint32_t worker, const float** out);
+
+/* Overwrites a state vector from src (DEVICE f32[n]) on the stream: restores a
+ * checkpoint, or loads a vector to be selected from with dgs_worker_pull. */
+int dgs_state_load(dgs_ctx* ctx, int which, uint32_t worker, const float* src);
+
+/* Waits for the stream and returns the sticky device status word in
+ * *device_status (0 = clean; negative dgs_error values are stored by kernels that
+ * detect an out-of-range index or give up a bounded wait). */
+int dgs_status(dgs_ctx* ctx, int* device_status);
+
+/* Waits for the stream and reports counters: out[0] selections served by the
+ * single-pass (speculative) route, out[1] selections that took the two-pass
+ * route, out[2] server timestamp t (packets applied), out[3] reserved. */
+int dgs_stats(dgs_ctx* ctx, uint64_t out[4]);
+
+/* prev(worker): the server timestamp at that worker's last pull, -1 before it. */
+int dgs_prev(dgs_ctx* ctx, uint32_t worker, int64_t* out);
+
+/* Number of kernels this context has launched so far (host-side count). */
+int dgs_launch_count(dgs_ctx* ctx, uint64_t* out);
+
+/* The cudaError_t of the last failed runtime call of this context (0 if none). */
+int dgs_last_cuda_error(dgs_ctx* ctx);
+
+/* Frees the host-side context.  The arena stays the caller's.  Waits for the stream. */
+int dgs_free(dgs_ctx* ctx);
+
+/* Static text for a dgs_error value. */
+const char* dgs_error_string(int err);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DGS_H_ */

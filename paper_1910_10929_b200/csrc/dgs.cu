@@ -1,0 +1,547 @@
+// Host side of the C ABI declared in include/dgs.h: argument checks, the layout of
+// the caller's arena, and the kernel launches of one push / apply / pull event.
+#include "dgs.h"
+
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "dgs_kernels.cuh"
+
+using namespace dgs;
+
+namespace {
+
+constexpr uint64_t kAlign = 256;
+constexpr uint32_t kMagic = 0x44475331u;  // "DGS1"
+constexpr uint32_t kNoBound = 0xFFFFFFFFu;
+
+inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+struct Layout {
+  uint64_t n_pad = 0;  // elements per state vector, padded to 256 bytes
+  uint32_t num_tiles = 0;
+  uint64_t K[2] = {0, 0};
+  // byte offsets into the arena
+  uint64_t theta, u, D, theta_local, grad_stage, pkt_idx[2], pkt_val[2];
+  uint64_t cand_idx, cand_val, tiles, segs, tile_count, tile_pre, cta_tot;
+  uint64_t hist1, hist2, hist3, sel, L_safe, L_next, u_slots, flags, status, stats;
+  uint64_t total = 0;
+};
+
+int check_config(const dgs_config* c) {
+  if (!c || !c->segments) return DGS_EINVAL;
+  if (c->n == 0 || c->n >= (1ull << 32)) return DGS_EINVAL;
+  if (c->num_workers == 0 || c->num_workers > 65535) return DGS_EINVAL;
+  if (c->num_segments == 0 || c->num_segments >= 65536) return DGS_EINVAL;
+  if (!std::isfinite(c->lr)) return DGS_EINVAL;
+  if (!(c->momentum > 0.0f) || !(c->momentum <= 1.0f)) return DGS_EINVAL;
+  uint64_t pos = 0;
+  for (uint32_t s = 0; s < c->num_segments; ++s) {
+    const dgs_segment& g = c->segments[s];
+    if (g.offset != pos || g.len == 0) return DGS_EINVAL;
+    if (g.k_push == 0 || g.k_push > g.len || g.k_pull == 0 || g.k_pull > g.len) return DGS_EINVAL;
+    pos += g.len;
+  }
+  if (pos != c->n) return DGS_EINVAL;
+  return DGS_OK;
+}
+
+// Tiles: every layer is cut at the global multiples of kWarpTile, so that all full
+// tiles start 2 KB-aligned and only the first and last tile of a layer can be ragged.
+void build_tiles(const dgs_config* c, std::vector<Tile>* tiles, std::vector<SegDesc>* segs) {
+  uint32_t koff[2] = {0, 0};
+  for (uint32_t s = 0; s < c->num_segments; ++s) {
+    const dgs_segment& g = c->segments[s];
+    SegDesc d;
+    d.tile_begin = tiles ? (uint32_t)tiles->size() : 0;
+    uint64_t pos = g.offset, end = g.offset + g.len;
+    uint32_t count = 0;
+    while (pos < end) {
+      const uint64_t next = std::min<uint64_t>(end, (pos / kWarpTile + 1) * kWarpTile);
+      if (tiles) {
+        Tile t;
+        t.start = (uint32_t)pos;
+        t.len = (uint16_t)(next - pos);
+        t.seg = (uint16_t)s;
+        tiles->push_back(t);
+      }
+      ++count;
+      pos = next;
+    }
+    d.tile_end = d.tile_begin + count;
+    d.k[0] = g.k_push;
+    d.k[1] = g.k_pull;
+    d.pkt_off[0] = koff[0];
+    d.pkt_off[1] = koff[1];
+    koff[0] += g.k_push;
+    koff[1] += g.k_pull;
+    if (segs) segs->push_back(d);
+  }
+}
+
+uint32_t count_tiles(const dgs_config* c) {
+  uint64_t tiles = 0;
+  for (uint32_t s = 0; s < c->num_segments; ++s) {
+    const dgs_segment& g = c->segments[s];
+    const uint64_t first = g.offset / kWarpTile, last = (g.offset + g.len - 1) / kWarpTile;
+    tiles += last - first + 1;
+  }
+  return (uint32_t)tiles;
+}
+
+void make_layout(const dgs_config* c, Layout* L) {
+  const uint64_t N = c->num_workers, S = c->num_segments;
+  L->n_pad = align_up(c->n, kAlign / 4);
+  L->num_tiles = count_tiles(c);
+  L->K[0] = L->K[1] = 0;
+  for (uint32_t s = 0; s < S; ++s) {
+    L->K[0] += c->segments[s].k_push;
+    L->K[1] += c->segments[s].k_pull;
+  }
+  uint64_t off = 0;
+  auto take = [&](uint64_t bytes) {
+    const uint64_t at = off;
+    off = align_up(off + bytes, kAlign);
+    return at;
+  };
+  const uint64_t vec = L->n_pad * 4;
+  L->theta = take(vec);
+  L->u = take(vec * (N + 1));  // N velocities and one spare that a push writes into
+  L->D = take(vec * N);
+  L->theta_local = (c->flags & DGS_KEEP_LOCAL_MODEL) ? take(vec * N) : 0;
+  L->grad_stage = (c->flags & DGS_HOST_IO) ? take(vec) : 0;
+  for (int p = 0; p < 2; ++p) {
+    L->pkt_idx[p] = take(L->K[p] * 4);
+    L->pkt_val[p] = take(L->K[p] * 4);
+  }
+  L->cand_idx = take(vec);
+  L->cand_val = take(vec);
+  L->tiles = take((uint64_t)L->num_tiles * sizeof(Tile));
+  L->segs = take(S * sizeof(SegDesc));
+  L->tile_count = take((uint64_t)L->num_tiles * 4);
+  L->tile_pre = take((uint64_t)L->num_tiles * sizeof(uint2));
+  L->cta_tot = take((uint64_t)kMaxGrid * sizeof(uint2));
+  L->hist1 = take(S * kBins1 * 4);
+  L->hist2 = take(S * kBins2 * 4);
+  L->hist3 = take(S * kBins3 * 4);
+  L->sel = take(S * sizeof(SegSel));
+  L->L_safe = take(S * 4);
+  L->L_next = take(2 * N * S * 4);
+  L->u_slots = take((N + 1) * sizeof(float*));
+  L->flags = take(kNumFlags * 4);
+  L->status = take(4);
+  L->stats = take(4 * 8);
+  L->total = off;
+}
+
+}  // namespace
+
+struct dgs_ctx {
+  uint32_t magic;
+  dgs_config cfg;
+  std::vector<dgs_segment> segments;
+  Layout lay;
+  char* base;
+  cudaStream_t stream;
+  Workspace ws;
+  float inv_m;
+  int stream_grid[3];    // CTAs of the stand-alone stream pass, per mode
+  int finalize_grid[3];  // CTAs of the cooperative finalize kernel, per mode
+  std::vector<uint8_t> seen[2];  // worker has a carried bound for [0] push, [1] pull
+  std::vector<int64_t> prev;
+  uint64_t timestamp;
+  uint64_t launches;
+  int last_cuda;
+  bool broken;
+
+  template <typename T>
+  T* at(uint64_t off) const { return reinterpret_cast<T*>(base + off); }
+  float* u_buf(uint32_t q) const { return at<float>(lay.u) + (uint64_t)q * lay.n_pad; }
+  float* D_buf(uint32_t q) const { return at<float>(lay.D) + (uint64_t)q * lay.n_pad; }
+  float* theta_local_buf(uint32_t q) const { return at<float>(lay.theta_local) + (uint64_t)q * lay.n_pad; }
+  float** u_slot(uint32_t q) const { return at<float*>(lay.u_slots) + q; }
+  uint32_t* L_next(int pm, uint32_t w) const {
+    return at<uint32_t>(lay.L_next) + ((uint64_t)pm * cfg.num_workers + w) * cfg.num_segments;
+  }
+};
+
+namespace {
+
+#define DGS_CUDA(ctx, call)                 \
+  do {                                      \
+    cudaError_t e_ = (call);                \
+    if (e_ != cudaSuccess) {                \
+      (ctx)->last_cuda = (int)e_;           \
+      (ctx)->broken = true;                 \
+      return DGS_ECUDA;                     \
+    }                                       \
+  } while (0)
+
+inline int live(dgs_ctx* c) {
+  if (!c || c->magic != kMagic) return DGS_ESTATE;
+  if (c->broken) return DGS_ESTATE;
+  return DGS_OK;
+}
+
+template <int MODE>
+int launch_select(dgs_ctx* c, const SelArgs& a_in, bool carried) {
+  SelArgs a = a_in;
+  a.speculate = (c->cfg.flags & DGS_NO_SPECULATION) ? 0 : 1;
+  const bool single_pass = a.speculate && carried;
+  a.force_two_pass = single_pass ? 0 : 1;
+  if (single_pass) {
+    k_stream<MODE><<<c->stream_grid[MODE], kThreads, 0, c->stream>>>(c->ws, a);
+    DGS_CUDA(c, cudaGetLastError());
+    c->launches += 1;
+  }
+  void* args[] = {(void*)&c->ws, (void*)&a};
+  DGS_CUDA(c, cudaLaunchCooperativeKernel((const void*)k_finalize<MODE>, dim3(c->finalize_grid[MODE]),
+                                          dim3(kThreads), args, 0, c->stream));
+  c->launches += 1;
+  return DGS_OK;
+}
+
+template <int MODE>
+int occupancy_grids(dgs_ctx* c, int sms) {
+  int occ = 0;
+  DGS_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_stream<MODE>, kThreads, 0));
+  if (occ < 1) occ = 1;
+  c->stream_grid[MODE] = sms * occ;
+  DGS_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_finalize<MODE>, kThreads, 0));
+  if (occ < 1) {
+    c->last_cuda = (int)cudaErrorCooperativeLaunchTooLarge;
+    c->broken = true;
+    return DGS_ECUDA;
+  }
+  if (occ > 2) occ = 2;
+  int g = sms * occ;
+  if (g > kMaxGrid) g = kMaxGrid;
+  c->finalize_grid[MODE] = g;
+  return DGS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* dgs_error_string(int err) {
+  switch (err) {
+    case DGS_OK: return "ok";
+    case DGS_EINVAL: return "invalid argument";
+    case DGS_ENOMEM: return "arena too small";
+    case DGS_ECUDA: return "CUDA runtime error";
+    case DGS_ETIMEOUT: return "bounded device wait expired";
+    case DGS_ESTATE: return "context freed or unusable";
+  }
+  return "unknown error";
+}
+
+int dgs_arena_bytes(const dgs_config* cfg, uint64_t* out_bytes) {
+  if (!out_bytes) return DGS_EINVAL;
+  const int rc = check_config(cfg);
+  if (rc != DGS_OK) return rc;
+  Layout L;
+  make_layout(cfg, &L);
+  *out_bytes = L.total;
+  return DGS_OK;
+}
+
+int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
+  if (!out) return DGS_EINVAL;
+  *out = nullptr;
+  int rc = check_config(cfg);
+  if (rc != DGS_OK) return rc;
+  if (!cfg->theta0 || !cfg->arena) return DGS_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(cfg->arena) % kAlign) != 0) return DGS_EINVAL;
+  dgs_ctx* c = new (std::nothrow) dgs_ctx();
+  if (!c) return DGS_ENOMEM;
+  c->magic = kMagic;
+  c->cfg = *cfg;
+  c->segments.assign(cfg->segments, cfg->segments + cfg->num_segments);
+  c->cfg.segments = c->segments.data();
+  make_layout(&c->cfg, &c->lay);
+  if (c->lay.total > cfg->arena_bytes) {
+    delete c;
+    return DGS_ENOMEM;
+  }
+  c->base = static_cast<char*>(cfg->arena);
+  c->stream = static_cast<cudaStream_t>(cfg->stream);
+  c->inv_m = 1.0f / cfg->momentum;  // one IEEE division; the kernels multiply by this constant
+  c->timestamp = 0;
+  c->launches = 0;
+  c->last_cuda = 0;
+  c->broken = false;
+  c->seen[0].assign(cfg->num_workers, 0);
+  c->seen[1].assign(cfg->num_workers, 0);
+  c->prev.assign(cfg->num_workers, -1);
+
+  auto fail = [&](int code) {
+    const int lc = c->last_cuda;
+    (void)lc;
+    c->magic = 0;
+    delete c;
+    return code;
+  };
+#define INIT_CUDA(call)                         \
+  do {                                          \
+    cudaError_t e_ = (call);                    \
+    if (e_ != cudaSuccess) return fail(DGS_ECUDA); \
+  } while (0)
+
+  int dev = 0, sms = 0, coop = 0;
+  INIT_CUDA(cudaGetDevice(&dev));
+  INIT_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  INIT_CUDA(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
+  if (!coop) return fail(DGS_ECUDA);
+  if (occupancy_grids<kPushSam>(c, sms) != DGS_OK || occupancy_grids<kPushResidual>(c, sms) != DGS_OK ||
+      occupancy_grids<kPull>(c, sms) != DGS_OK)
+    return fail(DGS_ECUDA);
+
+  const Layout& L = c->lay;
+  const uint64_t N = cfg->num_workers, vec = L.n_pad * 4;
+  std::vector<Tile> tiles;
+  std::vector<SegDesc> segs;
+  tiles.reserve(L.num_tiles);
+  build_tiles(&c->cfg, &tiles, &segs);
+  if (tiles.size() != L.num_tiles) return fail(DGS_EINVAL);
+  cudaStream_t st = c->stream;
+  // state: u = 0, D = 0 (initialisation lines of Algorithm 3 and Algorithm 2), theta = theta_0
+  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.u), 0, vec * (N + 1), st));
+  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.D), 0, vec * N, st));
+  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.theta), 0, vec, st));
+  INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.theta), cfg->theta0, cfg->n * 4, cudaMemcpyDeviceToDevice, st));
+  if (cfg->flags & DGS_KEEP_LOCAL_MODEL) {
+    INIT_CUDA(cudaMemsetAsync(c->at<char>(L.theta_local), 0, vec * N, st));
+    for (uint32_t q = 0; q < N; ++q)
+      INIT_CUDA(cudaMemcpyAsync(c->theta_local_buf(q), cfg->theta0, cfg->n * 4, cudaMemcpyDeviceToDevice, st));
+  }
+  // scratch that kernels expect to find cleared, and the static tables
+  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.hist1), 0, L.sel - L.hist1, st));
+  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.sel), 0, L.total - L.sel, st));
+  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.L_next), 0xFF, 2 * N * cfg->num_segments * 4, st));
+  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.tile_count), 0, (uint64_t)L.num_tiles * 4, st));
+  INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.tiles), tiles.data(), tiles.size() * sizeof(Tile), cudaMemcpyHostToDevice, st));
+  INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.segs), segs.data(), segs.size() * sizeof(SegDesc), cudaMemcpyHostToDevice, st));
+  std::vector<float*> slots(N + 1);
+  for (uint32_t q = 0; q <= N; ++q) slots[q] = c->u_buf(q);
+  INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.u_slots), slots.data(), slots.size() * sizeof(float*), cudaMemcpyHostToDevice, st));
+  INIT_CUDA(cudaStreamSynchronize(st));  // the host vectors above go out of scope
+#undef INIT_CUDA
+
+  Workspace& w = c->ws;
+  w.tiles = c->at<Tile>(L.tiles);
+  w.segs = c->at<SegDesc>(L.segs);
+  w.num_tiles = L.num_tiles;
+  w.num_segs = cfg->num_segments;
+  w.cand_idx = c->at<uint32_t>(L.cand_idx);
+  w.cand_val = c->at<float>(L.cand_val);
+  w.tile_count = c->at<uint32_t>(L.tile_count);
+  w.tile_pre = c->at<uint2>(L.tile_pre);
+  w.cta_tot = c->at<uint2>(L.cta_tot);
+  w.hist1 = c->at<uint32_t>(L.hist1);
+  w.hist2 = c->at<uint32_t>(L.hist2);
+  w.hist3 = c->at<uint32_t>(L.hist3);
+  w.sel = c->at<SegSel>(L.sel);
+  w.L_safe = c->at<uint32_t>(L.L_safe);
+  w.flags = c->at<uint32_t>(L.flags);
+  w.status = c->at<int>(L.status);
+  w.stats = c->at<unsigned long long>(L.stats);
+  *out = c;
+  return DGS_OK;
+}
+
+int dgs_worker_push(dgs_ctx* c, uint32_t worker, const float* grad, dgs_packet* out) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (worker >= c->cfg.num_workers || !grad) return DGS_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(grad) % 16) != 0) return DGS_EINVAL;
+  const Layout& L = c->lay;
+  SelArgs a;
+  std::memset(&a, 0, sizeof(a));
+  a.grad = grad;
+  a.u_cur_slot = c->u_slot(worker);
+  a.u_spare_slot = c->u_slot(c->cfg.num_workers);
+  a.L_next = c->L_next(0, worker);
+  a.pkt_idx = c->at<uint32_t>(L.pkt_idx[0]);
+  a.pkt_val = c->at<float>(L.pkt_val[0]);
+  a.pkt_count = (uint32_t)L.K[0];
+  a.m = c->cfg.momentum;
+  a.lr = c->cfg.lr;
+  a.inv_m = c->inv_m;
+  const bool carried = c->seen[0][worker] != 0;
+  rc = (c->cfg.flags & DGS_RESIDUAL_MODE) ? launch_select<kPushResidual>(c, a, carried)
+                                          : launch_select<kPushSam>(c, a, carried);
+  if (rc != DGS_OK) return rc;
+  c->seen[0][worker] = 1;
+  if (out) {
+    out->idx = a.pkt_idx;
+    out->val = a.pkt_val;
+    out->count = a.pkt_count;
+  }
+  return DGS_OK;
+}
+
+int dgs_server_apply(dgs_ctx* c, uint32_t worker, const dgs_packet* pkt) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (worker >= c->cfg.num_workers || !pkt) return DGS_EINVAL;
+  if (pkt->count > 0 && (!pkt->idx || !pkt->val)) return DGS_EINVAL;
+  if (pkt->count > 0) {
+    const dim3 grid((pkt->count + kThreads - 1) / kThreads, c->cfg.num_workers + 1);
+    k_scatter_sub<<<grid, kThreads, 0, c->stream>>>(pkt->idx, pkt->val, pkt->count, c->at<float>(c->lay.theta),
+                                                    c->at<float>(c->lay.D), c->lay.n_pad, c->cfg.num_workers,
+                                                    c->cfg.n, c->ws.status);
+    DGS_CUDA(c, cudaGetLastError());
+    c->launches += 1;
+  }
+  c->timestamp += 1;  // t counts updates made to the server parameters
+  return DGS_OK;
+}
+
+int dgs_worker_pull(dgs_ctx* c, uint32_t worker, dgs_packet* out) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (worker >= c->cfg.num_workers) return DGS_EINVAL;
+  const Layout& L = c->lay;
+  SelArgs a;
+  std::memset(&a, 0, sizeof(a));
+  a.D = c->D_buf(worker);
+  a.theta_local = (c->cfg.flags & DGS_KEEP_LOCAL_MODEL) ? c->theta_local_buf(worker) : nullptr;
+  a.L_next = c->L_next(1, worker);
+  a.pkt_idx = c->at<uint32_t>(L.pkt_idx[1]);
+  a.pkt_val = c->at<float>(L.pkt_val[1]);
+  a.pkt_count = (uint32_t)L.K[1];
+  a.m = c->cfg.momentum;
+  a.lr = c->cfg.lr;
+  a.inv_m = c->inv_m;
+  rc = launch_select<kPull>(c, a, c->seen[1][worker] != 0);
+  if (rc != DGS_OK) return rc;
+  c->seen[1][worker] = 1;
+  c->prev[worker] = (int64_t)c->timestamp;
+  if (out) {
+    out->idx = a.pkt_idx;
+    out->val = a.pkt_val;
+    out->count = a.pkt_count;
+  }
+  return DGS_OK;
+}
+
+int dgs_event(dgs_ctx* c, uint32_t worker, const float* grad, dgs_packet* push_out, dgs_packet* pull_out) {
+  dgs_packet p, g;
+  int rc = dgs_worker_push(c, worker, grad, &p);
+  if (rc != DGS_OK) return rc;
+  rc = dgs_server_apply(c, worker, &p);
+  if (rc != DGS_OK) return rc;
+  rc = dgs_worker_pull(c, worker, &g);
+  if (rc != DGS_OK) return rc;
+  if (push_out) *push_out = p;
+  if (pull_out) *pull_out = g;
+  return DGS_OK;
+}
+
+int dgs_event_host(dgs_ctx* c, uint32_t worker, const float* grad_host, uint32_t* out_idx, float* out_val) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (!(c->cfg.flags & DGS_HOST_IO) || !grad_host || worker >= c->cfg.num_workers) return DGS_EINVAL;
+  float* stage = c->at<float>(c->lay.grad_stage);
+  DGS_CUDA(c, cudaMemcpyAsync(stage, grad_host, c->cfg.n * 4, cudaMemcpyHostToDevice, c->stream));
+  dgs_packet g;
+  rc = dgs_event(c, worker, stage, nullptr, &g);
+  if (rc != DGS_OK) return rc;
+  if (out_idx) DGS_CUDA(c, cudaMemcpyAsync(out_idx, g.idx, (uint64_t)g.count * 4, cudaMemcpyDeviceToHost, c->stream));
+  if (out_val) DGS_CUDA(c, cudaMemcpyAsync(out_val, g.val, (uint64_t)g.count * 4, cudaMemcpyDeviceToHost, c->stream));
+  DGS_CUDA(c, cudaStreamSynchronize(c->stream));
+  return DGS_OK;
+}
+
+int dgs_state_ptr(dgs_ctx* c, int which, uint32_t worker, const float** out) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (!out) return DGS_EINVAL;
+  if (which != DGS_THETA && worker >= c->cfg.num_workers) return DGS_EINVAL;
+  switch (which) {
+    case DGS_THETA: *out = c->at<float>(c->lay.theta); break;
+    case DGS_D: *out = c->D_buf(worker); break;
+    case DGS_THETA_LOCAL:
+      if (!(c->cfg.flags & DGS_KEEP_LOCAL_MODEL)) return DGS_EINVAL;
+      *out = c->theta_local_buf(worker);
+      break;
+    case DGS_U: {
+      float* p = nullptr;
+      DGS_CUDA(c, cudaMemcpyAsync(&p, c->u_slot(worker), sizeof(p), cudaMemcpyDeviceToHost, c->stream));
+      DGS_CUDA(c, cudaStreamSynchronize(c->stream));
+      *out = p;
+      return DGS_OK;
+    }
+    default: return DGS_EINVAL;
+  }
+  DGS_CUDA(c, cudaStreamSynchronize(c->stream));
+  return DGS_OK;
+}
+
+int dgs_state_load(dgs_ctx* c, int which, uint32_t worker, const float* src) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (!src) return DGS_EINVAL;
+  const float* dst = nullptr;
+  rc = dgs_state_ptr(c, which, worker, &dst);
+  if (rc != DGS_OK) return rc;
+  DGS_CUDA(c, cudaMemcpyAsync(const_cast<float*>(dst), src, c->cfg.n * 4, cudaMemcpyDeviceToDevice, c->stream));
+  return DGS_OK;
+}
+
+int dgs_status(dgs_ctx* c, int* device_status) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (!device_status) return DGS_EINVAL;
+  DGS_CUDA(c, cudaMemcpyAsync(device_status, c->ws.status, 4, cudaMemcpyDeviceToHost, c->stream));
+  DGS_CUDA(c, cudaStreamSynchronize(c->stream));
+  return DGS_OK;
+}
+
+int dgs_stats(dgs_ctx* c, uint64_t out[4]) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (!out) return DGS_EINVAL;
+  unsigned long long s[4] = {0, 0, 0, 0};
+  DGS_CUDA(c, cudaMemcpyAsync(s, c->ws.stats, sizeof(s), cudaMemcpyDeviceToHost, c->stream));
+  DGS_CUDA(c, cudaStreamSynchronize(c->stream));
+  out[0] = s[0];
+  out[1] = s[1];
+  out[2] = c->timestamp;
+  out[3] = 0;
+  return DGS_OK;
+}
+
+int dgs_prev(dgs_ctx* c, uint32_t worker, int64_t* out) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (!out || worker >= c->cfg.num_workers) return DGS_EINVAL;
+  *out = c->prev[worker];
+  return DGS_OK;
+}
+
+int dgs_launch_count(dgs_ctx* c, uint64_t* out) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (!out) return DGS_EINVAL;
+  *out = c->launches;
+  return DGS_OK;
+}
+
+int dgs_last_cuda_error(dgs_ctx* c) {
+  if (!c || c->magic != kMagic) return 0;
+  return c->last_cuda;
+}
+
+int dgs_free(dgs_ctx* c) {
+  if (!c || c->magic != kMagic) return DGS_ESTATE;
+  cudaStreamSynchronize(c->stream);
+  c->magic = 0;
+  delete c;
+  return DGS_OK;
+}
+
+}  // extern "C"

@@ -10,6 +10,11 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu)")
+    # the CUDA library and the CPU checker are built in-tree on first use
+    from paper_1910_10929_b200 import build as _build
+    _build.build()
+    import oracle
+    oracle.build()
 
 
 def _has_gpu() -> bool:

@@ -1,0 +1,199 @@
+"""Parity of the CUDA library against the CPU checker, through the C ABI.
+
+Bar: selected index sets bit-exact (ties to the lowest index), packet values and
+apply results bit-exact, all float32 state within 1e-6 max relative error after
+the whole trajectory -- every step is one rounded IEEE operation in a fixed
+order, so the state is in fact required to be bit-identical."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1910_10929_b200 as dgs
+import workloads as W
+from _replay import bits, key, packet_to_numpy, replay_and_compare
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def select_on_gpu(x: np.ndarray, seg_sizes, ks, flags=0):
+    """Top-k per segment of a given vector via a pull on a one-worker context."""
+    n = x.shape[0]
+    off = np.concatenate([[0], np.cumsum(seg_sizes)[:-1]])
+    ctx = dgs.Context(n, 1, 0.1, 0.9, off, seg_sizes, ks, ks, torch.zeros(n, device=DEV), flags=flags)
+    ctx.state_load(dgs.DGS_D, 0, torch.from_numpy(x).to(DEV))
+    idx, val = packet_to_numpy(ctx, ctx.worker_pull(0))
+    left = ctx.state(dgs.DGS_D, 0).cpu().numpy()
+    assert ctx.status() == 0
+    return idx, val, left, ctx
+
+
+def expect_select(x, seg_sizes, ks):
+    out, base = [], 0
+    for ln, k in zip(seg_sizes, ks):
+        out.append(oracle.topk(x[base:base + ln], k) + base)
+        base += ln
+    return np.concatenate(out).astype(np.uint32)
+
+
+ADVERSARIAL = [
+    ("all_equal", np.ones(1500, np.float32), [1500], [37]),
+    ("all_zero", np.zeros(1029, np.float32), [1029], [5]),
+    ("signed_zeros", np.tile(np.array([0.0, -0.0], np.float32), 300), [600], [7]),
+    ("k_is_1", np.arange(777, dtype=np.float32) - 300, [777], [1]),
+    ("k_is_n", (np.arange(513, dtype=np.float32) - 77) / 3, [513], [513]),
+    ("one_element", np.array([-2.5], np.float32), [1], [1]),
+    ("denormals", np.concatenate([np.full(300, 1e-45, np.float32), np.zeros(300, np.float32),
+                                  np.full(5, -3e-40, np.float32)]), [605], [100]),
+    ("ties_across_tiles", np.tile(np.array([1, -1, 2, -2, 0.5], np.float32), 700), [3500], [1000]),
+    ("ragged_segments", np.sin(np.arange(2000, dtype=np.float32)), [3, 509, 1, 700, 787], [1, 100, 1, 7, 787]),
+    ("same_top_bits", (1.0 + np.arange(4096, dtype=np.float32) * 2.0 ** -20).astype(np.float32), [4096], [300]),
+]
+
+
+@pytest.mark.parametrize("name,x,segs,ks", ADVERSARIAL, ids=[c[0] for c in ADVERSARIAL])
+def test_selection_adversarial(name, x, segs, ks):
+    want = expect_select(x, segs, ks)
+    idx, val, left, _ = select_on_gpu(x, segs, ks)
+    assert np.array_equal(idx, want)
+    assert np.array_equal(bits(val), bits(x[want]))
+    # exact split: what was sent plus what stayed is the input, and the sent entries are cleared
+    back = left.copy()
+    assert not left[want].any()
+    back[want] = val
+    assert np.array_equal(bits(back), bits(x))
+
+
+@pytest.mark.parametrize("flags", [0, dgs.DGS_NO_SPECULATION, dgs.DGS_KEEP_LOCAL_MODEL, dgs.DGS_RESIDUAL_MODE,
+                                   dgs.DGS_RESIDUAL_MODE | dgs.DGS_KEEP_LOCAL_MODEL | dgs.DGS_NO_SPECULATION])
+def test_trajectory_small_ragged(flags):
+    # several tiles, ragged heads and tails, tiny layers, repeated arrivals of the same worker
+    wl = W.custom("ragged", [300, 7, 5000, 64, 1, 2049, 1531], 3, 30, 20_000, grad_kind="normal", grad_scale=1e-2)
+    ctx, _ = replay_and_compare(wl, flags=flags, compare_state_every=7)
+    single, two_pass, _, _ = ctx.stats()
+    assert single + two_pass == 2 * wl.num_events
+    if flags & dgs.DGS_NO_SPECULATION:
+        assert single == 0
+    else:
+        assert single > 0
+
+
+def test_trajectory_dense_limit_k_equals_n():
+    wl = W.custom("dense", [700, 333], 2, 8, 1_000_000, grad_kind="normal", grad_scale=1e-2)
+    assert wl.K_push == wl.n
+    replay_and_compare(wl, flags=dgs.DGS_KEEP_LOCAL_MODEL)
+
+
+def test_trajectory_pull_wants_more_than_is_nonzero():
+    # the server sends 5 % per layer while pushes deliver 0.5 %: early pulls are filled with zeros
+    wl = W.custom("zero_fill", [4000, 3000], 2, 10, 5_000, density_pull_ppm=50_000, grad_kind="laplace")
+    replay_and_compare(wl)
+
+
+def test_trajectory_momentum_one_and_half():
+    for m in (1.0, 0.5):
+        wl = W.custom("m", [3000], 2, 8, 10_000, momentum=m)
+        replay_and_compare(wl)
+
+
+def test_trajectory_flat_1m():
+    wl = W.flat_1m()
+    assert wl.K_push == 1049
+    replay_and_compare(wl, flags=dgs.DGS_KEEP_LOCAL_MODEL)
+
+
+def test_trajectory_resnet18_per_layer():
+    wl = W.resnet18(num_workers=32, num_events=40)
+    ctx, _ = replay_and_compare(wl)
+    assert ctx.stats()[0] > 0          # workers that came back took the single-pass route
+
+
+def test_trajectory_resnet50_global():
+    wl = W.resnet50(num_workers=32, num_events=36)
+    replay_and_compare(wl)
+
+
+def test_trajectory_gpt2_small_few_workers():
+    wl = W.gpt2_small(num_workers=3, num_events=7)
+    replay_and_compare(wl)
+
+
+@pytest.mark.parametrize("log2n", [16, 18, 20, 22, 24])
+@pytest.mark.parametrize("ppm", W.SWEEP_PPM)
+def test_sweep_selection(log2n, ppm):
+    n = 1 << log2n
+    x = W.sweep_values(n, index=log2n)
+    k = W.k_of(n, ppm)
+    want = expect_select(x, [n], [k])
+    idx, val, _, _ = select_on_gpu(x, [n], [k])
+    assert np.array_equal(idx, want)
+    assert np.array_equal(bits(val), bits(x[want]))
+
+
+def test_apply_foreign_packet_and_bad_index_is_reported():
+    n = 5000
+    ctx = dgs.Context(n, 2, 0.1, 0.9, [0], [n], [10], [10], torch.zeros(n, device=DEV))
+    idx = torch.tensor([1, 7, 4999], dtype=torch.int32, device=DEV)
+    val = torch.tensor([1.0, -2.0, 0.5], device=DEV)
+    pkt = dgs.dgs_packet(idx.data_ptr(), val.data_ptr(), 3)
+    ctx.server_apply(0, pkt)
+    th = ctx.state(dgs.DGS_THETA).cpu().numpy()
+    assert th[1] == -1.0 and th[7] == 2.0 and th[4999] == -0.5 and np.count_nonzero(th) == 3
+    for q in range(2):
+        assert np.array_equal(ctx.state(dgs.DGS_D, q).cpu().numpy(), th)
+    assert ctx.status() == 0
+    bad = torch.tensor([5000], dtype=torch.int32, device=DEV)   # out of range: skipped and flagged
+    ctx.server_apply(0, dgs.dgs_packet(bad.data_ptr(), val.data_ptr(), 1))
+    assert ctx.status() != 0
+    assert np.array_equal(ctx.state(dgs.DGS_THETA).cpu().numpy(), th)
+
+
+def test_argument_errors_on_a_live_context():
+    n = 4096
+    ctx = dgs.Context(n, 2, 0.1, 0.9, [0], [n], [4], [4], torch.zeros(n, device=DEV))
+    g = torch.zeros(n + 1, device=DEV)
+    L = dgs.lib()
+    import ctypes as C
+    p = dgs.dgs_packet()
+    assert L.dgs_worker_push(ctx.handle, 2, g.data_ptr(), C.byref(p)) == dgs.DGS_EINVAL   # worker out of range
+    assert L.dgs_worker_push(ctx.handle, 0, None, C.byref(p)) == dgs.DGS_EINVAL
+    assert L.dgs_worker_push(ctx.handle, 0, g.data_ptr() + 4, C.byref(p)) == dgs.DGS_EINVAL  # misaligned
+    assert L.dgs_worker_pull(ctx.handle, 5, C.byref(p)) == dgs.DGS_EINVAL
+    assert L.dgs_event_host(ctx.handle, 0, None, None, None) == dgs.DGS_EINVAL            # no DGS_HOST_IO
+    out = C.c_void_p()
+    assert L.dgs_state_ptr(ctx.handle, dgs.DGS_THETA_LOCAL, 0, C.byref(out)) == dgs.DGS_EINVAL
+    small = dgs.make_config(n, 2, 0.1, 0.9, [0], [n], [4], [4], theta0=g.data_ptr(),
+                            arena=ctx.arena.data_ptr(), arena_bytes=1024)
+    h = C.c_void_p()
+    assert L.dgs_init(C.byref(small), C.byref(h)) == dgs.DGS_ENOMEM
+
+
+def test_event_host_matches_device_path():
+    wl = W.custom("host", [70_000, 513], 2, 6, 10_000, grad_kind="laplace")
+    theta0 = torch.from_numpy(wl.theta0()).to(DEV)
+    a = dgs.Context.from_workload(wl, theta0=theta0, flags=dgs.DGS_HOST_IO)
+    b = dgs.Context.from_workload(wl, theta0=theta0)
+    idx = torch.empty(wl.K_pull, dtype=torch.int32).pin_memory()
+    val = torch.empty(wl.K_pull, dtype=torch.float32).pin_memory()
+    for e, w in enumerate(wl.schedule()):
+        g = torch.from_numpy(wl.gradient(e)).pin_memory()
+        a.event_host(int(w), g, idx, val)
+        _, pull = b.event(int(w), g.to(DEV))
+        bi, bv = packet_to_numpy(b, pull)
+        assert np.array_equal(idx.numpy().view(np.uint32), bi) and np.array_equal(bits(val.numpy()), bits(bv))
+    assert torch.equal(a.state(dgs.DGS_THETA), b.state(dgs.DGS_THETA))
+
+
+def test_two_runs_are_bit_identical():
+    wl = W.custom("det", [100_000], 3, 12, 1000)
+    outs = []
+    for _ in range(2):
+        ctx = dgs.Context.from_workload(wl)
+        for e, w in enumerate(wl.schedule()):
+            ctx.event(int(w), torch.from_numpy(wl.gradient(e)).to(DEV))
+        outs.append([ctx.state(dgs.DGS_THETA).clone()] +
+                    [ctx.state(dgs.DGS_U, q).clone() for q in range(3)] +
+                    [ctx.state(dgs.DGS_D, q).clone() for q in range(3)])
+    for x, y in zip(*outs):
+        assert torch.equal(x.view(torch.int32), y.view(torch.int32))
