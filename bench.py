@@ -1,0 +1,372 @@
+#!/usr/bin/env python
+"""Benchmark of the DGS push+apply+pull event loop.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet50] [--impl ours|reference]
+
+One "step" is one event (worker push, server apply, worker pull) of the chosen
+workload.  Default workload: ResNet-50 shapes, 25.56 M parameters, one global 0.1 %
+selection, 32 workers.  Prints ONE JSON line (rank 0).
+
+Timed region: K consecutive events with every gradient already resident in HBM,
+CUDA events on the library's stream, barrier + synchronize on both sides, max over
+ranks.  Before the W warm-up events an untimed pre-roll serves every worker once,
+so that the timed events are steady-state ones (a worker's first arrival takes the
+two-pass selection route).  Each event reads a different gradient, velocity and
+difference vector (3 x 102 MB at the default workload, more than the L2), so no
+L2 flush is needed between iterations.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as W  # noqa: E402
+
+METRIC = "push+apply+pull events/sec"
+UNIT = "events/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def make_workload(name: str, seed: int):
+    if name not in W.BY_NAME:
+        raise SystemExit(f"unknown workload {name}; choose from {sorted(W.BY_NAME)}")
+    return W.BY_NAME[name](seed=seed)
+
+
+def algorithmic_bytes_per_event(n: int, K_push: int, K_pull: int, N: int) -> dict:
+    """What the method itself must move per event (no scratch traffic counted).
+    push: read u and grad, write u', write the packet.  apply: read the packet once,
+    read+write one float per (entry, buffer) for theta and the N difference vectors.
+    pull: read D_w, write the packet, clear the sent entries."""
+    push = 12 * n + 8 * K_push
+    apply_ = 8 * K_push * (N + 1) + 8 * K_push
+    pull = 4 * n + 8 * K_pull + 4 * K_pull
+    return {"push": push, "apply": apply_, "pull": pull, "total": push + apply_ + pull}
+
+
+def hbm_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Polls nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+            self.thread.join(timeout=2)
+
+    def summary(self) -> dict:
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, cell in zip(names, r[4:8]):
+                if cell.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def generate_gradients(wl, events, out_tensors) -> None:
+    """Fills out_tensors[i] (pinned host float32[n]) with the gradient of events[i], in parallel."""
+    def one(i):
+        wl.gradient(int(events[i]), out=out_tensors[i].numpy())
+    wl._scales() if wl.grad_kind == "laplace" else None
+    with ThreadPoolExecutor(max_workers=min(32, os.cpu_count() or 1)) as ex:
+        list(ex.map(one, range(len(events))))
+
+
+def run_reference(args, wl) -> dict:
+    """The CPU checker, as it stands, on the host cores: one step = one full event."""
+    import oracle
+    sched = wl.schedule()
+    K, Wm = args.steps, args.warmup
+    o = oracle.Oracle.from_workload(wl)
+    # keep the whole run within a few minutes: estimate from the first warm-up event
+    budget_s = 240.0
+    done, t_first = 0, None
+    for e in range(Wm):
+        t0 = time.perf_counter()
+        o.event(int(sched[e % len(sched)]), wl.gradient(e))
+        t_first = time.perf_counter() - t0 if t_first is None else t_first
+    if t_first is None:
+        t0 = time.perf_counter()
+        o.event(int(sched[0]), wl.gradient(0))
+        t_first = time.perf_counter() - t0
+        Wm_eff = 1
+    else:
+        Wm_eff = Wm
+    K_eff = max(1, min(K, int(budget_s / max(t_first, 1e-6))))
+    grads = None
+    elapsed = 0.0
+    for i in range(K_eff):
+        e = Wm_eff + i
+        g = wl.gradient(e)                      # input generation is outside the timed region
+        t0 = time.perf_counter()
+        o.event(int(sched[e % len(sched)]), g)
+        elapsed += time.perf_counter() - t0
+        done += 1
+    value = done / elapsed
+    sample = (f"{done} consecutive events of the full {wl.name} workload (n={wl.n}, {wl.num_workers} workers) "
+              f"after {Wm_eff} untimed ones")
+    return {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": done, "warmup": Wm_eff, "ms_per_step": 1e3 * elapsed / done, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "n": wl.n, "workers": wl.num_workers, "K_push": wl.K_push,
+                   "K_pull": wl.K_pull, "seed": wl.seed},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+
+
+def cpu_baseline(wl, seconds: float = 20.0) -> dict:
+    import oracle
+    sched = wl.schedule()
+    o = oracle.Oracle.from_workload(wl)
+    elapsed, done, e = 0.0, 0, 0
+    while elapsed < seconds and e < len(sched) and done < 64:
+        g = wl.gradient(e)
+        t0 = time.perf_counter()
+        o.event(int(sched[e]), g)
+        elapsed += time.perf_counter() - t0
+        done += 1
+        e += 1
+    return {"value": done / elapsed, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"first {done} events of {wl.name} (n={wl.n}, {wl.num_workers} workers), "
+                      f"{elapsed:.1f} s of single-thread CPU time on a {os.cpu_count()}-core host"}
+
+
+def reduce_max_time(elapsed_s: float, events: int, dist) -> tuple:
+    """Max of the elapsed time over ranks and the sum of the events all ranks served."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return elapsed_s, events
+    import torch
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([elapsed_s], dtype=torch.float64, device=dev)
+    c = torch.tensor([events], dtype=torch.int64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(c.item())
+
+
+def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
+    import torch
+
+    import paper_1910_10929_b200 as dgs
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    N = wl.num_workers
+    sched_full = wl.schedule()
+    preroll = N if wl.schedule_kind == "cyclic" else 2 * N
+    K, Wm = args.steps, args.warmup
+    total_events = preroll + Wm + 2 * K          # timed pass + per-kernel timing pass
+    pool = min(total_events, args.grad_pool)
+    sched = np.resize(sched_full, total_events)
+
+    # gradients: generated on the host (same generator the CPU checker is fed from), resident in HBM
+    host = [torch.empty(wl.n, dtype=torch.float32).pin_memory() for _ in range(min(pool, 16))]
+    grads = []
+    for base in range(0, pool, len(host)):
+        ids = list(range(base, min(pool, base + len(host))))
+        generate_gradients(wl, ids, host[:len(ids)])
+        for j in range(len(ids)):
+            grads.append(host[j].to(dev, non_blocking=False))
+    theta0 = torch.from_numpy(wl.theta0()).to(dev)
+    ctx = dgs.Context.from_workload(wl, theta0=theta0, flags=dgs.DGS_HOST_IO)
+    stream = ctx.stream
+
+    def run_events(first: int, count: int) -> None:
+        for e in range(first, first + count):
+            ctx.event(int(sched[e]), grads[e % pool])
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if dist is not None and world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    run_events(0, preroll)
+    run_events(preroll, Wm)
+    stats0 = ctx.stats()
+    launches0 = ctx.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with ClockSampler(local_rank) as clocks:
+        ev0.record(stream)
+        run_events(preroll + Wm, K)
+        ev1.record(stream)
+        barrier()
+    elapsed = ev0.elapsed_time(ev1) * 1e-3
+    launches = ctx.launch_count() - launches0
+    stats1 = ctx.stats()
+    assert ctx.status() == 0, "device status word is not clean"
+    elapsed_max, events_all = reduce_max_time(elapsed, K, dist)
+
+    # per-kernel device time, same loop continued, events around each launch
+    dgs.dgs_timing_enable(ctx.handle, True)
+    run_events(preroll + Wm + K, K)
+    ktimes = dgs.dgs_timing_read(ctx.handle)
+    dgs.dgs_timing_enable(ctx.handle, False)
+
+    # end to end: host gradient in, pull packet out, every step
+    Ke = min(K, len(host), 16)
+    out_idx = torch.empty(wl.K_pull, dtype=torch.int32).pin_memory()
+    out_val = torch.empty(wl.K_pull, dtype=torch.float32).pin_memory()
+    first = preroll + Wm + 2 * K
+    sched_e = np.resize(sched_full, first + Ke + 3)
+    for j in range(3):
+        ctx.event_host(int(sched_e[first + j]), host[j % len(host)], out_idx, out_val)
+    barrier()
+    t0 = time.perf_counter()
+    for j in range(Ke):
+        ctx.event_host(int(sched_e[first + 3 + j]), host[j], out_idx, out_val)
+    torch.cuda.synchronize(dev)
+    e2e_elapsed = time.perf_counter() - t0
+    e2e_max, e2e_events = reduce_max_time(e2e_elapsed, Ke, dist)
+
+    if rank != 0:
+        return {}
+    ab = algorithmic_bytes_per_event(wl.n, wl.K_push, wl.K_pull, N)
+    peak, peak_kind = hbm_peak()
+    value = events_all / elapsed_max
+    eff_gbs = value / world * ab["total"] / 1e9
+    # dominant kernel = the one with the largest share of device time
+    tot_ms = sum(ms for ms, _ in ktimes.values()) or 1.0
+    dom = max(ktimes, key=lambda k: ktimes[k][0])
+    dom_ms, dom_cnt = ktimes[dom]
+    kernel_bytes = {
+        "stream_push": 12 * wl.n, "finalize_push": 8 * wl.K_push, "two_pass_push": 20 * wl.n,
+        "scatter": ab["apply"], "stream_pull": 4 * wl.n, "finalize_pull": 12 * wl.K_pull,
+        "two_pass_pull": 8 * wl.n,
+    }
+    achieved = kernel_bytes[dom] / (dom_ms * 1e-3 / max(dom_cnt, 1)) / 1e9
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": 1e3 * elapsed_max / K, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "n": wl.n, "workers": N, "K_push": wl.K_push, "K_pull": wl.K_pull,
+                   "segments": wl.num_segments, "lr": wl.lr, "momentum": wl.momentum, "seed": wl.seed,
+                   "preroll_events": preroll, "distinct_gradients": pool,
+                   "l2": "inputs larger than L2: every event reads a different gradient, velocity and "
+                         "difference vector", "replicas": world},
+        "effective_hbm": {"algorithmic_bytes_per_event": ab, "GB/s": eff_gbs,
+                          "frac_of_nominal_8TBs": eff_gbs / NOMINAL_HBM_GBS, "frac_of_peak": eff_gbs / peak,
+                          "peak_GB/s": peak, "peak_kind": peak_kind},
+        "selection_routes": {"single_pass": stats1[0] - stats0[0], "two_pass": stats1[1] - stats0[1]},
+        "kernels": {k: {"ms_total": ms, "launches": c, "us_per_launch": (1e3 * ms / c if c else None),
+                        "share": ms / tot_ms,
+                        "GB/s": (kernel_bytes[k] / (ms * 1e-3 / c) / 1e9 if c and ms > 0 else None)}
+                    for k, (ms, c) in ktimes.items()},
+        "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_kind": peak_kind, "traffic": args.traffic_bytes,
+                     "algorithmic_bytes_per_launch": kernel_bytes[dom]},
+        "e2e": {"value": e2e_events / e2e_max, "unit": UNIT, "steps": Ke, "h2d_bytes_per_step": 4 * wl.n,
+                "d2h_bytes_per_step": 8 * wl.K_pull},
+        "gpu_launches": launches,
+        "clocks": clocks.summary(),
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(wl, args.cpu_seconds)
+    return out
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=128)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet50", choices=sorted(W.BY_NAME))
+    ap.add_argument("--seed", type=int, default=W.DEFAULT_SEED)
+    ap.add_argument("--grad-pool", type=int, default=192, help="distinct gradients kept in HBM (reused cyclically)")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--traffic-bytes", type=float, default=None,
+                    help="ncu dram bytes per launch of the dominant kernel, copied from profiles/")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            print(json.dumps(run_reference(args, make_workload(args.workload, args.seed))), flush=True)
+        return
+
+    dist = None
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    # replicas only: the path has no exchange step, every rank runs its own workers and server
+    wl = make_workload(args.workload, args.seed + rank)
+    out = run_ours(args, wl, rank, world, local_rank, dist)
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

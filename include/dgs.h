@@ -162,6 +162,28 @@ int dgs_prev(dgs_ctx* ctx, uint32_t worker, int64_t* out);
 /* Number of kernels this context has launched so far (host-side count). */
 int dgs_launch_count(dgs_ctx* ctx, uint64_t* out);
 
+/* Kernels the library launches, as indices into the arrays of dgs_timing_read. */
+enum {
+  DGS_KERNEL_STREAM_PUSH = 0,   /* push, single-pass route: velocity update + candidate collection      */
+  DGS_KERNEL_FINALIZE_PUSH = 1, /* push, single-pass route: exact k-th key, ordered packet, fix-ups      */
+  DGS_KERNEL_TWO_PASS_PUSH = 2, /* push, two-pass route: histogram pass + stream pass + finalize, fused  */
+  DGS_KERNEL_SCATTER = 3,       /* apply                                                                 */
+  DGS_KERNEL_STREAM_PULL = 4,
+  DGS_KERNEL_FINALIZE_PULL = 5,
+  DGS_KERNEL_TWO_PASS_PULL = 6,
+  DGS_NUM_KERNELS = 7
+};
+
+/* Measurement aid (no counterpart in the paper).  While on, every kernel launch of
+ * this context is bracketed by two CUDA events on the context's stream (at most
+ * 65536 launches between two reads are recorded). */
+int dgs_timing_enable(dgs_ctx* ctx, int on);
+
+/* Waits for the stream; ms[i] / count[i] receive the summed device time in
+ * milliseconds and the number of recorded launches of kernel i since the last
+ * read, and the accumulators restart from zero. */
+int dgs_timing_read(dgs_ctx* ctx, double ms[DGS_NUM_KERNELS], uint64_t count[DGS_NUM_KERNELS]);
+
 /* The cudaError_t of the last failed runtime call of this context (0 if none). */
 int dgs_last_cuda_error(dgs_ctx* ctx);
 

@@ -23,7 +23,11 @@ EXPORTS = (
     "dgs_arena_bytes", "dgs_init", "dgs_worker_push", "dgs_server_apply", "dgs_worker_pull",
     "dgs_event", "dgs_event_host", "dgs_state_ptr", "dgs_state_load", "dgs_status", "dgs_stats",
     "dgs_prev", "dgs_launch_count", "dgs_last_cuda_error", "dgs_free", "dgs_error_string",
+    "dgs_timing_enable", "dgs_timing_read",
 )
+DGS_NUM_KERNELS = 7
+KERNEL_NAMES = ("stream_push", "finalize_push", "two_pass_push", "scatter", "stream_pull", "finalize_pull",
+                "two_pass_pull")
 
 
 class dgs_segment(C.Structure):
@@ -72,6 +76,8 @@ def lib() -> C.CDLL:
         L.dgs_prev.argtypes = [vp, u32, C.POINTER(C.c_int64)]
         L.dgs_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
         L.dgs_last_cuda_error.argtypes = [vp]
+        L.dgs_timing_enable.argtypes = [vp, i32]
+        L.dgs_timing_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
         L.dgs_free.argtypes = [vp]
         L.dgs_error_string.argtypes = [i32]
         L.dgs_error_string.restype = C.c_char_p
@@ -172,6 +178,18 @@ def dgs_launch_count(ctx: int) -> int:
     out = C.c_uint64(0)
     _check(lib().dgs_launch_count(ctx, C.byref(out)), "dgs_launch_count")
     return int(out.value)
+
+
+def dgs_timing_enable(ctx: int, on: bool) -> None:
+    _check(lib().dgs_timing_enable(ctx, int(bool(on))), "dgs_timing_enable")
+
+
+def dgs_timing_read(ctx: int):
+    """{kernel name: (milliseconds, launches)} since the last read."""
+    ms = (C.c_double * DGS_NUM_KERNELS)()
+    cnt = (C.c_uint64 * DGS_NUM_KERNELS)()
+    _check(lib().dgs_timing_read(ctx, ms, cnt), "dgs_timing_read")
+    return {KERNEL_NAMES[i]: (float(ms[i]), int(cnt[i])) for i in range(DGS_NUM_KERNELS)}
 
 
 def dgs_free(ctx: int) -> None:

@@ -155,6 +155,12 @@ struct dgs_ctx {
   uint64_t launches;
   int last_cuda;
   bool broken;
+  // optional per-kernel timing (CUDA events on the context's stream)
+  bool timing;
+  std::vector<cudaEvent_t> ev_pool;   // pairs: [2i] start, [2i+1] stop
+  std::vector<int> ev_kernel;         // kernel id of each recorded pair
+  double time_ms[DGS_NUM_KERNELS];
+  uint64_t time_count[DGS_NUM_KERNELS];
 
   template <typename T>
   T* at(uint64_t off) const { return reinterpret_cast<T*>(base + off); }
@@ -185,6 +191,29 @@ inline int live(dgs_ctx* c) {
   return DGS_OK;
 }
 
+constexpr size_t kMaxTimedLaunches = 1 << 16;
+
+// Records an event before and after one launch when timing is on.
+struct TimedLaunch {
+  dgs_ctx* c;
+  cudaEvent_t stop = nullptr;
+  TimedLaunch(dgs_ctx* ctx, int kernel_id) : c(ctx) {
+    if (!c->timing || c->ev_kernel.size() >= kMaxTimedLaunches) return;
+    const size_t i = c->ev_kernel.size();
+    while (c->ev_pool.size() < 2 * (i + 1)) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) return;
+      c->ev_pool.push_back(e);
+    }
+    if (cudaEventRecord(c->ev_pool[2 * i], c->stream) != cudaSuccess) return;
+    stop = c->ev_pool[2 * i + 1];
+    c->ev_kernel.push_back(kernel_id);
+  }
+  ~TimedLaunch() {
+    if (stop) cudaEventRecord(stop, c->stream);
+  }
+};
+
 template <int MODE>
 int launch_select(dgs_ctx* c, const SelArgs& a_in, bool carried) {
   SelArgs a = a_in;
@@ -192,14 +221,19 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, bool carried) {
   const bool single_pass = a.speculate && carried;
   a.force_two_pass = single_pass ? 0 : 1;
   if (single_pass) {
+    TimedLaunch t(c, MODE == kPull ? DGS_KERNEL_STREAM_PULL : DGS_KERNEL_STREAM_PUSH);
     k_stream<MODE><<<c->stream_grid[MODE], kThreads, 0, c->stream>>>(c->ws, a);
     DGS_CUDA(c, cudaGetLastError());
     c->launches += 1;
   }
-  void* args[] = {(void*)&c->ws, (void*)&a};
-  DGS_CUDA(c, cudaLaunchCooperativeKernel((const void*)k_finalize<MODE>, dim3(c->finalize_grid[MODE]),
-                                          dim3(kThreads), args, 0, c->stream));
-  c->launches += 1;
+  {
+    TimedLaunch t(c, MODE == kPull ? (single_pass ? DGS_KERNEL_FINALIZE_PULL : DGS_KERNEL_TWO_PASS_PULL)
+                                   : (single_pass ? DGS_KERNEL_FINALIZE_PUSH : DGS_KERNEL_TWO_PASS_PUSH));
+    void* args[] = {(void*)&c->ws, (void*)&a};
+    DGS_CUDA(c, cudaLaunchCooperativeKernel((const void*)k_finalize<MODE>, dim3(c->finalize_grid[MODE]),
+                                            dim3(kThreads), args, 0, c->stream));
+    c->launches += 1;
+  }
   return DGS_OK;
 }
 
@@ -273,6 +307,11 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   c->launches = 0;
   c->last_cuda = 0;
   c->broken = false;
+  c->timing = false;
+  for (int i = 0; i < DGS_NUM_KERNELS; ++i) {
+    c->time_ms[i] = 0.0;
+    c->time_count[i] = 0;
+  }
   c->seen[0].assign(cfg->num_workers, 0);
   c->seen[1].assign(cfg->num_workers, 0);
   c->prev.assign(cfg->num_workers, -1);
@@ -390,6 +429,7 @@ int dgs_server_apply(dgs_ctx* c, uint32_t worker, const dgs_packet* pkt) {
   if (pkt->count > 0 && (!pkt->idx || !pkt->val)) return DGS_EINVAL;
   if (pkt->count > 0) {
     const dim3 grid((pkt->count + kThreads - 1) / kThreads, c->cfg.num_workers + 1);
+    TimedLaunch t(c, DGS_KERNEL_SCATTER);
     k_scatter_sub<<<grid, kThreads, 0, c->stream>>>(pkt->idx, pkt->val, pkt->count, c->at<float>(c->lay.theta),
                                                     c->at<float>(c->lay.D), c->lay.n_pad, c->cfg.num_workers,
                                                     c->cfg.n, c->ws.status);
@@ -531,6 +571,34 @@ int dgs_launch_count(dgs_ctx* c, uint64_t* out) {
   return DGS_OK;
 }
 
+int dgs_timing_enable(dgs_ctx* c, int on) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  c->timing = on != 0;
+  return DGS_OK;
+}
+
+int dgs_timing_read(dgs_ctx* c, double ms[DGS_NUM_KERNELS], uint64_t count[DGS_NUM_KERNELS]) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (!ms || !count) return DGS_EINVAL;
+  DGS_CUDA(c, cudaStreamSynchronize(c->stream));
+  for (size_t i = 0; i < c->ev_kernel.size(); ++i) {
+    float t = 0.f;
+    DGS_CUDA(c, cudaEventElapsedTime(&t, c->ev_pool[2 * i], c->ev_pool[2 * i + 1]));
+    c->time_ms[c->ev_kernel[i]] += t;
+    c->time_count[c->ev_kernel[i]] += 1;
+  }
+  c->ev_kernel.clear();
+  for (int i = 0; i < DGS_NUM_KERNELS; ++i) {
+    ms[i] = c->time_ms[i];
+    count[i] = c->time_count[i];
+    c->time_ms[i] = 0.0;
+    c->time_count[i] = 0;
+  }
+  return DGS_OK;
+}
+
 int dgs_last_cuda_error(dgs_ctx* c) {
   if (!c || c->magic != kMagic) return 0;
   return c->last_cuda;
@@ -539,6 +607,7 @@ int dgs_last_cuda_error(dgs_ctx* c) {
 int dgs_free(dgs_ctx* c) {
   if (!c || c->magic != kMagic) return DGS_ESTATE;
   cudaStreamSynchronize(c->stream);
+  for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   c->magic = 0;
   delete c;
   return DGS_OK;
