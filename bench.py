@@ -41,9 +41,11 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
 
-def make_workload(name: str, seed: int):
+def make_workload(name: str, seed: int, workers: int = 0):
     if name not in W.BY_NAME:
         raise SystemExit(f"unknown workload {name}; choose from {sorted(W.BY_NAME)}")
+    if workers:
+        return W.BY_NAME[name](seed=seed, num_workers=workers)
     return W.BY_NAME[name](seed=seed)
 
 
@@ -309,7 +311,8 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
         "effective_hbm": {"algorithmic_bytes_per_event": ab, "GB/s": eff_gbs,
                           "frac_of_nominal_8TBs": eff_gbs / NOMINAL_HBM_GBS, "frac_of_peak": eff_gbs / peak,
                           "peak_GB/s": peak, "peak_kind": peak_kind},
-        "selection_routes": {"single_pass": stats1[0] - stats0[0], "two_pass": stats1[1] - stats0[1]},
+        "selection_routes": {"single_pass": stats1[0] - stats0[0], "two_pass": stats1[1] - stats0[1],
+                             "candidates_per_selection": (stats1[3] - stats0[3]) / max(1, 2 * K)},
         "kernels": {k: {"ms_total": ms, "launches": c, "us_per_launch": (1e3 * ms / c if c else None),
                         "share": ms / tot_ms,
                         "GB/s": (kernel_bytes[k] / (ms * 1e-3 / c) / 1e9 if c and ms > 0 else None)}
@@ -336,6 +339,8 @@ def main() -> None:
     ap.add_argument("--workload", default="resnet50", choices=sorted(W.BY_NAME))
     ap.add_argument("--seed", type=int, default=W.DEFAULT_SEED)
     ap.add_argument("--grad-pool", type=int, default=192, help="distinct gradients kept in HBM (reused cyclically)")
+    ap.add_argument("--workers", type=int, default=0,
+                    help="override the number of simulated workers (smaller state for profiler captures)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--traffic-bytes", type=float, default=None,
@@ -349,7 +354,7 @@ def main() -> None:
 
     if args.impl == "reference":
         if rank == 0:
-            print(json.dumps(run_reference(args, make_workload(args.workload, args.seed))), flush=True)
+            print(json.dumps(run_reference(args, make_workload(args.workload, args.seed, args.workers))), flush=True)
         return
 
     dist = None
@@ -359,7 +364,7 @@ def main() -> None:
         torch.cuda.set_device(local_rank)
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     # replicas only: the path has no exchange step, every rank runs its own workers and server
-    wl = make_workload(args.workload, args.seed + rank)
+    wl = make_workload(args.workload, args.seed + rank, args.workers)
     out = run_ours(args, wl, rank, world, local_rank, dist)
     if rank == 0:
         print(json.dumps(out), flush=True)

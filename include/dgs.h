@@ -153,7 +153,8 @@ int dgs_status(dgs_ctx* ctx, int* device_status);
 
 /* Waits for the stream and reports counters: out[0] selections served by the
  * single-pass (speculative) route, out[1] selections that took the two-pass
- * route, out[2] server timestamp t (packets applied), out[3] reserved. */
+ * route, out[2] server timestamp t (packets applied), out[3] candidates the finalize
+ * steps have examined in total (the k selected ones included). */
 int dgs_stats(dgs_ctx* ctx, uint64_t out[4]);
 
 /* prev(worker): the server timestamp at that worker's last pull, -1 before it. */
@@ -166,7 +167,7 @@ int dgs_launch_count(dgs_ctx* ctx, uint64_t* out);
 enum {
   DGS_KERNEL_STREAM_PUSH = 0,   /* push, single-pass route: velocity update + candidate collection      */
   DGS_KERNEL_FINALIZE_PUSH = 1, /* push, single-pass route: exact k-th key, ordered packet, fix-ups      */
-  DGS_KERNEL_TWO_PASS_PUSH = 2, /* push, two-pass route: histogram pass + stream pass + finalize, fused  */
+  DGS_KERNEL_TWO_PASS_PUSH = 2, /* push, two-pass route only: histogram of the whole input + bound pick  */
   DGS_KERNEL_SCATTER = 3,       /* apply                                                                 */
   DGS_KERNEL_STREAM_PULL = 4,
   DGS_KERNEL_FINALIZE_PULL = 5,

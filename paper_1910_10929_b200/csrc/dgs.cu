@@ -2,6 +2,7 @@
 // the caller's arena, and the kernel launches of one push / apply / pull event.
 #include "dgs.h"
 
+#include <algorithm>
 #include <cmath>
 #include <cstring>
 #include <new>
@@ -25,8 +26,8 @@ struct Layout {
   uint64_t K[2] = {0, 0};
   // byte offsets into the arena
   uint64_t theta, u, D, theta_local, grad_stage, pkt_idx[2], pkt_val[2];
-  uint64_t cand_idx, cand_val, tiles, segs, tile_count, tile_pre, cta_tot;
-  uint64_t hist1, hist2, hist3, sel, L_safe, L_next, u_slots, flags, status, stats;
+  uint64_t cand_idx, cand_val, tiles, segs, part_cands, part_slot0, seg_off, seg_tile0, tile_pre, cta_tot, tile_sel;
+  uint64_t hist1, hist2, hist3, sel, L_safe, L_next, u_slots, sync, status, stats;
   uint64_t total = 0;
 };
 
@@ -120,9 +121,13 @@ void make_layout(const dgs_config* c, Layout* L) {
   L->cand_val = take(vec);
   L->tiles = take((uint64_t)L->num_tiles * sizeof(Tile));
   L->segs = take(S * sizeof(SegDesc));
-  L->tile_count = take((uint64_t)L->num_tiles * 4);
+  L->part_cands = take((uint64_t)kMaxGrid * 4);
+  L->part_slot0 = take((uint64_t)kMaxGrid * 4);
+  L->seg_off = take((S + 1) * 4);
+  L->seg_tile0 = take(S * 4);
   L->tile_pre = take((uint64_t)L->num_tiles * sizeof(uint2));
-  L->cta_tot = take((uint64_t)kMaxGrid * sizeof(uint2));
+  L->cta_tot = take((uint64_t)kMaxWorkers * sizeof(uint2));
+  L->tile_sel = take((uint64_t)L->num_tiles * sizeof(uint2));
   L->hist1 = take(S * kBins1 * 4);
   L->hist2 = take(S * kBins2 * 4);
   L->hist3 = take(S * kBins3 * 4);
@@ -130,9 +135,9 @@ void make_layout(const dgs_config* c, Layout* L) {
   L->L_safe = take(S * 4);
   L->L_next = take(2 * N * S * 4);
   L->u_slots = take((N + 1) * sizeof(float*));
-  L->flags = take(kNumFlags * 4);
+  L->sync = take(kNumSyncWords * 4);
   L->status = take(4);
-  L->stats = take(4 * 8);
+  L->stats = take(32 * 8);
   L->total = off;
 }
 
@@ -149,7 +154,15 @@ struct dgs_ctx {
   float inv_m;
   int stream_grid[3];    // CTAs of the stand-alone stream pass, per mode
   int finalize_grid[3];  // CTAs of the cooperative finalize kernel, per mode
-  std::vector<uint8_t> seen[2];  // worker has a carried bound for [0] push, [1] pull
+  uint32_t select_seq;   // selections launched so far (tags the decision word of each finalize launch)
+  // Carried bounds: row (kind, worker) of L_next holds the bounds suggested by that worker's
+  // latest selection of that kind ([0] push, [1] pull).  row_age says in which state it was
+  // made: pushes the worker had done before (push), packets accumulated in D_w since its
+  // previous pull (pull).  Thresholds grow with that age, so a row made at an age no larger
+  // than the current one is a safe-side guess; the most recent such row is used.
+  std::vector<uint8_t> row_valid[2];
+  std::vector<uint64_t> row_time[2], row_age[2];
+  std::vector<uint64_t> pushes;  // pushes done per worker
   std::vector<int64_t> prev;
   uint64_t timestamp;
   uint64_t launches;
@@ -192,6 +205,7 @@ inline int live(dgs_ctx* c) {
 }
 
 constexpr size_t kMaxTimedLaunches = 1 << 16;
+constexpr int kFinalizeWorkers = 64;  // CTAs of the finalize kernel
 
 // Records an event before and after one launch when timing is on.
 struct TimedLaunch {
@@ -214,25 +228,58 @@ struct TimedLaunch {
   }
 };
 
+// Most recent row of this kind made at an age <= `age`; -1 if there is none.
+int pick_row(const dgs_ctx* c, int kind, uint64_t age) {
+  int best = -1;
+  for (uint32_t q = 0; q < c->cfg.num_workers; ++q) {
+    if (!c->row_valid[kind][q] || c->row_age[kind][q] > age) continue;
+    if (best < 0 || c->row_time[kind][q] > c->row_time[kind][best]) best = (int)q;
+  }
+  return best;
+}
+
 template <int MODE>
-int launch_select(dgs_ctx* c, const SelArgs& a_in, bool carried) {
+int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age) {
+  constexpr int KIND = MODE == kPull ? 1 : 0;
   SelArgs a = a_in;
   a.speculate = (c->cfg.flags & DGS_NO_SPECULATION) ? 0 : 1;
-  const bool single_pass = a.speculate && carried;
+  const int row = a.speculate ? pick_row(c, KIND, age) : -1;
+  const bool single_pass = row >= 0;
+  a.L_next = c->L_next(KIND, worker);
   a.force_two_pass = single_pass ? 0 : 1;
+  a.workers = (uint32_t)c->finalize_grid[MODE];
+  a.seq = ++c->select_seq;
   if (single_pass) {
+    a.L_in = c->L_next(KIND, (uint32_t)row);
+  } else {
+    // nothing to go by: histogram of the whole input first, its bounds cannot fail
+    a.L_in = c->ws.L_safe;
+    TimedLaunch t(c, MODE == kPull ? DGS_KERNEL_TWO_PASS_PULL : DGS_KERNEL_TWO_PASS_PUSH);
+    k_hist_all<MODE><<<c->stream_grid[MODE], kThreads, 0, c->stream>>>(c->ws, a);
+    DGS_CUDA(c, cudaGetLastError());
+    const int pick_grid = (int)std::min<uint32_t>(c->cfg.num_segments, 1024u);
+    k_pick_lower<MODE><<<pick_grid, kThreads, 0, c->stream>>>(c->ws);
+    DGS_CUDA(c, cudaGetLastError());
+    c->launches += 2;
+  }
+  {
     TimedLaunch t(c, MODE == kPull ? DGS_KERNEL_STREAM_PULL : DGS_KERNEL_STREAM_PUSH);
     k_stream<MODE><<<c->stream_grid[MODE], kThreads, 0, c->stream>>>(c->ws, a);
     DGS_CUDA(c, cudaGetLastError());
     c->launches += 1;
   }
   {
-    TimedLaunch t(c, MODE == kPull ? (single_pass ? DGS_KERNEL_FINALIZE_PULL : DGS_KERNEL_TWO_PASS_PULL)
-                                   : (single_pass ? DGS_KERNEL_FINALIZE_PUSH : DGS_KERNEL_TWO_PASS_PUSH));
+    // cooperative launch: the CTAs synchronise among themselves, so all must be resident
+    TimedLaunch t(c, MODE == kPull ? DGS_KERNEL_FINALIZE_PULL : DGS_KERNEL_FINALIZE_PUSH);
     void* args[] = {(void*)&c->ws, (void*)&a};
     DGS_CUDA(c, cudaLaunchCooperativeKernel((const void*)k_finalize<MODE>, dim3(c->finalize_grid[MODE]),
                                             dim3(kThreads), args, 0, c->stream));
     c->launches += 1;
+  }
+  if (a.speculate) {
+    c->row_valid[KIND][worker] = 1;
+    c->row_time[KIND][worker] = c->select_seq;
+    c->row_age[KIND][worker] = age;
   }
   return DGS_OK;
 }
@@ -242,17 +289,14 @@ int occupancy_grids(dgs_ctx* c, int sms) {
   int occ = 0;
   DGS_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_stream<MODE>, kThreads, 0));
   if (occ < 1) occ = 1;
-  c->stream_grid[MODE] = sms * occ;
+  c->stream_grid[MODE] = std::min(sms * occ, kMaxGrid);
   DGS_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_finalize<MODE>, kThreads, 0));
   if (occ < 1) {
     c->last_cuda = (int)cudaErrorCooperativeLaunchTooLarge;
     c->broken = true;
     return DGS_ECUDA;
   }
-  if (occ > 2) occ = 2;
-  int g = sms * occ;
-  if (g > kMaxGrid) g = kMaxGrid;
-  c->finalize_grid[MODE] = g;
+  c->finalize_grid[MODE] = std::min(std::min(sms * occ, kMaxWorkers), kFinalizeWorkers);
   return DGS_OK;
 }
 
@@ -304,6 +348,7 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   c->stream = static_cast<cudaStream_t>(cfg->stream);
   c->inv_m = 1.0f / cfg->momentum;  // one IEEE division; the kernels multiply by this constant
   c->timestamp = 0;
+  c->select_seq = 0;
   c->launches = 0;
   c->last_cuda = 0;
   c->broken = false;
@@ -312,8 +357,12 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
     c->time_ms[i] = 0.0;
     c->time_count[i] = 0;
   }
-  c->seen[0].assign(cfg->num_workers, 0);
-  c->seen[1].assign(cfg->num_workers, 0);
+  for (int k = 0; k < 2; ++k) {
+    c->row_valid[k].assign(cfg->num_workers, 0);
+    c->row_time[k].assign(cfg->num_workers, 0);
+    c->row_age[k].assign(cfg->num_workers, 0);
+  }
+  c->pushes.assign(cfg->num_workers, 0);
   c->prev.assign(cfg->num_workers, -1);
 
   auto fail = [&](int code) {
@@ -357,12 +406,20 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
       INIT_CUDA(cudaMemcpyAsync(c->theta_local_buf(q), cfg->theta0, cfg->n * 4, cudaMemcpyDeviceToDevice, st));
   }
   // scratch that kernels expect to find cleared, and the static tables
-  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.hist1), 0, L.sel - L.hist1, st));
+  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.tile_sel), 0, L.sel - L.tile_sel, st));
   INIT_CUDA(cudaMemsetAsync(c->at<char>(L.sel), 0, L.total - L.sel, st));
   INIT_CUDA(cudaMemsetAsync(c->at<char>(L.L_next), 0xFF, 2 * N * cfg->num_segments * 4, st));
-  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.tile_count), 0, (uint64_t)L.num_tiles * 4, st));
+  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.part_cands), 0, (uint64_t)kMaxGrid * 8, st));
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.tiles), tiles.data(), tiles.size() * sizeof(Tile), cudaMemcpyHostToDevice, st));
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.segs), segs.data(), segs.size() * sizeof(SegDesc), cudaMemcpyHostToDevice, st));
+  std::vector<uint32_t> seg_off(cfg->num_segments + 1), seg_tile0(cfg->num_segments);
+  for (uint32_t q = 0; q < cfg->num_segments; ++q) {
+    seg_off[q] = (uint32_t)cfg->segments[q].offset;
+    seg_tile0[q] = segs[q].tile_begin;
+  }
+  seg_off[cfg->num_segments] = (uint32_t)cfg->n;  // n < 2^32
+  INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.seg_off), seg_off.data(), seg_off.size() * 4, cudaMemcpyHostToDevice, st));
+  INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.seg_tile0), seg_tile0.data(), seg_tile0.size() * 4, cudaMemcpyHostToDevice, st));
   std::vector<float*> slots(N + 1);
   for (uint32_t q = 0; q <= N; ++q) slots[q] = c->u_buf(q);
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.u_slots), slots.data(), slots.size() * sizeof(float*), cudaMemcpyHostToDevice, st));
@@ -376,15 +433,19 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   w.num_segs = cfg->num_segments;
   w.cand_idx = c->at<uint32_t>(L.cand_idx);
   w.cand_val = c->at<float>(L.cand_val);
-  w.tile_count = c->at<uint32_t>(L.tile_count);
+  w.part_cands = c->at<uint32_t>(L.part_cands);
+  w.part_slot0 = c->at<uint32_t>(L.part_slot0);
+  w.seg_off = c->at<uint32_t>(L.seg_off);
+  w.seg_tile0 = c->at<uint32_t>(L.seg_tile0);
   w.tile_pre = c->at<uint2>(L.tile_pre);
+  w.tile_sel = c->at<uint2>(L.tile_sel);
   w.cta_tot = c->at<uint2>(L.cta_tot);
   w.hist1 = c->at<uint32_t>(L.hist1);
   w.hist2 = c->at<uint32_t>(L.hist2);
   w.hist3 = c->at<uint32_t>(L.hist3);
   w.sel = c->at<SegSel>(L.sel);
   w.L_safe = c->at<uint32_t>(L.L_safe);
-  w.flags = c->at<uint32_t>(L.flags);
+  w.sync = c->at<uint32_t>(L.sync);
   w.status = c->at<int>(L.status);
   w.stats = c->at<unsigned long long>(L.stats);
   *out = c;
@@ -402,18 +463,17 @@ int dgs_worker_push(dgs_ctx* c, uint32_t worker, const float* grad, dgs_packet* 
   a.grad = grad;
   a.u_cur_slot = c->u_slot(worker);
   a.u_spare_slot = c->u_slot(c->cfg.num_workers);
-  a.L_next = c->L_next(0, worker);
   a.pkt_idx = c->at<uint32_t>(L.pkt_idx[0]);
   a.pkt_val = c->at<float>(L.pkt_val[0]);
   a.pkt_count = (uint32_t)L.K[0];
   a.m = c->cfg.momentum;
   a.lr = c->cfg.lr;
   a.inv_m = c->inv_m;
-  const bool carried = c->seen[0][worker] != 0;
-  rc = (c->cfg.flags & DGS_RESIDUAL_MODE) ? launch_select<kPushResidual>(c, a, carried)
-                                          : launch_select<kPushSam>(c, a, carried);
+  const uint64_t age = c->pushes[worker];
+  rc = (c->cfg.flags & DGS_RESIDUAL_MODE) ? launch_select<kPushResidual>(c, a, worker, age)
+                                          : launch_select<kPushSam>(c, a, worker, age);
   if (rc != DGS_OK) return rc;
-  c->seen[0][worker] = 1;
+  c->pushes[worker] += 1;
   if (out) {
     out->idx = a.pkt_idx;
     out->val = a.pkt_val;
@@ -449,16 +509,16 @@ int dgs_worker_pull(dgs_ctx* c, uint32_t worker, dgs_packet* out) {
   std::memset(&a, 0, sizeof(a));
   a.D = c->D_buf(worker);
   a.theta_local = (c->cfg.flags & DGS_KEEP_LOCAL_MODEL) ? c->theta_local_buf(worker) : nullptr;
-  a.L_next = c->L_next(1, worker);
   a.pkt_idx = c->at<uint32_t>(L.pkt_idx[1]);
   a.pkt_val = c->at<float>(L.pkt_val[1]);
   a.pkt_count = (uint32_t)L.K[1];
   a.m = c->cfg.momentum;
   a.lr = c->cfg.lr;
   a.inv_m = c->inv_m;
-  rc = launch_select<kPull>(c, a, c->seen[1][worker] != 0);
+  // packets that entered D_worker since its previous pull
+  const uint64_t age = c->timestamp - (c->prev[worker] < 0 ? 0 : (uint64_t)c->prev[worker]);
+  rc = launch_select<kPull>(c, a, worker, age);
   if (rc != DGS_OK) return rc;
-  c->seen[1][worker] = 1;
   c->prev[worker] = (int64_t)c->timestamp;
   if (out) {
     out->idx = a.pkt_idx;
@@ -551,7 +611,7 @@ int dgs_stats(dgs_ctx* c, uint64_t out[4]) {
   out[0] = s[0];
   out[1] = s[1];
   out[2] = c->timestamp;
-  out[3] = 0;
+  out[3] = s[2];
   return DGS_OK;
 }
 

@@ -3,27 +3,29 @@
 // Selection scheme (used for the worker's top-k of the velocity, Algorithm 3, and
 // for the server's top-k of the model difference, Algorithm 2 / Eq. 6a):
 //
-//   stream pass   one read of the input.  Every element whose magnitude key is at
-//                 least a per-layer lower bound L becomes a "candidate": (index,
-//                 value) is appended, in index order, to the slot of its tile.
-//                 Everything below L is final at once (the push writes t*(1/m)).
-//   finalize      one cooperative kernel over the candidates only: three radix
-//                 levels (11+10+10 bits of the key) find the exact k-th largest
-//                 key T and the number r of entries equal to T that still fit;
-//                 an ordered count/scan/emit writes the packet in index order.
+//   stream pass   one read of the input by all SMs.  Every element whose magnitude
+//                 key is at least a per-layer lower bound L becomes a "candidate".
+//                 A warp handles one tile of 512 elements at a time and appends the
+//                 tile's candidates, in index order, as one "run" to its CTA's region
+//                 of the candidate buffer.  Everything below L is final at once (the
+//                 push writes t*(1/m) there).
+//   finalize      one small kernel (a few dozen co-resident CTAs with a barrier of
+//                 their own) over the candidates only: three radix levels (11+10+10
+//                 key bits) give the exact k-th largest key T and the number r of
+//                 entries equal to T that still fit; a count / scan / emit writes the
+//                 packet in index order.
 //
-// L is a guess carried from the worker's previous selection on that layer.  The
-// guess is checked exactly (a layer needs at least k candidates); when it fails,
-// or when there is no previous selection, finalize first runs a histogram pass
-// over the whole input to get a bound that cannot fail, and repeats the stream
-// pass itself.  The result never depends on the guess.
+// L is a guess carried over from an earlier selection of the same kind on that layer
+// (the host picks the most recent one made in a comparable state).  The guess is
+// checked exactly (a layer needs at least k candidates).  With nothing to carry
+// over, a histogram pass over the entire input comes first and gives a bound that
+// cannot fail; when a guess fails, finalize redoes both passes itself.  The result
+// never depends on the guess.
 #pragma once
-#include <cooperative_groups.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 namespace dgs {
-namespace cg = cooperative_groups;
 
 constexpr int kWarpTile = 512;      // elements per tile (one warp, 4 x float4 per lane)
 constexpr int kVecIters = 4;
@@ -35,7 +37,10 @@ constexpr int kBins3 = 1024;        // key bits  9..0
 constexpr uint32_t kFull = 0xFFFFFFFFu;
 constexpr uint32_t kSpecFactor = 3; // aim for max(3k, k+64) candidates next time
 constexpr uint32_t kSpecSlack = 64;
-constexpr int kMaxGrid = 2048;      // upper bound on the cooperative grid
+constexpr int kMaxGrid = 1024;      // upper bound on the grid of a stream pass (= parts of the candidate buffer)
+constexpr int kMaxWorkers = 128;    // upper bound on the grid of finalize
+constexpr uint32_t kSpinLimit = 1u << 22;  // bounded waits: give up and report after this many polls
+constexpr int kStatusTimeout = -4;  // = DGS_ETIMEOUT
 
 enum Mode : int { kPushSam = 0, kPushResidual = 1, kPull = 2 };
 
@@ -56,28 +61,34 @@ struct SegSel {        // per-layer selection state of the selection in flight
   uint32_t krem;       // entries still to take at or below the fixed prefix
   uint32_t T;          // k-th largest key
   uint32_t r;          // entries with key == T that are taken (lowest indices)
-  uint32_t pad[4];
 };
 
-enum Flag : int { kFlagFail = 0, kNumFlags = 4 };
+// word indices in Workspace::sync
+enum SyncWord : int { kBarCount = 0, kBarGen = 1, kDecision = 2, kFail = 3, kParts = 4, kNumSyncWords = 8 };
 
 struct Workspace {
   const Tile* tiles;
   const SegDesc* segs;
   uint32_t num_tiles, num_segs;
-  uint32_t* cand_idx;   // [n]  candidates of tile t live at [tiles[t].start, +tile_count[t])
-  float* cand_val;      // [n]
-  uint32_t* tile_count; // [num_tiles]
-  uint2* tile_pre;      // [num_tiles] CTA-local exclusive prefix of (key > T, key == T) counts
-  uint2* cta_tot;       // [kMaxGrid]
-  uint32_t* hist1;      // [S][kBins1]
-  uint32_t* hist2;      // [S][kBins2]
-  uint32_t* hist3;      // [S][kBins3]
-  SegSel* sel;          // [S]
-  uint32_t* L_safe;     // [S] bound from the whole-input histogram (two-pass route)
-  uint32_t* flags;      // [kNumFlags]
-  int* status;          // sticky device status word
-  unsigned long long* stats;  // [0] single-pass selections, [1] two-pass selections
+  // candidates: part p (CTA p of the grid that ran the stream pass, `parts` CTAs) owns the slots
+  // starting at the first element of its first tile
+  uint32_t* cand_idx;     // [n]
+  float* cand_val;        // [n]
+  uint32_t* part_cands;   // [kMaxGrid] candidates written by each part
+  uint32_t* part_slot0;   // [kMaxGrid] first slot of each part
+  const uint32_t* seg_off;   // [S+1] first element of each layer, and n
+  const uint32_t* seg_tile0; // [S]   first tile of each layer
+  uint2* tile_sel;        // [num_tiles] (#key > T, #key == T) per tile; all zero between selections
+  uint2* tile_pre;        // [num_tiles] exclusive prefix of tile_sel inside the scanning CTA's chunk
+  uint2* cta_tot;         // [kMaxWorkers]
+  uint32_t* hist1;        // [S][kBins1]
+  uint32_t* hist2;        // [S][kBins2]
+  uint32_t* hist3;        // [S][kBins3]
+  SegSel* sel;            // [S]
+  uint32_t* L_safe;       // [S] bound from the whole-input histogram (two-pass route)
+  uint32_t* sync;         // [kNumSyncWords]
+  int* status;            // sticky device status word
+  unsigned long long* stats;  // [0] single-pass selections, [1] two-pass selections, [2] candidates seen
 };
 
 struct SelArgs {
@@ -86,13 +97,16 @@ struct SelArgs {
   float** u_spare_slot;   // push: device slot holding the spare buffer pointer
   float* D;               // pull: D_w
   float* theta_local;     // pull: theta_w or null
-  uint32_t* L_next;       // [S] lower bounds carried to this worker's next selection of this kind
+  const uint32_t* L_in;   // [S] lower bounds guessed for this selection (single-pass route)
+  uint32_t* L_next;       // [S] receives the bounds this selection suggests for a later, similar one
   uint32_t* pkt_idx;
   float* pkt_val;
   uint32_t pkt_count;
   float m, lr, inv_m;
   int force_two_pass;
   int speculate;          // 0: never carry a bound (L_next is left alone)
+  uint32_t workers;       // CTAs of finalize that process the candidates
+  uint32_t seq;           // launch sequence number (tags the decision word)
 };
 
 __device__ __forceinline__ uint32_t key_of(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
@@ -100,6 +114,12 @@ __device__ __forceinline__ uint32_t lanemask_lt() {
   uint32_t m;
   asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
   return m;
+}
+__device__ __forceinline__ uint32_t ld_volatile(const uint32_t* p) {
+  return *reinterpret_cast<const volatile uint32_t*>(p);
+}
+__device__ __forceinline__ uint32_t part_first_tile(uint32_t part, uint32_t parts, uint32_t num_tiles) {
+  return (uint32_t)((uint64_t)part * num_tiles / parts);
 }
 
 // ---- the value an element contributes to the selection ------------------------
@@ -148,86 +168,11 @@ __device__ __forceinline__ void load_tile_vec(const float* __restrict__ a, const
 }
 
 // ---- stream pass ----------------------------------------------------------------
-// CTA `cta` of `G` handles a contiguous range of tiles, one tile per warp at a time.
-template <int MODE>
-__device__ void stream_tiles(const Workspace& ws, const SelArgs& a, const uint32_t* Larr,
-                             const float* __restrict__ in, float* __restrict__ out, uint32_t cta, uint32_t G) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t t0 = (uint32_t)((uint64_t)cta * ws.num_tiles / G);
-  const uint32_t t1 = (uint32_t)((uint64_t)(cta + 1) * ws.num_tiles / G);
-  const uint32_t lt = lanemask_lt();
-  for (uint32_t t = t0 + warp; t < t1; t += kWarps) {
-    const Tile tile = ws.tiles[t];
-    const uint32_t L = Larr[tile.seg];
-    uint32_t* h1 = ws.hist1 + (size_t)tile.seg * kBins1;
-    uint32_t running = 0;
-    if (tile.len == kWarpTile) {
-      float x[4 * kVecIters];
-      load_tile_vec<MODE>(in, a.grad, tile.start, lane, a.m, a.lr, x);
-      uint32_t mask = 0;
-#pragma unroll
-      for (int e = 0; e < 4 * kVecIters; ++e)
-        if (key_of(x[e]) >= L) mask |= 1u << e;
-      if (MODE != kPull) {
-        float4* po = reinterpret_cast<float4*>(out + tile.start) + lane;
-#pragma unroll
-        for (int j = 0; j < kVecIters; ++j) {
-          float4 o;
-          o.x = (mask >> (j * 4 + 0)) & 1 ? x[4 * j + 0] : unsent<MODE>(x[4 * j + 0], a.inv_m);
-          o.y = (mask >> (j * 4 + 1)) & 1 ? x[4 * j + 1] : unsent<MODE>(x[4 * j + 1], a.inv_m);
-          o.z = (mask >> (j * 4 + 2)) & 1 ? x[4 * j + 2] : unsent<MODE>(x[4 * j + 2], a.inv_m);
-          o.w = (mask >> (j * 4 + 3)) & 1 ? x[4 * j + 3] : unsent<MODE>(x[4 * j + 3], a.inv_m);
-          __stcs(po + j * 32, o);
-        }
-      }
-      if (__any_sync(kFull, mask != 0)) {
-#pragma unroll
-        for (int j = 0; j < kVecIters; ++j) {
-          const uint32_t mj = (mask >> (j * 4)) & 0xFu;
-          if (!__any_sync(kFull, mj != 0)) continue;
-          const uint32_t b0 = __ballot_sync(kFull, mj & 1u), b1 = __ballot_sync(kFull, mj & 2u);
-          const uint32_t b2 = __ballot_sync(kFull, mj & 4u), b3 = __ballot_sync(kFull, mj & 8u);
-          uint32_t pos = tile.start + running + __popc(b0 & lt) + __popc(b1 & lt) + __popc(b2 & lt) + __popc(b3 & lt);
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            if ((mj >> c) & 1u) {
-              const float v = x[4 * j + c];
-              ws.cand_idx[pos] = tile.start + j * 128 + lane * 4 + c;
-              ws.cand_val[pos] = v;
-              atomicAdd(h1 + (key_of(v) >> 20), 1u);
-              ++pos;
-            }
-          }
-          running += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
-        }
-      }
-    } else {
-      for (uint32_t base = 0; base < tile.len; base += 32) {
-        const uint32_t off = base + lane;
-        const bool valid = off < tile.len;
-        const uint32_t i = tile.start + off;
-        float x = 0.f;
-        bool cand = false;
-        if (valid) {
-          x = combine<MODE>(in[i], MODE != kPull ? a.grad[i] : 0.f, a.m, a.lr);
-          cand = key_of(x) >= L;
-          if (MODE != kPull) out[i] = cand ? x : unsent<MODE>(x, a.inv_m);
-        }
-        const uint32_t b = __ballot_sync(kFull, cand);
-        if (cand) {
-          const uint32_t pos = tile.start + running + __popc(b & lt);
-          ws.cand_idx[pos] = i;
-          ws.cand_val[pos] = x;
-          atomicAdd(h1 + (key_of(x) >> 20), 1u);
-        }
-        running += __popc(b);
-      }
-    }
-    if (lane == 0) ws.tile_count[t] = running;
-  }
-}
+struct StreamShared {
+  uint32_t hist[kBins1];  // top 11 key bits of the candidates of the layer being processed
+  uint32_t cursor;        // candidates appended by this CTA so far
+};
 
-// ---- histogram of ALL elements (top 11 key bits), for the bound that cannot fail ----
 __device__ __forceinline__ void flush_hist(uint32_t* s_hist, uint32_t* g_hist) {
   for (int b = threadIdx.x; b < kBins1; b += kThreads) {
     const uint32_t v = s_hist[b];
@@ -238,6 +183,132 @@ __device__ __forceinline__ void flush_hist(uint32_t* s_hist, uint32_t* g_hist) {
   }
 }
 
+// CTA `cta` of `G` handles a contiguous range of tiles, one tile per warp at a time,
+// layer by layer, so that the CTA's shared histogram always belongs to one layer; it
+// is added to the global one when the CTA leaves the layer.
+template <int MODE>
+__device__ void stream_tiles(const Workspace& ws, const SelArgs& a, const uint32_t* Larr,
+                             const float* __restrict__ in, float* __restrict__ out, uint32_t cta, uint32_t G,
+                             StreamShared& sh) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t t0 = part_first_tile(cta, G, ws.num_tiles), t1 = part_first_tile(cta + 1, G, ws.num_tiles);
+  const uint32_t lt = lanemask_lt();
+  for (int b = threadIdx.x; b < kBins1; b += kThreads) sh.hist[b] = 0;
+  if (threadIdx.x == 0) {
+    sh.cursor = 0;
+    if (cta == 0) ws.sync[kParts] = G;
+  }
+  __syncthreads();
+  if (t0 >= t1) {
+    if (threadIdx.x == 0) {
+      ws.part_cands[cta] = 0;
+      ws.part_slot0[cta] = 0;
+    }
+    return;
+  }
+  const uint32_t slot0 = ws.tiles[t0].start;  // first slot of this CTA's region
+  const uint32_t seg_first = ws.tiles[t0].seg, seg_last = ws.tiles[t1 - 1].seg;
+  for (uint32_t s = seg_first; s <= seg_last; ++s) {
+    const uint32_t a0 = max(t0, ws.segs[s].tile_begin), a1 = min(t1, ws.segs[s].tile_end);
+    const uint32_t L = Larr[s];
+    uint32_t t = a0 + warp;
+    Tile next;
+    next.start = 0; next.len = 0; next.seg = 0;
+    if (t < a1) next = ws.tiles[t];
+    for (; t < a1; t += kWarps) {
+      const Tile tile = next;
+      if (t + kWarps < a1) next = ws.tiles[t + kWarps];
+      if (tile.len == kWarpTile) {
+        float x[4 * kVecIters];
+        load_tile_vec<MODE>(in, a.grad, tile.start, lane, a.m, a.lr, x);
+        uint32_t mask = 0;
+#pragma unroll
+        for (int e = 0; e < 4 * kVecIters; ++e)
+          if (key_of(x[e]) >= L) mask |= 1u << e;
+        if (MODE != kPull) {
+          float4* po = reinterpret_cast<float4*>(out + tile.start) + lane;
+#pragma unroll
+          for (int j = 0; j < kVecIters; ++j) {
+            float4 o;
+            o.x = (mask >> (j * 4 + 0)) & 1 ? x[4 * j + 0] : unsent<MODE>(x[4 * j + 0], a.inv_m);
+            o.y = (mask >> (j * 4 + 1)) & 1 ? x[4 * j + 1] : unsent<MODE>(x[4 * j + 1], a.inv_m);
+            o.z = (mask >> (j * 4 + 2)) & 1 ? x[4 * j + 2] : unsent<MODE>(x[4 * j + 2], a.inv_m);
+            o.w = (mask >> (j * 4 + 3)) & 1 ? x[4 * j + 3] : unsent<MODE>(x[4 * j + 3], a.inv_m);
+            __stcs(po + j * 32, o);
+          }
+        }
+        const uint32_t total = __reduce_add_sync(kFull, (uint32_t)__popc(mask));
+        if (total) {
+          uint32_t base = 0;
+          if (lane == 0) base = slot0 + atomicAdd(&sh.cursor, total);
+          base = __shfl_sync(kFull, base, 0);
+#pragma unroll
+          for (int j = 0; j < kVecIters; ++j) {
+            const uint32_t mj = (mask >> (j * 4)) & 0xFu;
+            if (!__any_sync(kFull, mj != 0)) continue;
+            const uint32_t b0 = __ballot_sync(kFull, mj & 1u), b1 = __ballot_sync(kFull, mj & 2u);
+            const uint32_t b2 = __ballot_sync(kFull, mj & 4u), b3 = __ballot_sync(kFull, mj & 8u);
+            uint32_t pos = base + __popc(b0 & lt) + __popc(b1 & lt) + __popc(b2 & lt) + __popc(b3 & lt);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              if ((mj >> c) & 1u) {
+                const float v = x[4 * j + c];
+                ws.cand_idx[pos] = tile.start + j * 128 + lane * 4 + c;
+                ws.cand_val[pos] = v;
+                atomicAdd(sh.hist + (key_of(v) >> 20), 1u);
+                ++pos;
+              }
+            }
+            base += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
+          }
+        }
+      } else {
+        // ragged tile (first or last of a layer): one element per lane and step.  The tile
+        // has at most kWarpTile elements = 16 steps; candidate flags are kept as one bit per step.
+        uint32_t flags = 0;
+        for (int st = 0; st * 32 < (int)tile.len; ++st) {
+          const uint32_t off = st * 32 + lane;
+          if (off < tile.len) {
+            const uint32_t i = tile.start + off;
+            const float x = combine<MODE>(in[i], MODE != kPull ? a.grad[i] : 0.f, a.m, a.lr);
+            const bool cand = key_of(x) >= L;
+            if (MODE != kPull) out[i] = cand ? x : unsent<MODE>(x, a.inv_m);
+            if (cand) flags |= 1u << st;
+          }
+        }
+        const uint32_t total = __reduce_add_sync(kFull, (uint32_t)__popc(flags));
+        if (total) {
+          uint32_t base = 0;
+          if (lane == 0) base = slot0 + atomicAdd(&sh.cursor, total);
+          base = __shfl_sync(kFull, base, 0);
+          for (int st = 0; st * 32 < (int)tile.len; ++st) {
+            const bool cand = (flags >> st) & 1u;
+            const uint32_t b = __ballot_sync(kFull, cand);
+            if (cand) {
+              // a candidate's value is what this thread just stored (push) or the input itself (pull)
+              const uint32_t i = tile.start + st * 32 + lane;
+              const float x = MODE == kPull ? in[i] : out[i];
+              const uint32_t pos = base + __popc(b & lt);
+              ws.cand_idx[pos] = i;
+              ws.cand_val[pos] = x;
+              atomicAdd(sh.hist + (key_of(x) >> 20), 1u);
+            }
+            base += __popc(b);
+          }
+        }
+      }
+    }
+    __syncthreads();
+    flush_hist(sh.hist, ws.hist1 + (size_t)s * kBins1);
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    ws.part_cands[cta] = sh.cursor;
+    ws.part_slot0[cta] = slot0;
+  }
+}
+
+// ---- histogram of ALL elements (top 11 key bits), for the bound that cannot fail ----
 // Adds one warp-wide batch of bins to the shared histogram.  Lanes holding the same
 // bin as lane 0's are counted with one ballot (values cluster in few bins: zeros in a
 // sparse difference vector, the bulk of a bell-shaped gradient); the rest use atomics.
@@ -253,27 +324,15 @@ template <int MODE>
 __device__ void hist_all_tiles(const Workspace& ws, const SelArgs& a, const float* __restrict__ in,
                                uint32_t cta, uint32_t G, uint32_t* s_hist) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t t0 = (uint32_t)((uint64_t)cta * ws.num_tiles / G);
-  const uint32_t t1 = (uint32_t)((uint64_t)(cta + 1) * ws.num_tiles / G);
+  const uint32_t t0 = part_first_tile(cta, G, ws.num_tiles), t1 = part_first_tile(cta + 1, G, ws.num_tiles);
   for (int b = threadIdx.x; b < kBins1; b += kThreads) s_hist[b] = 0;
   __syncthreads();
   if (t0 >= t1) return;
-  uint32_t cur = ws.tiles[t0].seg;  // layer the shared histogram belongs to (CTA-uniform)
-  for (uint32_t chunk = t0; chunk < t1; chunk += kWarps) {
-    const uint32_t last = min(chunk + kWarps, t1) - 1;
-    const uint32_t seg_lo = ws.tiles[chunk].seg, seg_hi = ws.tiles[last].seg;
-    const uint32_t t = chunk + warp;
-    Tile tile;
-    tile.start = 0; tile.len = 0; tile.seg = 0xFFFF;
-    if (t < t1) tile = ws.tiles[t];
-    for (uint32_t s = seg_lo; s <= seg_hi; ++s) {
-      if (s != cur) {
-        __syncthreads();
-        flush_hist(s_hist, ws.hist1 + (size_t)cur * kBins1);
-        __syncthreads();
-        cur = s;
-      }
-      if (t >= t1 || tile.seg != s) continue;
+  const uint32_t seg_first = ws.tiles[t0].seg, seg_last = ws.tiles[t1 - 1].seg;
+  for (uint32_t s = seg_first; s <= seg_last; ++s) {
+    const uint32_t a0 = max(t0, ws.segs[s].tile_begin), a1 = min(t1, ws.segs[s].tile_end);
+    for (uint32_t t = a0 + warp; t < a1; t += kWarps) {
+      const Tile tile = ws.tiles[t];
       if (tile.len == kWarpTile) {
         float x[4 * kVecIters];
         load_tile_vec<MODE>(in, a.grad, tile.start, lane, a.m, a.lr, x);
@@ -292,10 +351,10 @@ __device__ void hist_all_tiles(const Workspace& ws, const SelArgs& a, const floa
         }
       }
     }
+    __syncthreads();
+    flush_hist(s_hist, ws.hist1 + (size_t)s * kBins1);
+    __syncthreads();
   }
-  __syncthreads();
-  flush_hist(s_hist, ws.hist1 + (size_t)cur * kBins1);
-  __syncthreads();
 }
 
 // ---- block-wide helpers (kThreads threads) -----------------------------------------
@@ -336,7 +395,7 @@ __device__ uint32_t block_pick(const uint32_t* hist, uint32_t k, uint32_t& bin, 
   const int top = B - 1 - threadIdx.x * PER;
 #pragma unroll
   for (int j = 0; j < PER; ++j) {
-    loc[j] = hist[top - j];
+    loc[j] = __ldcg(hist + top - j);
     sum += loc[j];
   }
   unsigned long long total;
@@ -359,48 +418,99 @@ __device__ uint32_t block_pick(const uint32_t* hist, uint32_t k, uint32_t& bin, 
   return (uint32_t)total;
 }
 
-// ---- radix level over the candidates ---------------------------------------------
-// LEVEL 2: candidates whose key bits 30..20 equal sel.prefix, digit = bits 19..10
-// LEVEL 3: candidates whose key bits 30..10 equal sel.prefix, digit = bits  9..0
-template <int LEVEL>
-__device__ void hist_candidates(const Workspace& ws, uint32_t gwarp, uint32_t nwarps) {
-  const int lane = threadIdx.x & 31;
-  uint32_t* hist = LEVEL == 2 ? ws.hist2 : ws.hist3;
-  constexpr int B = LEVEL == 2 ? kBins2 : kBins3;
-  constexpr int SH = LEVEL == 2 ? 20 : 10;
-  const uint32_t groups = (ws.num_tiles + 31) / 32;
-  for (uint32_t g = gwarp; g < groups; g += nwarps) {
-    const uint32_t t = g * 32 + lane;
-    const uint32_t cnt = t < ws.num_tiles ? ws.tile_count[t] : 0;
-    uint32_t nz = __ballot_sync(kFull, cnt != 0);
-    while (nz) {
-      const int src = __ffs(nz) - 1;
-      nz &= nz - 1;
-      const uint32_t c = __shfl_sync(kFull, cnt, src);
-      const Tile tile = ws.tiles[g * 32 + src];
-      const uint32_t prefix = ws.sel[tile.seg].prefix;
-      for (uint32_t i = lane; i < c; i += 32) {
-        const uint32_t key = key_of(ws.cand_val[tile.start + i]);
-        if ((key >> SH) == prefix) atomicAdd(hist + (size_t)tile.seg * B + ((key >> (SH - 10)) & 1023u), 1u);
+// Barrier among the first W CTAs of the grid (all resident: cooperative launch).
+// Bounded: returns false, with the status word set, if the others do not arrive.
+__device__ bool worker_barrier(uint32_t* sync, uint32_t W, int* status, int* s_ok) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int ok = 1;
+    __threadfence();
+    const uint32_t gen = ld_volatile(sync + kBarGen);
+    const uint32_t prev = atomicAdd(sync + kBarCount, 1u);
+    if (prev == W - 1) {
+      atomicExch(sync + kBarCount, 0u);
+      __threadfence();
+      atomicAdd(sync + kBarGen, 1u);
+    } else {
+      uint32_t spins = 0;
+      while (ld_volatile(sync + kBarGen) == gen) {
+        if (++spins > kSpinLimit) {
+          ok = 0;
+          atomicMin(status, kStatusTimeout);
+          break;
+        }
+        __nanosleep(20);
       }
     }
+    __threadfence();
+    *s_ok = ok;
   }
+  __syncthreads();
+  return *s_ok != 0;
 }
 
 // ---- finalize -------------------------------------------------------------------
+// The candidates are numbered flat over the parts: part p holds part_cands[p] of them in
+// consecutive slots from part_slot0[p] on, tile after tile (the tiles of a part in the
+// order its warps happened to finish them, each tile's candidates in index order).
+// Every phase below is one flat loop over that numbering; the layer and the tile of a
+// candidate follow from its index.
+constexpr int kSegCap = 1024;  // layers whose tables fit in shared memory; more fall back to global reads
+
+struct FinalizeShared {
+  StreamShared stream;                 // only used when the guess failed and the passes are redone here
+  unsigned long long warp_scan[kWarps];
+  uint32_t res[2];
+  int ok;
+  uint32_t pre_cands[kMaxGrid + 1];    // exclusive prefix of part_cands
+  uint32_t slot0[kMaxGrid];            // first slot of each part
+  uint2 base[kMaxWorkers];             // exclusive prefix of the scanning CTAs' (gt, eq) totals
+  uint32_t seg_off[kSegCap + 1];       // first element of each layer, and n
+  uint32_t seg_tile0[kSegCap];         // first tile of each layer
+  uint32_t seg_a[kSegCap];             // per-layer parameter of the current phase (prefix, or T)
+  uint32_t seg_b[kSegCap];             // second one (r)
+  uint2 seg_start[kSegCap];            // (gt, eq) counted before the layer's first tile
+};
+
+struct SegView {  // per-layer tables, in shared memory when they fit
+  const uint32_t* off;
+  const uint32_t* tile0;
+  uint32_t S;
+};
+
+// layer that holds element i: last s with off[s] <= i
+__device__ __forceinline__ uint32_t seg_of(const SegView& v, uint32_t i) {
+  uint32_t lo = 0, hi = v.S - 1;
+  while (lo < hi) {
+    const uint32_t mid = (lo + hi + 1) >> 1;
+    if (v.off[mid] <= i) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+// tiles of a layer are cut at the multiples of kWarpTile of the global index
+__device__ __forceinline__ uint32_t tile_of(const SegView& v, uint32_t seg, uint32_t i) {
+  return v.tile0[seg] + (i / kWarpTile - v.off[seg] / kWarpTile);
+}
+// slot of flat candidate p: last part with pre[part] <= p
+__device__ __forceinline__ uint32_t slot_of(const FinalizeShared& sh, uint32_t parts, uint32_t p, uint32_t* part_out) {
+  uint32_t lo = 0, hi = parts - 1;
+  while (lo < hi) {
+    const uint32_t mid = (lo + hi + 1) >> 1;
+    if (sh.pre_cands[mid] <= p) lo = mid; else hi = mid - 1;
+  }
+  if (part_out) *part_out = lo;
+  return sh.slot0[lo] + (p - sh.pre_cands[lo]);
+}
+
 template <int MODE>
 __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs a) {
-  cg::grid_group grid = cg::this_grid();
-  __shared__ uint32_t s_hist[kBins1];
-  __shared__ unsigned long long s_warp[kWarps];
-  __shared__ uint32_t s_res[2];
-  __shared__ uint2 s_base[kMaxGrid];
+  __shared__ FinalizeShared sh;
 
   constexpr int PM = MODE == kPull ? 1 : 0;
-  const uint32_t cta = blockIdx.x, G = gridDim.x;
+  const uint32_t cta = blockIdx.x, W = gridDim.x, S = ws.num_segs;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t gwarp = cta * kWarps + warp, nwarps = G * kWarps;
   const uint32_t lt = lanemask_lt();
+  const uint32_t gthread = cta * kThreads + threadIdx.x, nthreads = W * kThreads;
 
   // pointers are read once, before anything may exchange them
   const float* in = nullptr;
@@ -411,206 +521,274 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
     in = *a.u_cur_slot;
     out = *a.u_spare_slot;
   }
-  grid.sync();
 
-  bool two_pass = a.force_two_pass != 0;
+  // layer tables
+  const bool seg_smem = S <= (uint32_t)kSegCap;
+  if (seg_smem) {
+    for (uint32_t s = threadIdx.x; s <= S; s += kThreads) sh.seg_off[s] = ws.seg_off[s];
+    for (uint32_t s = threadIdx.x; s < S; s += kThreads) sh.seg_tile0[s] = ws.segs[s].tile_begin;
+  }
+  SegView sv;
+  sv.off = seg_smem ? sh.seg_off : ws.seg_off;
+  sv.tile0 = seg_smem ? sh.seg_tile0 : ws.seg_tile0;
+  sv.S = S;
+  __syncthreads();
+
+  bool redo = false;
   for (int attempt = 0; attempt < 2; ++attempt) {
-    if (two_pass) {
-      // bound that cannot fail: lower edge of the top-11-bit bin holding the k-th largest key
-      hist_all_tiles<MODE>(ws, a, in, cta, G, s_hist);
-      grid.sync();
-      for (uint32_t s = cta; s < ws.num_segs; s += G) {
+    if (redo) {
+      // the guess was too high for some layer: take the bound that cannot fail from a histogram of
+      // the whole input and repeat the stream pass, with the few CTAs this kernel has
+      hist_all_tiles<MODE>(ws, a, in, cta, W, sh.stream.hist);
+      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
+      for (uint32_t s = cta; s < S; s += W) {
         uint32_t bin, krem;
         uint32_t* h = ws.hist1 + (size_t)s * kBins1;
-        block_pick<kBins1>(h, ws.segs[s].k[PM], bin, krem, s_warp, s_res);
+        block_pick<kBins1>(h, ws.segs[s].k[PM], bin, krem, sh.warp_scan, sh.res);
         if (threadIdx.x == 0) ws.L_safe[s] = bin << 20;
         for (int b = threadIdx.x; b < kBins1; b += kThreads) h[b] = 0;
       }
-      if (cta == 0 && threadIdx.x == 0) ws.flags[kFlagFail] = 0;
-      grid.sync();
-      stream_tiles<MODE>(ws, a, ws.L_safe, in, out, cta, G);
-      grid.sync();
+      if (cta == 0 && threadIdx.x == 0) ws.sync[kFail] = 0;
+      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
+      stream_tiles<MODE>(ws, a, ws.L_safe, in, out, cta, W, sh.stream);
+      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
     }
     // level 1: pick the bin of the k-th largest among the candidates; check the guess
-    for (uint32_t s = cta; s < ws.num_segs; s += G) {
+    for (uint32_t s = cta; s < S; s += W) {
       uint32_t bin, krem;
       uint32_t* h = ws.hist1 + (size_t)s * kBins1;
       const uint32_t k = ws.segs[s].k[PM];
-      const uint32_t total = block_pick<kBins1>(h, k, bin, krem, s_warp, s_res);
+      const uint32_t total = block_pick<kBins1>(h, k, bin, krem, sh.warp_scan, sh.res);
       if (total < k) {
-        if (threadIdx.x == 0) atomicOr(ws.flags + kFlagFail, 1u);
+        if (threadIdx.x == 0) atomicOr(ws.sync + kFail, 1u);
       } else {
         if (threadIdx.x == 0) {
           ws.sel[s].prefix = bin;
           ws.sel[s].krem = krem;
+          atomicAdd(ws.stats + 2, (unsigned long long)total);
         }
         if (a.speculate) {
-          // bound for this worker's next selection on this layer
+          // bound suggested for a later selection on this layer
           const uint32_t want = max(k * kSpecFactor, k + kSpecSlack);
           uint32_t lbin, lrem;
           if (total >= want) {
-            block_pick<kBins1>(h, want, lbin, lrem, s_warp, s_res);
+            block_pick<kBins1>(h, want, lbin, lrem, sh.warp_scan, sh.res);
           } else {
-            const uint32_t used = (two_pass ? ws.L_safe[s] : a.L_next[s]) >> 20;
+            const uint32_t used = (redo ? __ldcg(ws.L_safe + s) : a.L_in[s]) >> 20;
             lbin = used > 0 ? used - 1 : 0;
           }
+          __syncthreads();
           if (threadIdx.x == 0) a.L_next[s] = lbin << 20;
         }
       }
       __syncthreads();
       for (int b = threadIdx.x; b < kBins1; b += kThreads) h[b] = 0;
     }
-    grid.sync();
-    if (two_pass || ws.flags[kFlagFail] == 0) break;
-    two_pass = true;  // the guess was too high somewhere: redo with a safe bound
+    if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
+    if (redo || ld_volatile(ws.sync + kFail) == 0) break;
+    redo = true;
   }
 
-  // level 2
-  hist_candidates<2>(ws, gwarp, nwarps);
-  grid.sync();
-  for (uint32_t s = cta; s < ws.num_segs; s += G) {
-    uint32_t bin, krem;
-    uint32_t* h = ws.hist2 + (size_t)s * kBins2;
-    block_pick<kBins2>(h, ws.sel[s].krem, bin, krem, s_warp, s_res);
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      ws.sel[s].prefix = (ws.sel[s].prefix << 10) | bin;
-      ws.sel[s].krem = krem;
-    }
-    for (int b = threadIdx.x; b < kBins2; b += kThreads) h[b] = 0;
-  }
-  grid.sync();
-  // level 3
-  hist_candidates<3>(ws, gwarp, nwarps);
-  grid.sync();
-  for (uint32_t s = cta; s < ws.num_segs; s += G) {
-    uint32_t bin, krem;
-    uint32_t* h = ws.hist3 + (size_t)s * kBins3;
-    block_pick<kBins3>(h, ws.sel[s].krem, bin, krem, s_warp, s_res);
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      ws.sel[s].T = (ws.sel[s].prefix << 10) | bin;
-      ws.sel[s].r = krem;
-    }
-    for (int b = threadIdx.x; b < kBins3; b += kThreads) h[b] = 0;
-  }
-  grid.sync();
-
-  // ---- ordered count: per tile (#key > T, #key == T), CTA-local exclusive prefix ----
-  const uint32_t t0 = (uint32_t)((uint64_t)cta * ws.num_tiles / G);
-  const uint32_t t1 = (uint32_t)((uint64_t)(cta + 1) * ws.num_tiles / G);
+  // flat numbering of the candidates
+  const uint32_t parts = ld_volatile(ws.sync + kParts);
   {
     unsigned long long carry = 0;
-    for (uint32_t chunk = t0; chunk < t1; chunk += kThreads) {
-      const uint32_t t = chunk + threadIdx.x;
-      const uint32_t cnt = t < t1 ? ws.tile_count[t] : 0;
-      uint32_t my_gt = 0, my_eq = 0;
-      uint32_t nz = __ballot_sync(kFull, cnt != 0);
-      while (nz) {
-        const int src = __ffs(nz) - 1;
-        nz &= nz - 1;
-        const uint32_t c = __shfl_sync(kFull, cnt, src);
-        const Tile tile = ws.tiles[chunk + warp * 32 + src];
-        const uint32_t T = ws.sel[tile.seg].T;
-        uint32_t gt = 0, eq = 0;
-        for (uint32_t i = lane; i < c; i += 32) {
-          const uint32_t key = key_of(ws.cand_val[tile.start + i]);
-          gt += key > T;
-          eq += key == T;
-        }
-        gt = __reduce_add_sync(kFull, gt);
-        eq = __reduce_add_sync(kFull, eq);
-        if (lane == src) {
-          my_gt = gt;
-          my_eq = eq;
+    for (uint32_t base = 0; base < parts; base += kThreads) {
+      const uint32_t p = base + threadIdx.x;
+      const unsigned long long v = p < parts ? __ldcg(ws.part_cands + p) : 0;
+      unsigned long long total;
+      const unsigned long long ex = block_excl_scan(v, sh.warp_scan, total) + carry;
+      if (p < parts) {
+        sh.pre_cands[p] = (uint32_t)ex;
+        sh.slot0[p] = __ldcg(ws.part_slot0 + p);
+      }
+      carry += total;
+    }
+    if (threadIdx.x == 0) sh.pre_cands[parts] = (uint32_t)carry;
+    __syncthreads();
+  }
+  const uint32_t C = sh.pre_cands[parts];
+
+  // ---- levels 2 and 3 ----------------------------------------------------------------
+#pragma unroll 1
+  for (int level = 2; level <= 3; ++level) {
+    uint32_t* hist = level == 2 ? ws.hist2 : ws.hist3;
+    const int B = level == 2 ? kBins2 : kBins3;   // both 1024
+    const int SH = level == 2 ? 20 : 10;
+    if (seg_smem) {
+      for (uint32_t s = threadIdx.x; s < S; s += kThreads) sh.seg_a[s] = __ldcg(&ws.sel[s].prefix);
+      __syncthreads();
+    }
+    for (uint32_t p = gthread; p < C; p += nthreads) {
+      const uint32_t slot = slot_of(sh, parts, p, nullptr);
+      const uint32_t key = key_of(__ldcg(ws.cand_val + slot));
+      uint32_t seg = 0;
+      if (S > 1) seg = seg_of(sv, __ldcg(ws.cand_idx + slot));
+      const uint32_t prefix = seg_smem ? sh.seg_a[seg] : __ldcg(&ws.sel[seg].prefix);
+      if ((key >> SH) == prefix) atomicAdd(hist + (size_t)seg * B + ((key >> (SH - 10)) & 1023u), 1u);
+    }
+    if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
+    for (uint32_t s = cta; s < S; s += W) {
+      uint32_t bin, krem;
+      uint32_t* h = hist + (size_t)s * B;
+      block_pick<kBins2>(h, __ldcg(&ws.sel[s].krem), bin, krem, sh.warp_scan, sh.res);
+      if (threadIdx.x == 0) {
+        const uint32_t pre = (__ldcg(&ws.sel[s].prefix) << 10) | bin;
+        ws.sel[s].prefix = pre;
+        ws.sel[s].krem = krem;
+        if (level == 3) {
+          ws.sel[s].T = pre;   // all 31 key bits are fixed now
+          ws.sel[s].r = krem;
         }
       }
+      for (int b = threadIdx.x; b < B; b += kThreads) h[b] = 0;
+    }
+    if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
+  }
+
+  // ---- count: per tile, how many candidates have key > T and key == T ----------------
+  // (tile_sel is all zero on entry: the scan below clears what it reads)
+  if (seg_smem) {
+    for (uint32_t s = threadIdx.x; s < S; s += kThreads) {
+      sh.seg_a[s] = __ldcg(&ws.sel[s].T);
+      sh.seg_b[s] = __ldcg(&ws.sel[s].r);
+    }
+    __syncthreads();
+  }
+  for (uint32_t p = gthread; p < C; p += nthreads) {
+    const uint32_t slot = slot_of(sh, parts, p, nullptr);
+    const uint32_t key = key_of(__ldcg(ws.cand_val + slot));
+    const uint32_t idx = __ldcg(ws.cand_idx + slot);
+    const uint32_t seg = S > 1 ? seg_of(sv, idx) : 0;
+    const uint32_t T = seg_smem ? sh.seg_a[seg] : __ldcg(&ws.sel[seg].T);
+    if (key >= T) {
+      uint2* c = ws.tile_sel + tile_of(sv, seg, idx);
+      atomicAdd(key > T ? &c->x : &c->y, 1u);
+    }
+  }
+  if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
+
+  // ---- scan over the tiles in index order: CTA c owns tiles [c*chunk, (c+1)*chunk) ----
+  const uint32_t chunk_tiles = (ws.num_tiles + W - 1) / W;
+  {
+    const uint32_t t0 = min(ws.num_tiles, cta * chunk_tiles), t1 = min(ws.num_tiles, t0 + chunk_tiles);
+    unsigned long long carry = 0;
+    for (uint32_t base = t0; base < t1; base += kThreads) {
+      const uint32_t t = base + threadIdx.x;
+      unsigned long long v = 0;
+      if (t < t1) {
+        const uint2 c = __ldcg(ws.tile_sel + t);
+        v = ((unsigned long long)c.x << 32) | c.y;
+        if (v) ws.tile_sel[t] = make_uint2(0, 0);
+      }
       unsigned long long total;
-      const unsigned long long v = ((unsigned long long)my_gt << 32) | my_eq;
-      const unsigned long long ex = block_excl_scan(v, s_warp, total) + carry;
+      const unsigned long long ex = block_excl_scan(v, sh.warp_scan, total) + carry;
       if (t < t1) ws.tile_pre[t] = make_uint2((uint32_t)(ex >> 32), (uint32_t)ex);
       carry += total;
     }
     if (threadIdx.x == 0) ws.cta_tot[cta] = make_uint2((uint32_t)(carry >> 32), (uint32_t)carry);
   }
-  grid.sync();
+  if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
 
   // ---- emit: packet in index order, and the state updates that depend on selection ----
   {
-    // exclusive prefix of the CTA totals (G <= kMaxGrid)
-    unsigned long long carry = 0;
-    for (uint32_t base = 0; base < G; base += kThreads) {
+    unsigned long long carry = 0;  // exclusive prefix of the CTAs' totals (W <= kMaxWorkers)
+    for (uint32_t base = 0; base < W; base += kThreads) {
       const uint32_t c = base + threadIdx.x;
       unsigned long long v = 0;
-      if (c < G) {
-        const uint2 q = ws.cta_tot[c];
+      if (c < W) {
+        const uint2 q = __ldcg(ws.cta_tot + c);
         v = ((unsigned long long)q.x << 32) | q.y;
       }
       unsigned long long total;
-      const unsigned long long ex = block_excl_scan(v, s_warp, total) + carry;
-      if (c < G) s_base[c] = make_uint2((uint32_t)(ex >> 32), (uint32_t)ex);
+      const unsigned long long ex = block_excl_scan(v, sh.warp_scan, total) + carry;
+      if (c < W) sh.base[c] = make_uint2((uint32_t)(ex >> 32), (uint32_t)ex);
       carry += total;
     }
     __syncthreads();
-    const uint2 my_base = s_base[cta];
-    for (uint32_t chunk = t0 + warp * 32; chunk < t1; chunk += kThreads) {
-      const uint32_t t = chunk + lane;
-      const uint32_t cnt = t < t1 ? ws.tile_count[t] : 0;
-      uint32_t nz = __ballot_sync(kFull, cnt != 0);
-      while (nz) {
-        const int src = __ffs(nz) - 1;
-        nz &= nz - 1;
-        const uint32_t c = __shfl_sync(kFull, cnt, src);
-        const uint32_t tt = chunk + src;
-        const Tile tile = ws.tiles[tt];
-        const SegDesc sd = ws.segs[tile.seg];
-        const uint32_t T = ws.sel[tile.seg].T, r = ws.sel[tile.seg].r;
-        // counts before this tile, and before this tile's layer, in global tile order
-        const uint2 pre = ws.tile_pre[tt];
-        const uint32_t tb = sd.tile_begin;
-        uint32_t owner = (uint32_t)(((uint64_t)tb * G) / ws.num_tiles);
-        while (owner + 1 < G && (uint32_t)((uint64_t)(owner + 1) * ws.num_tiles / G) <= tb) ++owner;
-        while (owner > 0 && (uint32_t)((uint64_t)owner * ws.num_tiles / G) > tb) --owner;
-        const uint2 pre0 = ws.tile_pre[tb];
-        const uint2 base0 = s_base[owner];
-        uint32_t gt_run = (my_base.x + pre.x) - (base0.x + pre0.x);
-        uint32_t eq_run = (my_base.y + pre.y) - (base0.y + pre0.y);
-        for (uint32_t i0 = 0; i0 < c; i0 += 32) {
-          const uint32_t i = i0 + lane;
-          const bool valid = i < c;
-          uint32_t idx = 0;
-          float val = 0.f;
-          uint32_t key = 0;
-          if (valid) {
-            idx = ws.cand_idx[tile.start + i];
-            val = ws.cand_val[tile.start + i];
-            key = key_of(val);
+    // (gt, eq) counted before tile t, over all layers
+    auto before_tile = [&](uint32_t t) {
+      const uint2 pre = __ldcg(ws.tile_pre + t), b = sh.base[t / chunk_tiles];
+      return make_uint2(b.x + pre.x, b.y + pre.y);
+    };
+    if (seg_smem) {
+      for (uint32_t s = threadIdx.x; s < S; s += kThreads) sh.seg_start[s] = before_tile(sh.seg_tile0[s]);
+      __syncthreads();
+    }
+    const uint32_t gwarp = cta * kWarps + warp, nwarps = W * kWarps;
+    for (uint32_t c0 = gwarp * 32; c0 < C; c0 += nwarps * 32) {
+      const uint32_t p = c0 + lane;
+      const bool valid = p < C;
+      uint32_t part = 0, idx = 0, key = 0, seg = 0, tile = 0xFFFFFFFFu, T = 0, r = 0;
+      float val = 0.f;
+      if (valid) {
+        const uint32_t slot = slot_of(sh, parts, p, &part);
+        idx = __ldcg(ws.cand_idx + slot);
+        val = __ldcg(ws.cand_val + slot);
+        key = key_of(val);
+        seg = S > 1 ? seg_of(sv, idx) : 0;
+        tile = tile_of(sv, seg, idx);
+        T = seg_smem ? sh.seg_a[seg] : __ldcg(&ws.sel[seg].T);
+        r = seg_smem ? sh.seg_b[seg] : __ldcg(&ws.sel[seg].r);
+      }
+      const bool is_gt = valid && key > T, is_eq = valid && key == T;
+      const uint32_t bgt = __ballot_sync(kFull, is_gt), beq = __ballot_sync(kFull, is_eq);
+      // the candidates of one tile are consecutive: a lane starts a tile if its left neighbour is in another one
+      const uint32_t left = __shfl_up_sync(kFull, tile, 1);
+      const uint32_t heads = __ballot_sync(kFull, lane == 0 || left != tile);
+      const int head = 31 - __clz(heads & (lt | (1u << lane)));       // first lane of my tile in this step
+      const uint32_t mine = lt & ~((1u << head) - 1u);                  // lanes of my tile before me
+      // the tile of lane 0 may have started in earlier slots of the same part: count what it holds there
+      uint32_t carry_gt = 0, carry_eq = 0;
+      {
+        const uint32_t tile0 = __shfl_sync(kFull, tile, 0), part0 = __shfl_sync(kFull, part, 0);
+        const uint32_t T0 = __shfl_sync(kFull, T, 0), seg0 = __shfl_sync(kFull, seg, 0);
+        const uint32_t first = sh.pre_cands[part0];                     // flat number of the part's first candidate
+        uint32_t back = c0;
+        while (back > first) {                                          // warp-uniform
+          const uint32_t lo = back - min(back - first, 32u);
+          const uint32_t pp = lo + lane;
+          bool same = false;
+          uint32_t k2 = 0;
+          if (pp < back) {
+            const uint32_t slot = sh.slot0[part0] + (pp - first);
+            const uint32_t i2 = __ldcg(ws.cand_idx + slot);
+            const uint32_t s2 = S > 1 ? seg_of(sv, i2) : 0;
+            same = s2 == seg0 && tile_of(sv, s2, i2) == tile0;
+            k2 = key_of(__ldcg(ws.cand_val + slot));
           }
-          const bool is_gt = valid && key > T, is_eq = valid && key == T;
-          const uint32_t bgt = __ballot_sync(kFull, is_gt), beq = __ballot_sync(kFull, is_eq);
-          const uint32_t gt_before = gt_run + __popc(bgt & lt);
-          const uint32_t eq_before = eq_run + __popc(beq & lt);
-          const bool sel = is_gt || (is_eq && eq_before < r);
-          if (valid) {
-            if (sel) {
-              const uint32_t pos = sd.pkt_off[PM] + gt_before + min(eq_before, r);
-              if (pos < a.pkt_count) {
-                a.pkt_idx[pos] = idx;
-                a.pkt_val[pos] = val;
-              } else {
-                atomicMin(ws.status, -1000 - MODE);
-              }
-              if (MODE == kPushResidual) out[idx] = 0.f;       // Algorithm 1: the sent part leaves v
-              if (MODE == kPull) {
-                a.D[idx] = 0.f;                                // Eq. 6b: v_k <- v_k + G
-                if (a.theta_local) a.theta_local[idx] = __fadd_rn(a.theta_local[idx], val);  // Eq. 5
-              }
-            } else {
-              if (MODE == kPushSam) out[idx] = __fmul_rn(val, a.inv_m);  // Eq. 12, lower branch
-            }
+          const uint32_t bs = __ballot_sync(kFull, same);
+          carry_gt += __popc(__ballot_sync(kFull, same && k2 > T0));
+          carry_eq += __popc(__ballot_sync(kFull, same && k2 == T0));
+          if (bs != __ballot_sync(kFull, pp < back)) break;             // reached another tile
+          back = lo;
+        }
+      }
+      if (valid) {
+        const uint2 tb = before_tile(tile);
+        const uint2 s0 = seg_smem ? sh.seg_start[seg] : before_tile(sv.tile0[seg]);
+        uint32_t gt_before = (tb.x - s0.x) + __popc(bgt & mine);
+        uint32_t eq_before = (tb.y - s0.y) + __popc(beq & mine);
+        if (head == 0) {
+          gt_before += carry_gt;
+          eq_before += carry_eq;
+        }
+        const bool sel = is_gt || (is_eq && eq_before < r);
+        if (sel) {
+          const uint32_t pos = ws.segs[seg].pkt_off[PM] + gt_before + min(eq_before, r);
+          if (pos < a.pkt_count) {
+            a.pkt_idx[pos] = idx;
+            a.pkt_val[pos] = val;
+          } else {
+            atomicMin(ws.status, -1000 - MODE);
           }
-          gt_run += __popc(bgt);
-          eq_run += __popc(beq);
+          if (MODE == kPushResidual) out[idx] = 0.f;       // Algorithm 1: the sent part leaves v
+          if (MODE == kPull) {
+            a.D[idx] = 0.f;                                // Eq. 6b: v_k <- v_k + G
+            if (a.theta_local) a.theta_local[idx] = __fadd_rn(a.theta_local[idx], val);  // Eq. 5
+          }
+        } else {
+          if (MODE == kPushSam) out[idx] = __fmul_rn(val, a.inv_m);  // Eq. 12, lower branch
         }
       }
     }
@@ -621,13 +799,37 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
       *a.u_cur_slot = *a.u_spare_slot;
       *a.u_spare_slot = cur;
     }
-    atomicAdd(ws.stats + (two_pass ? 1 : 0), 1ull);
+    atomicAdd(ws.stats + ((redo || a.force_two_pass) ? 1 : 0), 1ull);
+  }
+}
+
+// ---- the two passes as kernels of their own, for a selection with nothing to go by -------
+template <int MODE>
+__global__ void __launch_bounds__(kThreads, 4) k_hist_all(Workspace ws, SelArgs a) {
+  __shared__ uint32_t s_hist[kBins1];
+  const float* in = MODE == kPull ? a.D : *a.u_cur_slot;
+  hist_all_tiles<MODE>(ws, a, in, blockIdx.x, gridDim.x, s_hist);
+}
+
+// one CTA per layer (strided): L_safe = lower edge of the top-11-bit bin holding the k-th largest key
+template <int MODE>
+__global__ void __launch_bounds__(kThreads) k_pick_lower(Workspace ws) {
+  __shared__ unsigned long long s_warp[kWarps];
+  __shared__ uint32_t s_res[2];
+  constexpr int PM = MODE == kPull ? 1 : 0;
+  for (uint32_t s = blockIdx.x; s < ws.num_segs; s += gridDim.x) {
+    uint32_t bin, krem;
+    uint32_t* h = ws.hist1 + (size_t)s * kBins1;
+    block_pick<kBins1>(h, ws.segs[s].k[PM], bin, krem, s_warp, s_res);
+    if (threadIdx.x == 0) ws.L_safe[s] = bin << 20;
+    for (int b = threadIdx.x; b < kBins1; b += kThreads) h[b] = 0;
   }
 }
 
 // ---- stand-alone stream pass with the carried bound -------------------------------
 template <int MODE>
 __global__ void __launch_bounds__(kThreads, 4) k_stream(Workspace ws, SelArgs a) {
+  __shared__ StreamShared sh;
   const float* in;
   float* out = nullptr;
   if (MODE == kPull) {
@@ -636,7 +838,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_stream(Workspace ws, SelArgs a)
     in = *a.u_cur_slot;
     out = *a.u_spare_slot;
   }
-  stream_tiles<MODE>(ws, a, a.L_next, in, out, blockIdx.x, gridDim.x);
+  stream_tiles<MODE>(ws, a, a.L_in, in, out, blockIdx.x, gridDim.x, sh);
 }
 
 // ---- server apply ---------------------------------------------------------------
