@@ -47,7 +47,8 @@ typedef enum {
   DGS_ENOMEM = -2,   /* arena too small */
   DGS_ECUDA = -3,    /* a CUDA runtime call or launch failed; see dgs_last_cuda_error */
   DGS_ETIMEOUT = -4, /* a bounded device-side wait gave up (reported by dgs_status) */
-  DGS_ESTATE = -5    /* context already freed or unusable after an earlier error */
+  DGS_ESTATE = -5,   /* context already freed or unusable after an earlier error */
+  DGS_ELIMIT = -6    /* size beyond the fixed capacity of dgs_topk_encode_static */
 } dgs_error;
 
 typedef struct dgs_ctx dgs_ctx; /* opaque, host side */
@@ -190,6 +191,37 @@ int dgs_last_cuda_error(dgs_ctx* ctx);
 
 /* Frees the host-side context.  The arena stays the caller's.  Waits for the stream. */
 int dgs_free(dgs_ctx* ctx);
+
+/* Largest vector dgs_topk_encode_static accepts (elements). */
+#define DGS_STATIC_MAX_N (1u << 20)
+
+/* Top-k selection and coordinate-format encoding of one flat vector, for callers that
+ * must not allocate.  (No counterpart in the paper: this is the selection + encode() step
+ * of dgs_worker_pull offered on its own, for one layer, without a context.)
+ *
+ * Who needs it: code that runs where device allocation is off limits -- inside a region
+ * whose memory plan is frozen (a pre-sized pool that must not grow, a real-time or
+ * serving loop that may not call into the allocator), or a plug-in that is handed
+ * buffers but no allocator.  Such a caller cannot give dgs_init an arena either.  Here
+ * every byte of scratch (a private copy of x, the candidate list, histograms, the
+ * barrier words: about 12.6 MB) lives in one fixed array that is part of the library's
+ * device image; each GPU that loads the library holds it until the process exits.
+ *
+ *   x        DEVICE f32[n], read only
+ *   n, k     1 <= k <= n <= DGS_STATIC_MAX_N; a larger n returns DGS_ELIMIT, other bad
+ *            arguments DGS_EINVAL, and nothing is enqueued
+ *   out_idx  DEVICE u32[k], out_val DEVICE f32[k]: the k entries of largest |x| (ties to
+ *            the lowest index), ascending index, exactly as dgs_worker_pull would list them
+ *   stream   cudaStream_t; the work is enqueued there and the call returns
+ *
+ * The function calls no cudaMalloc / cudaFree and no allocating library routine.  The
+ * first call on each device looks up the address of the array for that device (the
+ * device must be current, as for every call) and sizes its launches; make that first
+ * call outside any stream capture.  All calls on a device share the one array: it keeps
+ * what the previous call left, the function clears what has to start at zero itself, and
+ * two calls whose work overlaps on the GPU (different streams, no ordering) race on it --
+ * order them. */
+int dgs_topk_encode_static(const float* x, uint32_t n, uint32_t k, uint32_t* out_idx, float* out_val, void* stream);
 
 /* Static text for a dgs_error value. */
 const char* dgs_error_string(int err);

@@ -23,8 +23,10 @@ EXPORTS = (
     "dgs_arena_bytes", "dgs_init", "dgs_worker_push", "dgs_server_apply", "dgs_worker_pull",
     "dgs_event", "dgs_event_host", "dgs_state_ptr", "dgs_state_load", "dgs_status", "dgs_stats",
     "dgs_prev", "dgs_launch_count", "dgs_last_cuda_error", "dgs_free", "dgs_error_string",
-    "dgs_timing_enable", "dgs_timing_read",
+    "dgs_timing_enable", "dgs_timing_read", "dgs_topk_encode_static",
 )
+DGS_ELIMIT = -6
+DGS_STATIC_MAX_N = 1 << 20
 DGS_NUM_KERNELS = 7
 KERNEL_NAMES = ("stream_push", "finalize_push", "two_pass_push", "scatter", "stream_pull", "finalize_pull",
                 "two_pass_pull")
@@ -76,6 +78,7 @@ def lib() -> C.CDLL:
         L.dgs_prev.argtypes = [vp, u32, C.POINTER(C.c_int64)]
         L.dgs_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
         L.dgs_last_cuda_error.argtypes = [vp]
+        L.dgs_topk_encode_static.argtypes = [vp, u32, u32, vp, vp, vp]
         L.dgs_timing_enable.argtypes = [vp, i32]
         L.dgs_timing_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
         L.dgs_free.argtypes = [vp]
@@ -190,6 +193,13 @@ def dgs_timing_read(ctx: int):
     cnt = (C.c_uint64 * DGS_NUM_KERNELS)()
     _check(lib().dgs_timing_read(ctx, ms, cnt), "dgs_timing_read")
     return {KERNEL_NAMES[i]: (float(ms[i]), int(cnt[i])) for i in range(DGS_NUM_KERNELS)}
+
+
+def dgs_topk_encode_static(x_ptr: int, n: int, k: int, out_idx_ptr: int, out_val_ptr: int, stream: int = 0) -> None:
+    """Top-k + encode of a flat device vector with no allocation anywhere (scratch is a
+    fixed array inside the library, n <= DGS_STATIC_MAX_N).  Enqueues on `stream`."""
+    _check(lib().dgs_topk_encode_static(x_ptr, n, k, out_idx_ptr, out_val_ptr, stream or None),
+           "dgs_topk_encode_static")
 
 
 def dgs_free(ctx: int) -> None:

@@ -4,7 +4,9 @@
 
 #include <algorithm>
 #include <cmath>
+#include <cstddef>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -312,6 +314,7 @@ const char* dgs_error_string(int err) {
     case DGS_ECUDA: return "CUDA runtime error";
     case DGS_ETIMEOUT: return "bounded device wait expired";
     case DGS_ESTATE: return "context freed or unusable";
+    case DGS_ELIMIT: return "size beyond the fixed capacity of the static scratch";
   }
   return "unknown error";
 }
@@ -674,3 +677,170 @@ int dgs_free(dgs_ctx* c) {
 }
 
 }  // extern "C"
+
+// ---- top-k + encode with all scratch in the device image (dgs_topk_encode_static) --------
+namespace {
+
+constexpr uint32_t kStaticMaxN = DGS_STATIC_MAX_N;
+constexpr uint32_t kStaticMaxTiles = kStaticMaxN / kWarpTile;  // one layer starting at 0: no ragged head
+
+struct StaticScratch {
+  float x[kStaticMaxN];            // private copy of the input (the selection clears what it sends)
+  uint32_t cand_idx[kStaticMaxN];
+  float cand_val[kStaticMaxN];
+  Tile tiles[kStaticMaxTiles];
+  uint2 tile_sel[kStaticMaxTiles];
+  uint2 tile_pre[kStaticMaxTiles];
+  uint32_t part_cands[kMaxGrid];
+  uint32_t part_slot0[kMaxGrid];
+  uint2 cta_tot[kMaxWorkers];
+  uint32_t hist1[kBins1];
+  uint32_t hist2[kBins2];
+  uint32_t hist3[kBins3];
+  SegDesc seg;
+  SegSel sel;
+  uint32_t seg_off[2];
+  uint32_t seg_tile0[1];
+  uint32_t L_safe[1];
+  uint32_t L_next[1];
+  uint32_t sync[kNumSyncWords];
+  int status;
+  unsigned long long stats[4];
+};
+
+// The scratch itself.  In host code this name is only a handle for cudaGetSymbolAddress,
+// never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
+
+// Tables of a one-layer problem and everything that has to start at zero.
+__global__ void k_static_prepare(StaticScratch* sc, uint32_t n, uint32_t k, uint32_t num_tiles) {
+  const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < num_tiles) {
+    Tile t;
+    t.start = i * kWarpTile;
+    t.len = (uint16_t)min((uint32_t)kWarpTile, n - i * kWarpTile);
+    t.seg = 0;
+    sc->tiles[i] = t;
+    sc->tile_sel[i] = make_uint2(0, 0);
+  }
+  if (i < kBins1) sc->hist1[i] = 0;
+  if (i < kBins2) sc->hist2[i] = 0;
+  if (i < kBins3) sc->hist3[i] = 0;
+  if (i < kMaxGrid) {
+    sc->part_cands[i] = 0;
+    sc->part_slot0[i] = 0;
+  }
+  if (i == 0) {
+    sc->seg.tile_begin = 0;
+    sc->seg.tile_end = num_tiles;
+    sc->seg.k[0] = sc->seg.k[1] = k;
+    sc->seg.pkt_off[0] = sc->seg.pkt_off[1] = 0;
+    sc->seg_off[0] = 0;
+    sc->seg_off[1] = n;
+    sc->seg_tile0[0] = 0;
+    sc->sync[kBarCount] = 0;
+    sc->sync[kFail] = 0;
+    sc->status = 0;
+  }
+}
+
+struct StaticDevice {
+  bool ready = false;
+  StaticScratch* scratch = nullptr;  // device address of g_static_scratch on this device
+  int stream_grid = 0, hist_grid = 0, finalize_grid = 0;
+};
+constexpr int kMaxDevices = 64;
+StaticDevice g_static_dev[kMaxDevices];
+std::mutex g_static_mu;
+
+// Once per device, with that device current.
+int static_setup(int dev, StaticDevice** out) {
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  StaticDevice& d = g_static_dev[dev];
+  if (!d.ready) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return DGS_ECUDA;
+    int sms = 0, coop = 0, occ = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return DGS_ECUDA;
+    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return DGS_ECUDA;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_stream<kPull>, kThreads, 0) != cudaSuccess) return DGS_ECUDA;
+    d.stream_grid = std::min(sms * std::max(occ, 1), kMaxGrid);
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_hist_all<kPull>, kThreads, 0) != cudaSuccess) return DGS_ECUDA;
+    d.hist_grid = std::min(sms * std::max(occ, 1), kMaxGrid);
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_finalize<kPull>, kThreads, 0) != cudaSuccess || occ < 1)
+      return DGS_ECUDA;
+    d.finalize_grid = std::min(std::min(sms * occ, kMaxWorkers), kFinalizeWorkers);
+    d.scratch = static_cast<StaticScratch*>(p);
+    d.ready = true;
+  }
+  *out = &d;
+  return DGS_OK;
+}
+
+}  // namespace
+
+extern "C" int dgs_topk_encode_static(const float* x, uint32_t n, uint32_t k, uint32_t* out_idx, float* out_val,
+                                      void* stream) {
+  if (!x || !out_idx || !out_val || n == 0 || k == 0 || k > n) return DGS_EINVAL;
+  if (n > kStaticMaxN) return DGS_ELIMIT;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return DGS_ECUDA;
+  StaticDevice* d = nullptr;
+  const int rc = static_setup(dev, &d);
+  if (rc != DGS_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  StaticScratch* sc = d->scratch;  // device address: only ever dereferenced by kernels
+  const uint32_t num_tiles = (n + kWarpTile - 1) / kWarpTile;
+
+  Workspace ws;
+  ws.tiles = sc->tiles;
+  ws.segs = &sc->seg;
+  ws.num_tiles = num_tiles;
+  ws.num_segs = 1;
+  ws.cand_idx = sc->cand_idx;
+  ws.cand_val = sc->cand_val;
+  ws.part_cands = sc->part_cands;
+  ws.part_slot0 = sc->part_slot0;
+  ws.seg_off = sc->seg_off;
+  ws.seg_tile0 = sc->seg_tile0;
+  ws.tile_sel = sc->tile_sel;
+  ws.tile_pre = sc->tile_pre;
+  ws.cta_tot = sc->cta_tot;
+  ws.hist1 = sc->hist1;
+  ws.hist2 = sc->hist2;
+  ws.hist3 = sc->hist3;
+  ws.sel = &sc->sel;
+  ws.L_safe = sc->L_safe;
+  ws.sync = sc->sync;
+  ws.status = &sc->status;
+  ws.stats = sc->stats;
+
+  SelArgs a;
+  std::memset(&a, 0, sizeof(a));
+  a.D = sc->x;
+  a.L_in = sc->L_safe;
+  a.L_next = sc->L_next;
+  a.pkt_idx = out_idx;
+  a.pkt_val = out_val;
+  a.pkt_count = k;
+  a.m = 1.0f;
+  a.inv_m = 1.0f;
+  a.force_two_pass = 1;
+  a.speculate = 0;
+  a.workers = (uint32_t)d->finalize_grid;
+  a.seq = 0;
+
+  if (cudaMemcpyAsync(sc->x, x, (size_t)n * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return DGS_ECUDA;
+  const uint32_t prep_items = std::max<uint32_t>(num_tiles, kBins1);
+  k_static_prepare<<<(prep_items + kThreads - 1) / kThreads, kThreads, 0, st>>>(sc, n, k, num_tiles);
+  k_hist_all<kPull><<<d->hist_grid, kThreads, 0, st>>>(ws, a);
+  k_pick_lower<kPull><<<1, kThreads, 0, st>>>(ws);
+  k_stream<kPull><<<d->stream_grid, kThreads, 0, st>>>(ws, a);
+  if (cudaGetLastError() != cudaSuccess) return DGS_ECUDA;
+  void* args[] = {(void*)&ws, (void*)&a};
+  if (cudaLaunchCooperativeKernel((const void*)k_finalize<kPull>, dim3(d->finalize_grid), dim3(kThreads), args, 0,
+                                  st) != cudaSuccess)
+    return DGS_ECUDA;
+  return DGS_OK;
+}
+
