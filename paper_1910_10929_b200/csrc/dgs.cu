@@ -155,6 +155,7 @@ struct dgs_ctx {
   Workspace ws;
   float inv_m;
   int stream_grid[3];    // CTAs of the stand-alone stream pass, per mode
+  int hist_grid[3];      // CTAs of the whole-input histogram pass, per mode
   int finalize_grid[3];  // CTAs of the cooperative finalize kernel, per mode
   uint32_t select_seq;   // selections launched so far (tags the decision word of each finalize launch)
   // Carried bounds: row (kind, worker) of L_next holds the bounds suggested by that worker's
@@ -257,7 +258,7 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age
     // nothing to go by: histogram of the whole input first, its bounds cannot fail
     a.L_in = c->ws.L_safe;
     TimedLaunch t(c, MODE == kPull ? DGS_KERNEL_TWO_PASS_PULL : DGS_KERNEL_TWO_PASS_PUSH);
-    k_hist_all<MODE><<<c->stream_grid[MODE], kThreads, 0, c->stream>>>(c->ws, a);
+    k_hist_all<MODE><<<c->hist_grid[MODE], kThreads, 0, c->stream>>>(c->ws, a);
     DGS_CUDA(c, cudaGetLastError());
     const int pick_grid = (int)std::min<uint32_t>(c->cfg.num_segments, 1024u);
     k_pick_lower<MODE><<<pick_grid, kThreads, 0, c->stream>>>(c->ws);
@@ -266,7 +267,7 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age
   }
   {
     TimedLaunch t(c, MODE == kPull ? DGS_KERNEL_STREAM_PULL : DGS_KERNEL_STREAM_PUSH);
-    k_stream<MODE><<<c->stream_grid[MODE], kThreads, 0, c->stream>>>(c->ws, a);
+    k_stream<MODE><<<c->stream_grid[MODE], kThreads, StreamRing<MODE>::kBytes, c->stream>>>(c->ws, a);
     DGS_CUDA(c, cudaGetLastError());
     c->launches += 1;
   }
@@ -289,9 +290,15 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age
 template <int MODE>
 int occupancy_grids(dgs_ctx* c, int sms) {
   int occ = 0;
-  DGS_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_stream<MODE>, kThreads, 0));
+  DGS_CUDA(c, cudaFuncSetAttribute(k_stream<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   StreamRing<MODE>::kBytes));
+  DGS_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_stream<MODE>, kThreads,
+                                                            StreamRing<MODE>::kBytes));
   if (occ < 1) occ = 1;
   c->stream_grid[MODE] = std::min(sms * occ, kMaxGrid);
+  DGS_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_hist_all<MODE>, kThreads, 0));
+  if (occ < 1) occ = 1;
+  c->hist_grid[MODE] = std::min(sms * occ, kMaxGrid);
   DGS_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_finalize<MODE>, kThreads, 0));
   if (occ < 1) {
     c->last_cuda = (int)cudaErrorCooperativeLaunchTooLarge;
@@ -763,7 +770,12 @@ int static_setup(int dev, StaticDevice** out) {
     int sms = 0, coop = 0, occ = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return DGS_ECUDA;
     if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return DGS_ECUDA;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_stream<kPull>, kThreads, 0) != cudaSuccess) return DGS_ECUDA;
+    if (cudaFuncSetAttribute(k_stream<kPull>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             StreamRing<kPull>::kBytes) != cudaSuccess)
+      return DGS_ECUDA;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_stream<kPull>, kThreads, StreamRing<kPull>::kBytes) !=
+        cudaSuccess)
+      return DGS_ECUDA;
     d.stream_grid = std::min(sms * std::max(occ, 1), kMaxGrid);
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_hist_all<kPull>, kThreads, 0) != cudaSuccess) return DGS_ECUDA;
     d.hist_grid = std::min(sms * std::max(occ, 1), kMaxGrid);
@@ -835,7 +847,7 @@ extern "C" int dgs_topk_encode_static(const float* x, uint32_t n, uint32_t k, ui
   k_static_prepare<<<(prep_items + kThreads - 1) / kThreads, kThreads, 0, st>>>(sc, n, k, num_tiles);
   k_hist_all<kPull><<<d->hist_grid, kThreads, 0, st>>>(ws, a);
   k_pick_lower<kPull><<<1, kThreads, 0, st>>>(ws);
-  k_stream<kPull><<<d->stream_grid, kThreads, 0, st>>>(ws, a);
+  k_stream<kPull><<<d->stream_grid, kThreads, StreamRing<kPull>::kBytes, st>>>(ws, a);
   if (cudaGetLastError() != cudaSuccess) return DGS_ECUDA;
   void* args[] = {(void*)&ws, (void*)&a};
   if (cudaLaunchCooperativeKernel((const void*)k_finalize<kPull>, dim3(d->finalize_grid), dim3(kThreads), args, 0,

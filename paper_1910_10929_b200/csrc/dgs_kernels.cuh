@@ -183,9 +183,100 @@ __device__ __forceinline__ void flush_hist(uint32_t* s_hist, uint32_t* g_hist) {
   }
 }
 
+// What follows the loads of a full tile: x[16] holds this lane's values (4 float4 at
+// elements j*128 + lane*4 + c of the tile).  Writes the new velocity (push), appends the
+// tile's candidates in index order to the CTA's region, histograms their top key bits.
+template <int MODE>
+__device__ __forceinline__ void finish_full_tile(const Workspace& ws, const SelArgs& a, StreamShared& sh,
+                                                 uint32_t tile_start, const float (&x)[4 * kVecIters], uint32_t L,
+                                                 uint32_t slot0, int lane, uint32_t lt, float* __restrict__ out) {
+  uint32_t mask = 0;
+#pragma unroll
+  for (int e = 0; e < 4 * kVecIters; ++e)
+    if (key_of(x[e]) >= L) mask |= 1u << e;
+  if (MODE != kPull) {
+    float4* po = reinterpret_cast<float4*>(out + tile_start) + lane;
+#pragma unroll
+    for (int j = 0; j < kVecIters; ++j) {
+      float4 o;
+      o.x = (mask >> (j * 4 + 0)) & 1 ? x[4 * j + 0] : unsent<MODE>(x[4 * j + 0], a.inv_m);
+      o.y = (mask >> (j * 4 + 1)) & 1 ? x[4 * j + 1] : unsent<MODE>(x[4 * j + 1], a.inv_m);
+      o.z = (mask >> (j * 4 + 2)) & 1 ? x[4 * j + 2] : unsent<MODE>(x[4 * j + 2], a.inv_m);
+      o.w = (mask >> (j * 4 + 3)) & 1 ? x[4 * j + 3] : unsent<MODE>(x[4 * j + 3], a.inv_m);
+      __stcs(po + j * 32, o);
+    }
+  }
+  const uint32_t total = __reduce_add_sync(kFull, (uint32_t)__popc(mask));
+  if (total) {
+    uint32_t base = 0;
+    if (lane == 0) base = slot0 + atomicAdd(&sh.cursor, total);
+    base = __shfl_sync(kFull, base, 0);
+#pragma unroll
+    for (int j = 0; j < kVecIters; ++j) {
+      const uint32_t mj = (mask >> (j * 4)) & 0xFu;
+      if (!__any_sync(kFull, mj != 0)) continue;
+      const uint32_t b0 = __ballot_sync(kFull, mj & 1u), b1 = __ballot_sync(kFull, mj & 2u);
+      const uint32_t b2 = __ballot_sync(kFull, mj & 4u), b3 = __ballot_sync(kFull, mj & 8u);
+      uint32_t pos = base + __popc(b0 & lt) + __popc(b1 & lt) + __popc(b2 & lt) + __popc(b3 & lt);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        if ((mj >> c) & 1u) {
+          const float v = x[4 * j + c];
+          ws.cand_idx[pos] = tile_start + j * 128 + lane * 4 + c;
+          ws.cand_val[pos] = v;
+          atomicAdd(sh.hist + (key_of(v) >> 20), 1u);
+          ++pos;
+        }
+      }
+      base += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
+    }
+  }
+}
+
+// A ragged tile (first or last of a layer, fewer than kWarpTile elements or not 16-byte
+// aligned): one element per lane and step, straight from global memory.  At most 16
+// steps; candidate flags are kept as one bit per step.
+template <int MODE>
+__device__ __forceinline__ void ragged_tile(const Workspace& ws, const SelArgs& a, StreamShared& sh, const Tile tile,
+                                            uint32_t L, uint32_t slot0, int lane, uint32_t lt,
+                                            const float* __restrict__ in, float* __restrict__ out) {
+  uint32_t flags = 0;
+  for (int st = 0; st * 32 < (int)tile.len; ++st) {
+    const uint32_t off = st * 32 + lane;
+    if (off < tile.len) {
+      const uint32_t i = tile.start + off;
+      const float x = combine<MODE>(in[i], MODE != kPull ? a.grad[i] : 0.f, a.m, a.lr);
+      const bool cand = key_of(x) >= L;
+      if (MODE != kPull) out[i] = cand ? x : unsent<MODE>(x, a.inv_m);
+      if (cand) flags |= 1u << st;
+    }
+  }
+  const uint32_t total = __reduce_add_sync(kFull, (uint32_t)__popc(flags));
+  if (total) {
+    uint32_t base = 0;
+    if (lane == 0) base = slot0 + atomicAdd(&sh.cursor, total);
+    base = __shfl_sync(kFull, base, 0);
+    for (int st = 0; st * 32 < (int)tile.len; ++st) {
+      const bool cand = (flags >> st) & 1u;
+      const uint32_t b = __ballot_sync(kFull, cand);
+      if (cand) {
+        // a candidate's value is what this thread just stored (push) or the input itself (pull)
+        const uint32_t i = tile.start + st * 32 + lane;
+        const float x = MODE == kPull ? in[i] : out[i];
+        const uint32_t pos = base + __popc(b & lt);
+        ws.cand_idx[pos] = i;
+        ws.cand_val[pos] = x;
+        atomicAdd(sh.hist + (key_of(x) >> 20), 1u);
+      }
+      base += __popc(b);
+    }
+  }
+}
+
 // CTA `cta` of `G` handles a contiguous range of tiles, one tile per warp at a time,
 // layer by layer, so that the CTA's shared histogram always belongs to one layer; it
-// is added to the global one when the CTA leaves the layer.
+// is added to the global one when the CTA leaves the layer.  Loads go straight from
+// global memory to registers (used where only a few CTAs run the pass).
 template <int MODE>
 __device__ void stream_tiles(const Workspace& ws, const SelArgs& a, const uint32_t* Larr,
                              const float* __restrict__ in, float* __restrict__ out, uint32_t cta, uint32_t G,
@@ -221,85 +312,212 @@ __device__ void stream_tiles(const Workspace& ws, const SelArgs& a, const uint32
       if (tile.len == kWarpTile) {
         float x[4 * kVecIters];
         load_tile_vec<MODE>(in, a.grad, tile.start, lane, a.m, a.lr, x);
-        uint32_t mask = 0;
-#pragma unroll
-        for (int e = 0; e < 4 * kVecIters; ++e)
-          if (key_of(x[e]) >= L) mask |= 1u << e;
-        if (MODE != kPull) {
-          float4* po = reinterpret_cast<float4*>(out + tile.start) + lane;
-#pragma unroll
-          for (int j = 0; j < kVecIters; ++j) {
-            float4 o;
-            o.x = (mask >> (j * 4 + 0)) & 1 ? x[4 * j + 0] : unsent<MODE>(x[4 * j + 0], a.inv_m);
-            o.y = (mask >> (j * 4 + 1)) & 1 ? x[4 * j + 1] : unsent<MODE>(x[4 * j + 1], a.inv_m);
-            o.z = (mask >> (j * 4 + 2)) & 1 ? x[4 * j + 2] : unsent<MODE>(x[4 * j + 2], a.inv_m);
-            o.w = (mask >> (j * 4 + 3)) & 1 ? x[4 * j + 3] : unsent<MODE>(x[4 * j + 3], a.inv_m);
-            __stcs(po + j * 32, o);
-          }
-        }
-        const uint32_t total = __reduce_add_sync(kFull, (uint32_t)__popc(mask));
-        if (total) {
-          uint32_t base = 0;
-          if (lane == 0) base = slot0 + atomicAdd(&sh.cursor, total);
-          base = __shfl_sync(kFull, base, 0);
-#pragma unroll
-          for (int j = 0; j < kVecIters; ++j) {
-            const uint32_t mj = (mask >> (j * 4)) & 0xFu;
-            if (!__any_sync(kFull, mj != 0)) continue;
-            const uint32_t b0 = __ballot_sync(kFull, mj & 1u), b1 = __ballot_sync(kFull, mj & 2u);
-            const uint32_t b2 = __ballot_sync(kFull, mj & 4u), b3 = __ballot_sync(kFull, mj & 8u);
-            uint32_t pos = base + __popc(b0 & lt) + __popc(b1 & lt) + __popc(b2 & lt) + __popc(b3 & lt);
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              if ((mj >> c) & 1u) {
-                const float v = x[4 * j + c];
-                ws.cand_idx[pos] = tile.start + j * 128 + lane * 4 + c;
-                ws.cand_val[pos] = v;
-                atomicAdd(sh.hist + (key_of(v) >> 20), 1u);
-                ++pos;
-              }
-            }
-            base += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
-          }
-        }
+        finish_full_tile<MODE>(ws, a, sh, tile.start, x, L, slot0, lane, lt, out);
       } else {
-        // ragged tile (first or last of a layer): one element per lane and step.  The tile
-        // has at most kWarpTile elements = 16 steps; candidate flags are kept as one bit per step.
-        uint32_t flags = 0;
-        for (int st = 0; st * 32 < (int)tile.len; ++st) {
-          const uint32_t off = st * 32 + lane;
-          if (off < tile.len) {
-            const uint32_t i = tile.start + off;
-            const float x = combine<MODE>(in[i], MODE != kPull ? a.grad[i] : 0.f, a.m, a.lr);
-            const bool cand = key_of(x) >= L;
-            if (MODE != kPull) out[i] = cand ? x : unsent<MODE>(x, a.inv_m);
-            if (cand) flags |= 1u << st;
-          }
-        }
-        const uint32_t total = __reduce_add_sync(kFull, (uint32_t)__popc(flags));
-        if (total) {
-          uint32_t base = 0;
-          if (lane == 0) base = slot0 + atomicAdd(&sh.cursor, total);
-          base = __shfl_sync(kFull, base, 0);
-          for (int st = 0; st * 32 < (int)tile.len; ++st) {
-            const bool cand = (flags >> st) & 1u;
-            const uint32_t b = __ballot_sync(kFull, cand);
-            if (cand) {
-              // a candidate's value is what this thread just stored (push) or the input itself (pull)
-              const uint32_t i = tile.start + st * 32 + lane;
-              const float x = MODE == kPull ? in[i] : out[i];
-              const uint32_t pos = base + __popc(b & lt);
-              ws.cand_idx[pos] = i;
-              ws.cand_val[pos] = x;
-              atomicAdd(sh.hist + (key_of(x) >> 20), 1u);
-            }
-            base += __popc(b);
-          }
-        }
+        ragged_tile<MODE>(ws, a, sh, tile, L, slot0, lane, lt, in, out);
       }
     }
     __syncthreads();
     flush_hist(sh.hist, ws.hist1 + (size_t)s * kBins1);
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    ws.part_cands[cta] = sh.cursor;
+    ws.part_slot0[cta] = slot0;
+  }
+}
+
+// The same for a tile staged in shared memory (su: the tile of the state vector, sg: the
+// tile of the gradient, push only).  The cost beyond the streaming part is kept
+// proportional to the number of candidates: one packed warp scan gives every lane the
+// rank of its candidates (lane l holds elements j*128 + l*4 + c, order is j-major, so the
+// four per-j counts travel as four bytes of one word), and a lane that has candidates
+// walks its set bits and recomputes their values from shared memory.
+template <int MODE>
+__device__ __forceinline__ void finish_full_tile_smem(const Workspace& ws, const SelArgs& a, StreamShared& sh,
+                                                      uint32_t tile_start, const float* su, const float* sg,
+                                                      uint32_t L, uint32_t slot0, int lane,
+                                                      float* __restrict__ out) {
+  const float Lf = __uint_as_float(L);   // |x| >= Lf  <=>  key(x) >= L for finite x (no flush-to-zero)
+  const float4* pu = reinterpret_cast<const float4*>(su) + lane;
+  const float4* pg = reinterpret_cast<const float4*>(sg) + lane;
+  uint32_t mask = 0;
+#pragma unroll
+  for (int j = 0; j < kVecIters; ++j) {
+    float4 x = pu[j * 32];
+    if (MODE != kPull) {
+      const float4 g = pg[j * 32];
+      x.x = combine<MODE>(x.x, g.x, a.m, a.lr);
+      x.y = combine<MODE>(x.y, g.y, a.m, a.lr);
+      x.z = combine<MODE>(x.z, g.z, a.m, a.lr);
+      x.w = combine<MODE>(x.w, g.w, a.m, a.lr);
+    }
+    const bool c0 = fabsf(x.x) >= Lf, c1 = fabsf(x.y) >= Lf, c2 = fabsf(x.z) >= Lf, c3 = fabsf(x.w) >= Lf;
+    mask |= ((c0 ? 1u : 0u) | (c1 ? 2u : 0u) | (c2 ? 4u : 0u) | (c3 ? 8u : 0u)) << (4 * j);
+    if (MODE != kPull) {
+      float4 o;
+      o.x = c0 ? x.x : unsent<MODE>(x.x, a.inv_m);
+      o.y = c1 ? x.y : unsent<MODE>(x.y, a.inv_m);
+      o.z = c2 ? x.z : unsent<MODE>(x.z, a.inv_m);
+      o.w = c3 ? x.w : unsent<MODE>(x.w, a.inv_m);
+      __stcs(reinterpret_cast<float4*>(out + tile_start) + lane + j * 32, o);
+    }
+  }
+  if (!__any_sync(kFull, mask != 0)) return;
+  // per-j candidate counts of this lane, one per byte
+  uint32_t t = mask - ((mask >> 1) & 0x5555u);
+  t = (t & 0x3333u) + ((t >> 2) & 0x3333u);                       // nibble j = count of nibble j of mask
+  const uint32_t packed = (t & 0xFu) | ((t & 0xF0u) << 4) | ((t & 0xF00u) << 8) | ((t & 0xF000u) << 12);
+  uint32_t incl = packed;                                          // byte j: inclusive prefix over lanes (<= 128)
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t o = __shfl_up_sync(kFull, incl, d);
+    if (lane >= d) incl += o;
+  }
+  const uint32_t tot = __shfl_sync(kFull, incl, 31);
+  const uint32_t t0 = tot & 0xFFu, t1 = (tot >> 8) & 0xFFu, t2 = (tot >> 16) & 0xFFu, t3 = tot >> 24;
+  uint32_t base = 0;
+  if (lane == 0) base = slot0 + atomicAdd(&sh.cursor, t0 + t1 + t2 + t3);
+  base = __shfl_sync(kFull, base, 0);
+  if (mask) {
+    const uint32_t excl = incl - packed;                           // byte j: candidates of lower lanes at step j
+    uint32_t m = mask;
+    while (m) {
+      const int e = __ffs(m) - 1;
+      m &= m - 1;
+      const int j = e >> 2, c = e & 3;
+      const uint32_t before_j = j == 0 ? 0u : (j == 1 ? t0 : (j == 2 ? t0 + t1 : t0 + t1 + t2));
+      const uint32_t in_lane = __popc((mask >> (4 * j)) & ((1u << c) - 1u));
+      const uint32_t pos = base + before_j + ((excl >> (8 * j)) & 0xFFu) + in_lane;
+      const uint32_t off = j * 128 + lane * 4 + c;
+      const float v = combine<MODE>(su[off], MODE != kPull ? sg[off] : 0.f, a.m, a.lr);
+      ws.cand_idx[pos] = tile_start + off;
+      ws.cand_val[pos] = v;
+      atomicAdd(sh.hist + (key_of(v) >> 20), 1u);
+    }
+  }
+}
+
+// ---- the same pass with TMA-staged tiles --------------------------------------------
+// Full tiles are brought into a ring of shared-memory stages by bulk asynchronous copies
+// (cp.async.bulk, completion counted on an mbarrier per stage), kStageTiles tiles of each
+// input per stage, so that several stages are in flight while the warps work on one: the
+// bytes in flight no longer depend on how many warps are waiting at a load.
+constexpr int kStageTiles = kWarps;                        // one tile per warp and stage
+constexpr int kStageFloats = kStageTiles * kWarpTile;      // per input array
+template <int MODE> struct StreamRing {
+  static constexpr int kInputs = MODE == kPull ? 1 : 2;
+  static constexpr int kStages = MODE == kPull ? 5 : 3;
+  static constexpr int kStageBytes = kInputs * kStageFloats * 4;
+  static constexpr int kBytes = kStages * kStageBytes;     // 80 KB (pull) / 96 KB (push)
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// bounded wait: false if the copies did not land within the poll limit
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  for (uint32_t spins = 0; spins < kSpinLimit; ++spins)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+// global -> shared bulk copy; src and dst 16-byte aligned, bytes a multiple of 16
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+
+template <int MODE>
+__device__ void stream_tiles_tma(const Workspace& ws, const SelArgs& a, const uint32_t* Larr,
+                                 const float* __restrict__ in, float* __restrict__ out, uint32_t cta, uint32_t G,
+                                 StreamShared& sh, float* ring, uint64_t* full, int* s_dead) {
+  using R = StreamRing<MODE>;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t t0 = part_first_tile(cta, G, ws.num_tiles), t1 = part_first_tile(cta + 1, G, ws.num_tiles);
+  const uint32_t lt = lanemask_lt();
+  for (int b = threadIdx.x; b < kBins1; b += kThreads) sh.hist[b] = 0;
+  if (threadIdx.x == 0) {
+    sh.cursor = 0;
+    *s_dead = 0;
+    if (cta == 0) ws.sync[kParts] = G;
+    for (int st = 0; st < R::kStages; ++st) mbar_init(full + st, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (t0 >= t1) {
+    if (threadIdx.x == 0) {
+      ws.part_cands[cta] = 0;
+      ws.part_slot0[cta] = 0;
+    }
+    return;
+  }
+  const uint32_t slot0 = ws.tiles[t0].start;
+  const uint32_t seg_first = ws.tiles[t0].seg, seg_last = ws.tiles[t1 - 1].seg;
+  uint32_t uses = 0;  // stage uses so far (same in every thread): stage = use % kStages, parity = (use / kStages) & 1
+  for (uint32_t s = seg_first; s <= seg_last; ++s) {
+    const uint32_t a0 = max(t0, ws.segs[s].tile_begin), a1 = min(t1, ws.segs[s].tile_end);
+    const uint32_t L = Larr[s];
+    // only the first and the last tile of a layer can be ragged
+    const bool head = ws.tiles[a0].len != kWarpTile;
+    const bool tail = (a1 - 1 > a0 || !head) && ws.tiles[a1 - 1].len != kWarpTile;
+    const uint32_t f0 = a0 + (head ? 1u : 0u), f1 = a1 - (tail ? 1u : 0u);   // full tiles [f0, f1)
+    if (head && warp == 0) ragged_tile<MODE>(ws, a, sh, ws.tiles[a0], L, slot0, lane, lt, in, out);
+    if (tail && warp == 1) ragged_tile<MODE>(ws, a, sh, ws.tiles[a1 - 1], L, slot0, lane, lt, in, out);
+    const uint32_t nfull = f1 > f0 ? f1 - f0 : 0;
+    const uint32_t nchunks = (nfull + kStageTiles - 1) / kStageTiles;
+    const uint32_t e0 = nfull ? ws.tiles[f0].start : 0;   // first element of the full tiles (multiple of kWarpTile)
+    auto issue = [&](uint32_t chunk, uint32_t use) {      // thread 0 only
+      const uint32_t st = use % R::kStages;
+      const uint32_t tiles_here = min((uint32_t)kStageTiles, nfull - chunk * kStageTiles);
+      const uint32_t bytes = tiles_here * kWarpTile * 4;
+      const size_t elem = (size_t)e0 + (size_t)chunk * kStageFloats;
+      float* dst = ring + (size_t)st * (R::kStageBytes / 4);
+      mbar_expect_tx(full + st, bytes * R::kInputs);
+      bulk_load(dst, in + elem, bytes, full + st);
+      if (MODE != kPull) bulk_load(dst + kStageFloats, a.grad + elem, bytes, full + st);
+    };
+    if (threadIdx.x == 0)
+      for (uint32_t c = 0; c < min(nchunks, (uint32_t)R::kStages); ++c) issue(c, uses + c);
+    for (uint32_t c = 0; c < nchunks; ++c) {
+      const uint32_t use = uses + c, st = use % R::kStages;
+      if (!mbar_wait(full + st, (use / R::kStages) & 1u)) *s_dead = 1;
+      const uint32_t tl = c * kStageTiles + warp;          // this warp's tile among the full ones
+      if (tl < nfull && !*s_dead) {
+        const float* su = ring + (size_t)st * (R::kStageBytes / 4) + warp * kWarpTile;
+        finish_full_tile_smem<MODE>(ws, a, sh, e0 + tl * kWarpTile, su, su + kStageFloats, L, slot0, lane, out);
+      }
+      __syncthreads();                                     // every warp is done reading this stage
+      if (*s_dead) break;
+      if (threadIdx.x == 0 && c + R::kStages < nchunks) issue(c + R::kStages, use + R::kStages);
+    }
+    if (*s_dead) break;
+    uses += nchunks;
+    __syncthreads();
+    flush_hist(sh.hist, ws.hist1 + (size_t)s * kBins1);
+    __syncthreads();
+  }
+  if (*s_dead) {
+    // a copy did not land in time: report, give the copies still in flight one more bounded wait, leave
+    if (threadIdx.x == 0) {
+      atomicMin(ws.status, kStatusTimeout);
+      for (int st = 0; st < R::kStages; ++st) {
+        mbar_wait(full + st, 0);
+        mbar_wait(full + st, 1);
+      }
+    }
     __syncthreads();
   }
   if (threadIdx.x == 0) {
@@ -456,6 +674,7 @@ __device__ bool worker_barrier(uint32_t* sync, uint32_t W, int* status, int* s_o
 // Every phase below is one flat loop over that numbering; the layer and the tile of a
 // candidate follow from its index.
 constexpr int kSegCap = 1024;  // layers whose tables fit in shared memory; more fall back to global reads
+constexpr int kBatch = 8;       // independent loads a thread issues before using any (latency-bound loops)
 
 struct FinalizeShared {
   StreamShared stream;                 // only used when the guess failed and the passes are redone here
@@ -500,6 +719,30 @@ __device__ __forceinline__ uint32_t slot_of(const FinalizeShared& sh, uint32_t p
   }
   if (part_out) *part_out = lo;
   return sh.slot0[lo] + (p - sh.pre_cands[lo]);
+}
+
+// Walks the flat numbering: a thread (or a lane) owns consecutive flat candidates, finds
+// the first one by binary search and then only steps.
+struct Cursor {
+  uint32_t part, slot, left;   // part of the current candidate, its slot, candidates left in that part (>= 1 if valid)
+};
+__device__ __forceinline__ Cursor cursor_at(const FinalizeShared& sh, uint32_t parts, uint32_t p) {
+  Cursor c;
+  c.slot = slot_of(sh, parts, p, &c.part);
+  c.left = sh.pre_cands[c.part + 1] - p;
+  return c;
+}
+// advance by n candidates; the caller never advances past the last candidate + 1
+__device__ __forceinline__ void cursor_advance(const FinalizeShared& sh, uint32_t parts, Cursor& c, uint32_t n) {
+  while (n >= c.left) {
+    n -= c.left;
+    do { ++c.part; } while (c.part < parts && sh.pre_cands[c.part + 1] == sh.pre_cands[c.part]);
+    if (c.part >= parts) { c.left = 0xFFFFFFFFu; c.slot = 0; return; }   // ran off the end: never dereferenced
+    c.slot = sh.slot0[c.part];
+    c.left = sh.pre_cands[c.part + 1] - sh.pre_cands[c.part];
+  }
+  c.slot += n;
+  c.left -= n;
 }
 
 template <int MODE>
@@ -592,22 +835,32 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
   // flat numbering of the candidates
   const uint32_t parts = ld_volatile(ws.sync + kParts);
   {
+    constexpr int PER = kMaxGrid / kThreads;   // parts <= kMaxGrid
+    uint32_t cnt[PER];
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      const uint32_t p = j * kThreads + threadIdx.x;
+      cnt[j] = p < parts ? __ldcg(ws.part_cands + p) : 0;
+      if (p < parts) sh.slot0[p] = __ldcg(ws.part_slot0 + p);
+    }
     unsigned long long carry = 0;
-    for (uint32_t base = 0; base < parts; base += kThreads) {
-      const uint32_t p = base + threadIdx.x;
-      const unsigned long long v = p < parts ? __ldcg(ws.part_cands + p) : 0;
-      unsigned long long total;
-      const unsigned long long ex = block_excl_scan(v, sh.warp_scan, total) + carry;
-      if (p < parts) {
-        sh.pre_cands[p] = (uint32_t)ex;
-        sh.slot0[p] = __ldcg(ws.part_slot0 + p);
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      if ((uint32_t)(j * kThreads) < parts) {   // CTA-uniform
+        const uint32_t p = j * kThreads + threadIdx.x;
+        unsigned long long total;
+        const unsigned long long ex = block_excl_scan(cnt[j], sh.warp_scan, total) + carry;
+        if (p < parts) sh.pre_cands[p] = (uint32_t)ex;
+        carry += total;
       }
-      carry += total;
     }
     if (threadIdx.x == 0) sh.pre_cands[parts] = (uint32_t)carry;
     __syncthreads();
   }
   const uint32_t C = sh.pre_cands[parts];
+  // every thread owns the flat candidates [my_lo, my_hi)
+  const uint32_t per_thread = (C + nthreads - 1) / nthreads;
+  const uint32_t my_lo = min(C, gthread * per_thread), my_hi = min(C, my_lo + per_thread);
 
   // ---- levels 2 and 3 ----------------------------------------------------------------
 #pragma unroll 1
@@ -619,13 +872,49 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
       for (uint32_t s = threadIdx.x; s < S; s += kThreads) sh.seg_a[s] = __ldcg(&ws.sel[s].prefix);
       __syncthreads();
     }
-    for (uint32_t p = gthread; p < C; p += nthreads) {
-      const uint32_t slot = slot_of(sh, parts, p, nullptr);
-      const uint32_t key = key_of(__ldcg(ws.cand_val + slot));
-      uint32_t seg = 0;
-      if (S > 1) seg = seg_of(sv, __ldcg(ws.cand_idx + slot));
-      const uint32_t prefix = seg_smem ? sh.seg_a[seg] : __ldcg(&ws.sel[seg].prefix);
-      if ((key >> SH) == prefix) atomicAdd(hist + (size_t)seg * B + ((key >> (SH - 10)) & 1023u), 1u);
+    if (S == 1) {
+      for (int b = threadIdx.x; b < B; b += kThreads) sh.stream.hist[b] = 0;
+      __syncthreads();
+    }
+    if (my_lo < my_hi) {
+      Cursor cur = cursor_at(sh, parts, my_lo);
+      for (uint32_t p = my_lo; p < my_hi; p += kBatch) {
+        // all loads of the batch are issued before any loaded value is touched (a use right
+        // after its load would make the loads wait for one another)
+        float raw[kBatch];
+        uint32_t key[kBatch], idx[kBatch];
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+          raw[u] = 0.f;
+          idx[u] = 0;
+          if (p + u < my_hi) {
+            raw[u] = __ldcg(ws.cand_val + cur.slot);
+            if (S > 1) idx[u] = __ldcg(ws.cand_idx + cur.slot);
+            cursor_advance(sh, parts, cur, 1);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) key[u] = key_of(raw[u]);
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+          if (p + u < my_hi) {
+            const uint32_t seg = S > 1 ? seg_of(sv, idx[u]) : 0;
+            const uint32_t prefix = seg_smem ? sh.seg_a[seg] : __ldcg(&ws.sel[seg].prefix);
+            if ((key[u] >> SH) == prefix) {
+              const uint32_t digit = (key[u] >> (SH - 10)) & 1023u;
+              if (S == 1) atomicAdd(sh.stream.hist + digit, 1u);       // one layer: CTA-private histogram first
+              else atomicAdd(hist + (size_t)seg * B + digit, 1u);
+            }
+          }
+        }
+      }
+    }
+    if (S == 1) {
+      __syncthreads();
+      for (int b = threadIdx.x; b < B; b += kThreads) {
+        const uint32_t v = sh.stream.hist[b];
+        if (v) atomicAdd(hist + b, v);
+      }
     }
     if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
     for (uint32_t s = cta; s < S; s += W) {
@@ -655,15 +944,34 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
     }
     __syncthreads();
   }
-  for (uint32_t p = gthread; p < C; p += nthreads) {
-    const uint32_t slot = slot_of(sh, parts, p, nullptr);
-    const uint32_t key = key_of(__ldcg(ws.cand_val + slot));
-    const uint32_t idx = __ldcg(ws.cand_idx + slot);
-    const uint32_t seg = S > 1 ? seg_of(sv, idx) : 0;
-    const uint32_t T = seg_smem ? sh.seg_a[seg] : __ldcg(&ws.sel[seg].T);
-    if (key >= T) {
-      uint2* c = ws.tile_sel + tile_of(sv, seg, idx);
-      atomicAdd(key > T ? &c->x : &c->y, 1u);
+  if (my_lo < my_hi) {
+    Cursor cur = cursor_at(sh, parts, my_lo);
+    for (uint32_t p = my_lo; p < my_hi; p += kBatch) {
+      float raw[kBatch];
+      uint32_t key[kBatch], idx[kBatch];
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) {
+        raw[u] = 0.f;
+        idx[u] = 0;
+        if (p + u < my_hi) {
+          raw[u] = __ldcg(ws.cand_val + cur.slot);
+          idx[u] = __ldcg(ws.cand_idx + cur.slot);
+          cursor_advance(sh, parts, cur, 1);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) key[u] = key_of(raw[u]);
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) {
+        if (p + u < my_hi) {
+          const uint32_t seg = S > 1 ? seg_of(sv, idx[u]) : 0;
+          const uint32_t T = seg_smem ? sh.seg_a[seg] : __ldcg(&ws.sel[seg].T);
+          if (key[u] >= T) {
+            uint2* c = ws.tile_sel + tile_of(sv, seg, idx[u]);
+            atomicAdd(key[u] > T ? &c->x : &c->y, 1u);
+          }
+        }
+      }
     }
   }
   if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
@@ -673,18 +981,28 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
   {
     const uint32_t t0 = min(ws.num_tiles, cta * chunk_tiles), t1 = min(ws.num_tiles, t0 + chunk_tiles);
     unsigned long long carry = 0;
-    for (uint32_t base = t0; base < t1; base += kThreads) {
-      const uint32_t t = base + threadIdx.x;
-      unsigned long long v = 0;
-      if (t < t1) {
-        const uint2 c = __ldcg(ws.tile_sel + t);
-        v = ((unsigned long long)c.x << 32) | c.y;
-        if (v) ws.tile_sel[t] = make_uint2(0, 0);
+    for (uint32_t base0 = t0; base0 < t1; base0 += kThreads * kBatch) {
+      unsigned long long v[kBatch];
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) {
+        const uint32_t t = base0 + u * kThreads + threadIdx.x;
+        v[u] = 0;
+        if (t < t1) {
+          const uint2 c = __ldcg(ws.tile_sel + t);
+          v[u] = ((unsigned long long)c.x << 32) | c.y;
+        }
       }
-      unsigned long long total;
-      const unsigned long long ex = block_excl_scan(v, sh.warp_scan, total) + carry;
-      if (t < t1) ws.tile_pre[t] = make_uint2((uint32_t)(ex >> 32), (uint32_t)ex);
-      carry += total;
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) {
+        if (base0 + u * kThreads < t1) {   // CTA-uniform
+          const uint32_t t = base0 + u * kThreads + threadIdx.x;
+          if (v[u]) ws.tile_sel[t] = make_uint2(0, 0);
+          unsigned long long total;
+          const unsigned long long ex = block_excl_scan(v[u], sh.warp_scan, total) + carry;
+          if (t < t1) ws.tile_pre[t] = make_uint2((uint32_t)(ex >> 32), (uint32_t)ex);
+          carry += total;
+        }
+      }
     }
     if (threadIdx.x == 0) ws.cta_tot[cta] = make_uint2((uint32_t)(carry >> 32), (uint32_t)carry);
   }
@@ -715,21 +1033,30 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
       for (uint32_t s = threadIdx.x; s < S; s += kThreads) sh.seg_start[s] = before_tile(sh.seg_tile0[s]);
       __syncthreads();
     }
+    // every warp owns a run of consecutive flat candidates, 32 per step
     const uint32_t gwarp = cta * kWarps + warp, nwarps = W * kWarps;
-    for (uint32_t c0 = gwarp * 32; c0 < C; c0 += nwarps * 32) {
+    const uint32_t per_warp = ((C + nwarps - 1) / nwarps + 31) / 32 * 32;
+    const uint32_t w_lo = min(C, gwarp * per_warp), w_hi = min(C, w_lo + per_warp);
+    Cursor cur;
+    cur.part = 0; cur.slot = 0; cur.left = 0xFFFFFFFFu;
+    if (w_lo + lane < w_hi) cur = cursor_at(sh, parts, w_lo + lane);
+    // counts carried from the previous step for the tile its last lane was in
+    uint32_t carry_gt = 0, carry_eq = 0, carry_tile = 0xFFFFFFFFu, carry_part = 0xFFFFFFFFu;
+    for (uint32_t c0 = w_lo; c0 < w_hi; c0 += 32) {
       const uint32_t p = c0 + lane;
-      const bool valid = p < C;
-      uint32_t part = 0, idx = 0, key = 0, seg = 0, tile = 0xFFFFFFFFu, T = 0, r = 0;
+      const bool valid = p < w_hi;
+      uint32_t part = 0xFFFFFFFEu, idx = 0, key = 0, seg = 0, tile = 0xFFFFFFFFu, T = 0, r = 0;
       float val = 0.f;
       if (valid) {
-        const uint32_t slot = slot_of(sh, parts, p, &part);
-        idx = __ldcg(ws.cand_idx + slot);
-        val = __ldcg(ws.cand_val + slot);
+        part = cur.part;
+        idx = __ldcg(ws.cand_idx + cur.slot);
+        val = __ldcg(ws.cand_val + cur.slot);
         key = key_of(val);
         seg = S > 1 ? seg_of(sv, idx) : 0;
         tile = tile_of(sv, seg, idx);
         T = seg_smem ? sh.seg_a[seg] : __ldcg(&ws.sel[seg].T);
         r = seg_smem ? sh.seg_b[seg] : __ldcg(&ws.sel[seg].r);
+        if (p + 32 < w_hi) cursor_advance(sh, parts, cur, 32);
       }
       const bool is_gt = valid && key > T, is_eq = valid && key == T;
       const uint32_t bgt = __ballot_sync(kFull, is_gt), beq = __ballot_sync(kFull, is_eq);
@@ -738,10 +1065,16 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
       const uint32_t heads = __ballot_sync(kFull, lane == 0 || left != tile);
       const int head = 31 - __clz(heads & (lt | (1u << lane)));       // first lane of my tile in this step
       const uint32_t mine = lt & ~((1u << head) - 1u);                  // lanes of my tile before me
-      // the tile of lane 0 may have started in earlier slots of the same part: count what it holds there
-      uint32_t carry_gt = 0, carry_eq = 0;
-      {
-        const uint32_t tile0 = __shfl_sync(kFull, tile, 0), part0 = __shfl_sync(kFull, part, 0);
+      // what the tile of lane 0 holds in earlier slots
+      const uint32_t tile0 = __shfl_sync(kFull, tile, 0), part0 = __shfl_sync(kFull, part, 0);
+      uint32_t pre_gt = 0, pre_eq = 0;
+      if (c0 != w_lo) {
+        if (carry_tile == tile0 && carry_part == part0) {
+          pre_gt = carry_gt;
+          pre_eq = carry_eq;
+        }
+      } else {
+        // first step of this warp: the tile may have begun in slots that belong to the previous warp
         const uint32_t T0 = __shfl_sync(kFull, T, 0), seg0 = __shfl_sync(kFull, seg, 0);
         const uint32_t first = sh.pre_cands[part0];                     // flat number of the part's first candidate
         uint32_t back = c0;
@@ -758,8 +1091,8 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
             k2 = key_of(__ldcg(ws.cand_val + slot));
           }
           const uint32_t bs = __ballot_sync(kFull, same);
-          carry_gt += __popc(__ballot_sync(kFull, same && k2 > T0));
-          carry_eq += __popc(__ballot_sync(kFull, same && k2 == T0));
+          pre_gt += __popc(__ballot_sync(kFull, same && k2 > T0));
+          pre_eq += __popc(__ballot_sync(kFull, same && k2 == T0));
           if (bs != __ballot_sync(kFull, pp < back)) break;             // reached another tile
           back = lo;
         }
@@ -770,8 +1103,8 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
         uint32_t gt_before = (tb.x - s0.x) + __popc(bgt & mine);
         uint32_t eq_before = (tb.y - s0.y) + __popc(beq & mine);
         if (head == 0) {
-          gt_before += carry_gt;
-          eq_before += carry_eq;
+          gt_before += pre_gt;
+          eq_before += pre_eq;
         }
         const bool sel = is_gt || (is_eq && eq_before < r);
         if (sel) {
@@ -790,6 +1123,15 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
         } else {
           if (MODE == kPushSam) out[idx] = __fmul_rn(val, a.inv_m);  // Eq. 12, lower branch
         }
+      }
+      // carry for the next step: counts of the tile that lane 31 is in (all lanes of a full step are valid)
+      {
+        const int head31 = 31 - __clz(heads);
+        const uint32_t tail_lanes = ~((1u << head31) - 1u);
+        carry_gt = __popc(bgt & tail_lanes) + (head31 == 0 ? pre_gt : 0u);
+        carry_eq = __popc(beq & tail_lanes) + (head31 == 0 ? pre_eq : 0u);
+        carry_tile = __shfl_sync(kFull, tile, 31);
+        carry_part = __shfl_sync(kFull, part, 31);
       }
     }
   }
@@ -828,8 +1170,11 @@ __global__ void __launch_bounds__(kThreads) k_pick_lower(Workspace ws) {
 
 // ---- stand-alone stream pass with the carried bound -------------------------------
 template <int MODE>
-__global__ void __launch_bounds__(kThreads, 4) k_stream(Workspace ws, SelArgs a) {
+__global__ void __launch_bounds__(kThreads, 2) k_stream(Workspace ws, SelArgs a) {
+  extern __shared__ __align__(128) unsigned char dyn_smem[];   // the ring of stages
   __shared__ StreamShared sh;
+  __shared__ __align__(8) uint64_t full[StreamRing<MODE>::kStages];
+  __shared__ int s_dead;
   const float* in;
   float* out = nullptr;
   if (MODE == kPull) {
@@ -838,7 +1183,8 @@ __global__ void __launch_bounds__(kThreads, 4) k_stream(Workspace ws, SelArgs a)
     in = *a.u_cur_slot;
     out = *a.u_spare_slot;
   }
-  stream_tiles<MODE>(ws, a, a.L_in, in, out, blockIdx.x, gridDim.x, sh);
+  stream_tiles_tma<MODE>(ws, a, a.L_in, in, out, blockIdx.x, gridDim.x, sh, reinterpret_cast<float*>(dyn_smem), full,
+                         &s_dead);
 }
 
 // ---- server apply ---------------------------------------------------------------
