@@ -246,6 +246,7 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
 
     run_events(0, preroll)
     run_events(preroll, Wm)
+    ctx.flush()
     stats0 = ctx.stats()
     launches0 = ctx.launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -253,6 +254,7 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
     with ClockSampler(local_rank) as clocks:
         ev0.record(stream)
         run_events(preroll + Wm, K)
+        ctx.flush()
         ev1.record(stream)
         barrier()
     elapsed = ev0.elapsed_time(ev1) * 1e-3

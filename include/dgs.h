@@ -25,10 +25,14 @@
  *     Exactly k_j entries are kept per layer; among equal magnitudes the lowest
  *     index wins.  Packets list (index, value) pairs in ascending index order.
  *   - DEVICE pointers are marked DEVICE, everything else is host memory.
- *   - The caller owns all device memory (the arena) and the stream; the library
- *     allocates no device memory.  Calls only enqueue work on the stream given at
- *     dgs_init and return; results are ready when the stream reaches them.
- *     One host thread per context.
+ *   - The caller owns all device memory (the arena); the library allocates no device
+ *     memory.  Calls only enqueue work and return.  The work runs on two streams of the
+ *     library's own (one for the pushes, one for apply and pull, so that the push of the
+ *     next event overlaps the server side of the current one); it is ordered after
+ *     everything the caller had enqueued on the stream given at dgs_init when the call
+ *     was made.  Results (packets, state) are complete for that stream after dgs_flush,
+ *     and for the host after any call that is documented to wait.  One host thread per
+ *     context.
  *   - Every function returns DGS_OK (0) or a negative dgs_error.  Nothing aborts,
  *     throws or waits without bound.
  */
@@ -110,8 +114,9 @@ int dgs_arena_bytes(const dgs_config* cfg, uint64_t* out_bytes);
 int dgs_init(const dgs_config* cfg, dgs_ctx** out);
 
 /* Worker push (Algorithm 3, velocity update through encode(); Eq. 11a, Eq. 12).
- * grad: DEVICE f32[n], 16-byte aligned, read only, must stay valid until the
- * stream has run this call.  On return *out describes the push packet slot. */
+ * grad: DEVICE f32[n], 16-byte aligned, read only, must stay valid until the work of
+ * this call has run (dgs_flush, then the stream reaching that point).  On return *out
+ * describes the push packet slot (two slots are used alternately). */
 int dgs_worker_push(dgs_ctx* ctx, uint32_t worker, const float* grad, dgs_packet* out);
 
 /* Server apply (Algorithm 2, "M <- M - decode(g)"; Eq. 1-3): theta[i] -= val and
@@ -130,15 +135,20 @@ int dgs_worker_pull(dgs_ctx* ctx, uint32_t worker, dgs_packet* out);
  * pointer may be NULL. */
 int dgs_event(dgs_ctx* ctx, uint32_t worker, const float* grad, dgs_packet* push_out, dgs_packet* pull_out);
 
+/* Makes the stream given at dgs_init wait (on the device, not the host) for all work
+ * enqueued by earlier calls: what that stream runs afterwards sees their packets and
+ * state.  (No counterpart in the paper: it joins the library's two streams.) */
+int dgs_flush(dgs_ctx* ctx);
+
 /* The same event with HOST buffers (needs DGS_HOST_IO): copies grad (HOST f32[n],
  * ideally pinned) to the device, runs the event, copies the pull packet back into
  * out_idx / out_val (HOST, sum(k_pull) entries each, may be NULL to skip) and
- * waits for the stream.  This is the end-to-end path: what a worker process
+ * waits for that work.  This is the end-to-end path: what a worker process
  * without its own device buffers would call. */
 int dgs_event_host(dgs_ctx* ctx, uint32_t worker, const float* grad_host, uint32_t* out_idx, float* out_val);
 
 /* Pointer to a state vector, DEVICE f32[n]: which = DGS_THETA (worker ignored),
- * DGS_U, DGS_D or DGS_THETA_LOCAL.  Waits for the stream (velocity buffers are
+ * DGS_U, DGS_D or DGS_THETA_LOCAL.  Waits for all work in flight (velocity buffers are
  * exchanged with a spare on the device, so their address is only known then).
  * The pointer is valid until the next push of that worker (DGS_U) or dgs_free. */
 int dgs_state_ptr(dgs_ctx* ctx, int which, uint32_t worker, const float** out);
@@ -147,12 +157,12 @@ int dgs_state_ptr(dgs_ctx* ctx, int which, uint32_t worker, const float** out);
  * checkpoint, or loads a vector to be selected from with dgs_worker_pull. */
 int dgs_state_load(dgs_ctx* ctx, int which, uint32_t worker, const float* src);
 
-/* Waits for the stream and returns the sticky device status word in
+/* Waits for all work in flight and returns the sticky device status word in
  * *device_status (0 = clean; negative dgs_error values are stored by kernels that
  * detect an out-of-range index or give up a bounded wait). */
 int dgs_status(dgs_ctx* ctx, int* device_status);
 
-/* Waits for the stream and reports counters: out[0] selections served by the
+/* Waits for all work in flight and reports counters: out[0] selections served by the
  * single-pass (speculative) route, out[1] selections that took the two-pass
  * route, out[2] server timestamp t (packets applied), out[3] candidates the finalize
  * steps have examined in total (the k selected ones included). */
@@ -181,7 +191,7 @@ enum {
  * 65536 launches between two reads are recorded). */
 int dgs_timing_enable(dgs_ctx* ctx, int on);
 
-/* Waits for the stream; ms[i] / count[i] receive the summed device time in
+/* Waits for all work in flight; ms[i] / count[i] receive the summed device time in
  * milliseconds and the number of recorded launches of kernel i since the last
  * read, and the accumulators restart from zero. */
 int dgs_timing_read(dgs_ctx* ctx, double ms[DGS_NUM_KERNELS], uint64_t count[DGS_NUM_KERNELS]);
@@ -189,7 +199,7 @@ int dgs_timing_read(dgs_ctx* ctx, double ms[DGS_NUM_KERNELS], uint64_t count[DGS
 /* The cudaError_t of the last failed runtime call of this context (0 if none). */
 int dgs_last_cuda_error(dgs_ctx* ctx);
 
-/* Frees the host-side context.  The arena stays the caller's.  Waits for the stream. */
+/* Frees the host-side context.  The arena stays the caller's.  Waits for all work in flight. */
 int dgs_free(dgs_ctx* ctx);
 
 /* Largest vector dgs_topk_encode_static accepts (elements). */

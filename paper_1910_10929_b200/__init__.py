@@ -21,7 +21,7 @@ DGS_THETA, DGS_U, DGS_D, DGS_THETA_LOCAL = 0, 1, 2, 3
 
 EXPORTS = (
     "dgs_arena_bytes", "dgs_init", "dgs_worker_push", "dgs_server_apply", "dgs_worker_pull",
-    "dgs_event", "dgs_event_host", "dgs_state_ptr", "dgs_state_load", "dgs_status", "dgs_stats",
+    "dgs_event", "dgs_flush", "dgs_event_host", "dgs_state_ptr", "dgs_state_load", "dgs_status", "dgs_stats",
     "dgs_prev", "dgs_launch_count", "dgs_last_cuda_error", "dgs_free", "dgs_error_string",
     "dgs_timing_enable", "dgs_timing_read", "dgs_topk_encode_static",
 )
@@ -70,6 +70,7 @@ def lib() -> C.CDLL:
         L.dgs_server_apply.argtypes = [vp, u32, C.POINTER(dgs_packet)]
         L.dgs_worker_pull.argtypes = [vp, u32, C.POINTER(dgs_packet)]
         L.dgs_event.argtypes = [vp, u32, vp, C.POINTER(dgs_packet), C.POINTER(dgs_packet)]
+        L.dgs_flush.argtypes = [vp]
         L.dgs_event_host.argtypes = [vp, u32, vp, vp, vp]
         L.dgs_state_ptr.argtypes = [vp, i32, u32, C.POINTER(vp)]
         L.dgs_state_load.argtypes = [vp, i32, u32, vp]
@@ -142,6 +143,10 @@ def dgs_event(ctx: int, worker: int, grad_ptr: int) -> Tuple[dgs_packet, dgs_pac
     p, g = dgs_packet(), dgs_packet()
     _check(lib().dgs_event(ctx, worker, grad_ptr, C.byref(p), C.byref(g)), "dgs_event")
     return p, g
+
+
+def dgs_flush(ctx: int) -> None:
+    _check(lib().dgs_flush(ctx), "dgs_flush")
 
 
 def dgs_event_host(ctx: int, worker: int, grad_host_ptr: int, out_idx_ptr: int = 0, out_val_ptr: int = 0) -> None:

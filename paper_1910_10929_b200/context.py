@@ -74,8 +74,14 @@ class Context:
         assert 0 <= off and off + 4 * count <= self.arena_bytes
         return self.arena[off:off + 4 * count].view(dtype)
 
+    def flush(self) -> None:
+        """Orders the context's stream after all work enqueued so far."""
+        dgs.dgs_flush(self.handle)
+
     def packet(self, pkt: "dgs.dgs_packet") -> Tuple[torch.Tensor, torch.Tensor]:
-        """(idx int32 view holding uint32 bits, val float32) views of a packet slot."""
+        """(idx int32 view holding uint32 bits, val float32) views of a packet slot, readable on
+        the context's stream (flushes first)."""
+        self.flush()
         return self._view(pkt.idx, pkt.count, torch.int32), self._view(pkt.val, pkt.count, torch.float32)
 
     def state(self, which: int, worker: int = 0) -> torch.Tensor:

@@ -1,5 +1,13 @@
 // Host side of the C ABI declared in include/dgs.h: argument checks, the layout of
 // the caller's arena, and the kernel launches of one push / apply / pull event.
+//
+// Work runs on two streams of the library's own.  The worker stream takes the pushes
+// (stream pass + finalize), the server stream takes apply and pull.  A push touches only
+// the worker's velocity, the gradient and its own scratch, so the push of the next event
+// runs while the server side of the current one is still busy; the small, latency-bound
+// finalize kernels then share the GPU with the bandwidth-bound passes of the other stream.
+// Order between the two is kept with CUDA events: an apply waits for the push that made
+// its packet, and a push that reuses a packet slot waits for the apply that read it.
 #include "dgs.h"
 
 #include <algorithm>
@@ -18,18 +26,27 @@ namespace {
 
 constexpr uint64_t kAlign = 256;
 constexpr uint32_t kMagic = 0x44475331u;  // "DGS1"
-constexpr uint32_t kNoBound = 0xFFFFFFFFu;
+constexpr int kPushSlots = 2;             // push packet slots, used alternately
 
 inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+// Scratch of one selection pipeline ([0] push, on the worker stream; [1] pull, on the server stream)
+struct ScratchLayout {
+  uint64_t cand_idx, cand_val, part_cands, part_slot0, tile_pre, cta_tot, tile_sel;
+  uint64_t hist1, hist2, hist3, sel, L_safe, sync;
+  uint64_t zero_begin, zero_end;  // [tile_sel, end of sync): cleared at init
+};
 
 struct Layout {
   uint64_t n_pad = 0;  // elements per state vector, padded to 256 bytes
   uint32_t num_tiles = 0;
   uint64_t K[2] = {0, 0};
   // byte offsets into the arena
-  uint64_t theta, u, D, theta_local, grad_stage, pkt_idx[2], pkt_val[2];
-  uint64_t cand_idx, cand_val, tiles, segs, part_cands, part_slot0, seg_off, seg_tile0, tile_pre, cta_tot, tile_sel;
-  uint64_t hist1, hist2, hist3, sel, L_safe, L_next, u_slots, sync, status, stats;
+  uint64_t theta, u, D, theta_local, grad_stage;
+  uint64_t pkt_idx[kPushSlots + 1], pkt_val[kPushSlots + 1];  // push slots, then the pull slot
+  uint64_t tiles, segs, seg_off, seg_tile0;
+  ScratchLayout sc[2];
+  uint64_t L_next, u_slots, status, stats;
   uint64_t total = 0;
 };
 
@@ -58,18 +75,16 @@ void build_tiles(const dgs_config* c, std::vector<Tile>* tiles, std::vector<SegD
   for (uint32_t s = 0; s < c->num_segments; ++s) {
     const dgs_segment& g = c->segments[s];
     SegDesc d;
-    d.tile_begin = tiles ? (uint32_t)tiles->size() : 0;
+    d.tile_begin = (uint32_t)tiles->size();
     uint64_t pos = g.offset, end = g.offset + g.len;
     uint32_t count = 0;
     while (pos < end) {
       const uint64_t next = std::min<uint64_t>(end, (pos / kWarpTile + 1) * kWarpTile);
-      if (tiles) {
-        Tile t;
-        t.start = (uint32_t)pos;
-        t.len = (uint16_t)(next - pos);
-        t.seg = (uint16_t)s;
-        tiles->push_back(t);
-      }
+      Tile t;
+      t.start = (uint32_t)pos;
+      t.len = (uint16_t)(next - pos);
+      t.seg = (uint16_t)s;
+      tiles->push_back(t);
       ++count;
       pos = next;
     }
@@ -80,7 +95,7 @@ void build_tiles(const dgs_config* c, std::vector<Tile>* tiles, std::vector<SegD
     d.pkt_off[1] = koff[1];
     koff[0] += g.k_push;
     koff[1] += g.k_pull;
-    if (segs) segs->push_back(d);
+    segs->push_back(d);
   }
 }
 
@@ -115,29 +130,35 @@ void make_layout(const dgs_config* c, Layout* L) {
   L->D = take(vec * N);
   L->theta_local = (c->flags & DGS_KEEP_LOCAL_MODEL) ? take(vec * N) : 0;
   L->grad_stage = (c->flags & DGS_HOST_IO) ? take(vec) : 0;
-  for (int p = 0; p < 2; ++p) {
-    L->pkt_idx[p] = take(L->K[p] * 4);
-    L->pkt_val[p] = take(L->K[p] * 4);
+  for (int p = 0; p <= kPushSlots; ++p) {
+    const uint64_t K = L->K[p < kPushSlots ? 0 : 1];
+    L->pkt_idx[p] = take(K * 4);
+    L->pkt_val[p] = take(K * 4);
   }
-  L->cand_idx = take(vec);
-  L->cand_val = take(vec);
   L->tiles = take((uint64_t)L->num_tiles * sizeof(Tile));
   L->segs = take(S * sizeof(SegDesc));
-  L->part_cands = take((uint64_t)kMaxGrid * 4);
-  L->part_slot0 = take((uint64_t)kMaxGrid * 4);
   L->seg_off = take((S + 1) * 4);
   L->seg_tile0 = take(S * 4);
-  L->tile_pre = take((uint64_t)L->num_tiles * sizeof(uint2));
-  L->cta_tot = take((uint64_t)kMaxWorkers * sizeof(uint2));
-  L->tile_sel = take((uint64_t)L->num_tiles * sizeof(uint2));
-  L->hist1 = take(S * kBins1 * 4);
-  L->hist2 = take(S * kBins2 * 4);
-  L->hist3 = take(S * kBins3 * 4);
-  L->sel = take(S * sizeof(SegSel));
-  L->L_safe = take(S * 4);
+  for (int k = 0; k < 2; ++k) {
+    ScratchLayout& sc = L->sc[k];
+    sc.cand_idx = take(vec);
+    sc.cand_val = take(vec);
+    sc.part_cands = take((uint64_t)kMaxGrid * 4);
+    sc.part_slot0 = take((uint64_t)kMaxGrid * 4);
+    sc.tile_pre = take((uint64_t)L->num_tiles * sizeof(uint2));
+    sc.cta_tot = take((uint64_t)kMaxWorkers * sizeof(uint2));
+    sc.tile_sel = take((uint64_t)L->num_tiles * sizeof(uint2));
+    sc.zero_begin = sc.tile_sel;
+    sc.hist1 = take(S * kBins1 * 4);
+    sc.hist2 = take(S * kBins2 * 4);
+    sc.hist3 = take(S * kBins3 * 4);
+    sc.sel = take(S * sizeof(SegSel));
+    sc.L_safe = take(S * 4);
+    sc.sync = take(kNumSyncWords * 4);
+    sc.zero_end = off;
+  }
   L->L_next = take(2 * N * S * 4);
   L->u_slots = take((N + 1) * sizeof(float*));
-  L->sync = take(kNumSyncWords * 4);
   L->status = take(4);
   L->stats = take(32 * 8);
   L->total = off;
@@ -151,13 +172,20 @@ struct dgs_ctx {
   std::vector<dgs_segment> segments;
   Layout lay;
   char* base;
-  cudaStream_t stream;
-  Workspace ws;
+  cudaStream_t user;       // the caller's stream: entry point of dependencies, target of dgs_flush
+  cudaStream_t st[2];      // [0] worker stream (push), [1] server stream (apply, pull)
+  cudaEvent_t ev_in;       // "everything the caller had enqueued when the call was made"
+  cudaEvent_t ev_push[kPushSlots];   // push packet in slot i is complete
+  cudaEvent_t ev_apply[kPushSlots];  // the apply that read slot i is done
+  bool apply_pending[kPushSlots];    // ev_apply[i] has been recorded since slot i was last written
+  cudaEvent_t ev_tail[2];  // for dgs_flush
+  uint64_t push_count;
+  Workspace ws[2];         // [0] push pipeline, [1] pull pipeline
   float inv_m;
   int stream_grid[3];    // CTAs of the stand-alone stream pass, per mode
   int hist_grid[3];      // CTAs of the whole-input histogram pass, per mode
   int finalize_grid[3];  // CTAs of the cooperative finalize kernel, per mode
-  uint32_t select_seq;   // selections launched so far (tags the decision word of each finalize launch)
+  uint32_t select_seq;   // selections launched so far
   // Carried bounds: row (kind, worker) of L_next holds the bounds suggested by that worker's
   // latest selection of that kind ([0] push, [1] pull).  row_age says in which state it was
   // made: pushes the worker had done before (push), packets accumulated in D_w since its
@@ -171,7 +199,7 @@ struct dgs_ctx {
   uint64_t launches;
   int last_cuda;
   bool broken;
-  // optional per-kernel timing (CUDA events on the context's stream)
+  // optional per-kernel timing (CUDA events on the launching stream)
   bool timing;
   std::vector<cudaEvent_t> ev_pool;   // pairs: [2i] start, [2i+1] stop
   std::vector<int> ev_kernel;         // kernel id of each recorded pair
@@ -213,8 +241,9 @@ constexpr int kFinalizeWorkers = 64;  // CTAs of the finalize kernel
 // Records an event before and after one launch when timing is on.
 struct TimedLaunch {
   dgs_ctx* c;
+  cudaStream_t st;
   cudaEvent_t stop = nullptr;
-  TimedLaunch(dgs_ctx* ctx, int kernel_id) : c(ctx) {
+  TimedLaunch(dgs_ctx* ctx, cudaStream_t stream, int kernel_id) : c(ctx), st(stream) {
     if (!c->timing || c->ev_kernel.size() >= kMaxTimedLaunches) return;
     const size_t i = c->ev_kernel.size();
     while (c->ev_pool.size() < 2 * (i + 1)) {
@@ -222,14 +251,29 @@ struct TimedLaunch {
       if (cudaEventCreate(&e) != cudaSuccess) return;
       c->ev_pool.push_back(e);
     }
-    if (cudaEventRecord(c->ev_pool[2 * i], c->stream) != cudaSuccess) return;
+    if (cudaEventRecord(c->ev_pool[2 * i], st) != cudaSuccess) return;
     stop = c->ev_pool[2 * i + 1];
     c->ev_kernel.push_back(kernel_id);
   }
   ~TimedLaunch() {
-    if (stop) cudaEventRecord(stop, c->stream);
+    if (stop) cudaEventRecord(stop, st);
   }
 };
+
+// Makes internal stream `which` wait for everything the caller has enqueued on its stream so far.
+int fork_from_user(dgs_ctx* c, int which) {
+  DGS_CUDA(c, cudaEventRecord(c->ev_in, c->user));
+  DGS_CUDA(c, cudaStreamWaitEvent(c->st[which], c->ev_in, 0));
+  return DGS_OK;
+}
+
+// Waits (on the host) for both internal streams and the caller's stream.
+int sync_all(dgs_ctx* c) {
+  DGS_CUDA(c, cudaStreamSynchronize(c->st[0]));
+  DGS_CUDA(c, cudaStreamSynchronize(c->st[1]));
+  DGS_CUDA(c, cudaStreamSynchronize(c->user));
+  return DGS_OK;
+}
 
 // Most recent row of this kind made at an age <= `age`; -1 if there is none.
 int pick_row(const dgs_ctx* c, int kind, uint64_t age) {
@@ -244,6 +288,8 @@ int pick_row(const dgs_ctx* c, int kind, uint64_t age) {
 template <int MODE>
 int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age) {
   constexpr int KIND = MODE == kPull ? 1 : 0;
+  cudaStream_t st = c->st[KIND];
+  Workspace& ws = c->ws[KIND];
   SelArgs a = a_in;
   a.speculate = (c->cfg.flags & DGS_NO_SPECULATION) ? 0 : 1;
   const int row = a.speculate ? pick_row(c, KIND, age) : -1;
@@ -256,27 +302,27 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age
     a.L_in = c->L_next(KIND, (uint32_t)row);
   } else {
     // nothing to go by: histogram of the whole input first, its bounds cannot fail
-    a.L_in = c->ws.L_safe;
-    TimedLaunch t(c, MODE == kPull ? DGS_KERNEL_TWO_PASS_PULL : DGS_KERNEL_TWO_PASS_PUSH);
-    k_hist_all<MODE><<<c->hist_grid[MODE], kThreads, 0, c->stream>>>(c->ws, a);
+    a.L_in = ws.L_safe;
+    TimedLaunch t(c, st, MODE == kPull ? DGS_KERNEL_TWO_PASS_PULL : DGS_KERNEL_TWO_PASS_PUSH);
+    k_hist_all<MODE><<<c->hist_grid[MODE], kThreads, 0, st>>>(ws, a);
     DGS_CUDA(c, cudaGetLastError());
     const int pick_grid = (int)std::min<uint32_t>(c->cfg.num_segments, 1024u);
-    k_pick_lower<MODE><<<pick_grid, kThreads, 0, c->stream>>>(c->ws);
+    k_pick_lower<MODE><<<pick_grid, kThreads, 0, st>>>(ws);
     DGS_CUDA(c, cudaGetLastError());
     c->launches += 2;
   }
   {
-    TimedLaunch t(c, MODE == kPull ? DGS_KERNEL_STREAM_PULL : DGS_KERNEL_STREAM_PUSH);
-    k_stream<MODE><<<c->stream_grid[MODE], kThreads, StreamRing<MODE>::kBytes, c->stream>>>(c->ws, a);
+    TimedLaunch t(c, st, MODE == kPull ? DGS_KERNEL_STREAM_PULL : DGS_KERNEL_STREAM_PUSH);
+    k_stream<MODE><<<c->stream_grid[MODE], kThreads, StreamRing<MODE>::kBytes, st>>>(ws, a);
     DGS_CUDA(c, cudaGetLastError());
     c->launches += 1;
   }
   {
     // cooperative launch: the CTAs synchronise among themselves, so all must be resident
-    TimedLaunch t(c, MODE == kPull ? DGS_KERNEL_FINALIZE_PULL : DGS_KERNEL_FINALIZE_PUSH);
-    void* args[] = {(void*)&c->ws, (void*)&a};
+    TimedLaunch t(c, st, MODE == kPull ? DGS_KERNEL_FINALIZE_PULL : DGS_KERNEL_FINALIZE_PUSH);
+    void* args[] = {(void*)&ws, (void*)&a};
     DGS_CUDA(c, cudaLaunchCooperativeKernel((const void*)k_finalize<MODE>, dim3(c->finalize_grid[MODE]),
-                                            dim3(kThreads), args, 0, c->stream));
+                                            dim3(kThreads), args, 0, st));
     c->launches += 1;
   }
   if (a.speculate) {
@@ -307,6 +353,21 @@ int occupancy_grids(dgs_ctx* c, int sms) {
   }
   c->finalize_grid[MODE] = std::min(std::min(sms * occ, kMaxWorkers), kFinalizeWorkers);
   return DGS_OK;
+}
+
+void destroy_ctx(dgs_ctx* c) {
+  for (int i = 0; i < 2; ++i) {
+    if (c->st[i]) cudaStreamDestroy(c->st[i]);
+    if (c->ev_tail[i]) cudaEventDestroy(c->ev_tail[i]);
+  }
+  for (int i = 0; i < kPushSlots; ++i) {
+    if (c->ev_push[i]) cudaEventDestroy(c->ev_push[i]);
+    if (c->ev_apply[i]) cudaEventDestroy(c->ev_apply[i]);
+  }
+  if (c->ev_in) cudaEventDestroy(c->ev_in);
+  for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
+  c->magic = 0;
+  delete c;
 }
 
 }  // namespace
@@ -350,12 +411,20 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   c->segments.assign(cfg->segments, cfg->segments + cfg->num_segments);
   c->cfg.segments = c->segments.data();
   make_layout(&c->cfg, &c->lay);
+  c->st[0] = c->st[1] = nullptr;
+  c->ev_in = nullptr;
+  for (int i = 0; i < kPushSlots; ++i) {
+    c->ev_push[i] = c->ev_apply[i] = nullptr;
+    c->apply_pending[i] = false;
+  }
+  c->ev_tail[0] = c->ev_tail[1] = nullptr;
   if (c->lay.total > cfg->arena_bytes) {
     delete c;
     return DGS_ENOMEM;
   }
   c->base = static_cast<char*>(cfg->arena);
-  c->stream = static_cast<cudaStream_t>(cfg->stream);
+  c->user = static_cast<cudaStream_t>(cfg->stream);
+  c->push_count = 0;
   c->inv_m = 1.0f / cfg->momentum;  // one IEEE division; the kernels multiply by this constant
   c->timestamp = 0;
   c->select_seq = 0;
@@ -376,10 +445,7 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   c->prev.assign(cfg->num_workers, -1);
 
   auto fail = [&](int code) {
-    const int lc = c->last_cuda;
-    (void)lc;
-    c->magic = 0;
-    delete c;
+    destroy_ctx(c);
     return code;
   };
 #define INIT_CUDA(call)                         \
@@ -396,6 +462,15 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   if (occupancy_grids<kPushSam>(c, sms) != DGS_OK || occupancy_grids<kPushResidual>(c, sms) != DGS_OK ||
       occupancy_grids<kPull>(c, sms) != DGS_OK)
     return fail(DGS_ECUDA);
+  for (int i = 0; i < 2; ++i) {
+    INIT_CUDA(cudaStreamCreateWithFlags(&c->st[i], cudaStreamNonBlocking));
+    INIT_CUDA(cudaEventCreateWithFlags(&c->ev_tail[i], cudaEventDisableTiming));
+  }
+  for (int i = 0; i < kPushSlots; ++i) {
+    INIT_CUDA(cudaEventCreateWithFlags(&c->ev_push[i], cudaEventDisableTiming));
+    INIT_CUDA(cudaEventCreateWithFlags(&c->ev_apply[i], cudaEventDisableTiming));
+  }
+  INIT_CUDA(cudaEventCreateWithFlags(&c->ev_in, cudaEventDisableTiming));
 
   const Layout& L = c->lay;
   const uint64_t N = cfg->num_workers, vec = L.n_pad * 4;
@@ -404,7 +479,7 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   tiles.reserve(L.num_tiles);
   build_tiles(&c->cfg, &tiles, &segs);
   if (tiles.size() != L.num_tiles) return fail(DGS_EINVAL);
-  cudaStream_t st = c->stream;
+  cudaStream_t st = c->user;
   // state: u = 0, D = 0 (initialisation lines of Algorithm 3 and Algorithm 2), theta = theta_0
   INIT_CUDA(cudaMemsetAsync(c->at<char>(L.u), 0, vec * (N + 1), st));
   INIT_CUDA(cudaMemsetAsync(c->at<char>(L.D), 0, vec * N, st));
@@ -416,10 +491,14 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
       INIT_CUDA(cudaMemcpyAsync(c->theta_local_buf(q), cfg->theta0, cfg->n * 4, cudaMemcpyDeviceToDevice, st));
   }
   // scratch that kernels expect to find cleared, and the static tables
-  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.tile_sel), 0, L.sel - L.tile_sel, st));
-  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.sel), 0, L.total - L.sel, st));
+  for (int k = 0; k < 2; ++k) {
+    const ScratchLayout& sc = L.sc[k];
+    INIT_CUDA(cudaMemsetAsync(c->at<char>(sc.zero_begin), 0, sc.zero_end - sc.zero_begin, st));
+    INIT_CUDA(cudaMemsetAsync(c->at<char>(sc.part_cands), 0, (uint64_t)kMaxGrid * 4, st));
+    INIT_CUDA(cudaMemsetAsync(c->at<char>(sc.part_slot0), 0, (uint64_t)kMaxGrid * 4, st));
+  }
   INIT_CUDA(cudaMemsetAsync(c->at<char>(L.L_next), 0xFF, 2 * N * cfg->num_segments * 4, st));
-  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.part_cands), 0, (uint64_t)kMaxGrid * 8, st));
+  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.status), 0, L.total - L.status, st));
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.tiles), tiles.data(), tiles.size() * sizeof(Tile), cudaMemcpyHostToDevice, st));
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.segs), segs.data(), segs.size() * sizeof(SegDesc), cudaMemcpyHostToDevice, st));
   std::vector<uint32_t> seg_off(cfg->num_segments + 1), seg_tile0(cfg->num_segments);
@@ -433,31 +512,35 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   std::vector<float*> slots(N + 1);
   for (uint32_t q = 0; q <= N; ++q) slots[q] = c->u_buf(q);
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.u_slots), slots.data(), slots.size() * sizeof(float*), cudaMemcpyHostToDevice, st));
-  INIT_CUDA(cudaStreamSynchronize(st));  // the host vectors above go out of scope
+  // the host vectors above go out of scope, and the library's own streams start from a ready arena
+  INIT_CUDA(cudaStreamSynchronize(st));
 #undef INIT_CUDA
 
-  Workspace& w = c->ws;
-  w.tiles = c->at<Tile>(L.tiles);
-  w.segs = c->at<SegDesc>(L.segs);
-  w.num_tiles = L.num_tiles;
-  w.num_segs = cfg->num_segments;
-  w.cand_idx = c->at<uint32_t>(L.cand_idx);
-  w.cand_val = c->at<float>(L.cand_val);
-  w.part_cands = c->at<uint32_t>(L.part_cands);
-  w.part_slot0 = c->at<uint32_t>(L.part_slot0);
-  w.seg_off = c->at<uint32_t>(L.seg_off);
-  w.seg_tile0 = c->at<uint32_t>(L.seg_tile0);
-  w.tile_pre = c->at<uint2>(L.tile_pre);
-  w.tile_sel = c->at<uint2>(L.tile_sel);
-  w.cta_tot = c->at<uint2>(L.cta_tot);
-  w.hist1 = c->at<uint32_t>(L.hist1);
-  w.hist2 = c->at<uint32_t>(L.hist2);
-  w.hist3 = c->at<uint32_t>(L.hist3);
-  w.sel = c->at<SegSel>(L.sel);
-  w.L_safe = c->at<uint32_t>(L.L_safe);
-  w.sync = c->at<uint32_t>(L.sync);
-  w.status = c->at<int>(L.status);
-  w.stats = c->at<unsigned long long>(L.stats);
+  for (int k = 0; k < 2; ++k) {
+    Workspace& w = c->ws[k];
+    const ScratchLayout& sc = L.sc[k];
+    w.tiles = c->at<Tile>(L.tiles);
+    w.segs = c->at<SegDesc>(L.segs);
+    w.num_tiles = L.num_tiles;
+    w.num_segs = cfg->num_segments;
+    w.seg_off = c->at<uint32_t>(L.seg_off);
+    w.seg_tile0 = c->at<uint32_t>(L.seg_tile0);
+    w.cand_idx = c->at<uint32_t>(sc.cand_idx);
+    w.cand_val = c->at<float>(sc.cand_val);
+    w.part_cands = c->at<uint32_t>(sc.part_cands);
+    w.part_slot0 = c->at<uint32_t>(sc.part_slot0);
+    w.tile_pre = c->at<uint2>(sc.tile_pre);
+    w.tile_sel = c->at<uint2>(sc.tile_sel);
+    w.cta_tot = c->at<uint2>(sc.cta_tot);
+    w.hist1 = c->at<uint32_t>(sc.hist1);
+    w.hist2 = c->at<uint32_t>(sc.hist2);
+    w.hist3 = c->at<uint32_t>(sc.hist3);
+    w.sel = c->at<SegSel>(sc.sel);
+    w.L_safe = c->at<uint32_t>(sc.L_safe);
+    w.sync = c->at<uint32_t>(sc.sync);
+    w.status = c->at<int>(L.status);
+    w.stats = c->at<unsigned long long>(L.stats);
+  }
   *out = c;
   return DGS_OK;
 }
@@ -468,13 +551,20 @@ int dgs_worker_push(dgs_ctx* c, uint32_t worker, const float* grad, dgs_packet* 
   if (worker >= c->cfg.num_workers || !grad) return DGS_EINVAL;
   if ((reinterpret_cast<uintptr_t>(grad) % 16) != 0) return DGS_EINVAL;
   const Layout& L = c->lay;
+  const int slot = (int)(c->push_count % kPushSlots);
+  rc = fork_from_user(c, 0);  // the gradient may have been produced on the caller's stream
+  if (rc != DGS_OK) return rc;
+  if (c->apply_pending[slot]) {  // the packet that lived in this slot must have been applied
+    DGS_CUDA(c, cudaStreamWaitEvent(c->st[0], c->ev_apply[slot], 0));
+    c->apply_pending[slot] = false;
+  }
   SelArgs a;
   std::memset(&a, 0, sizeof(a));
   a.grad = grad;
   a.u_cur_slot = c->u_slot(worker);
   a.u_spare_slot = c->u_slot(c->cfg.num_workers);
-  a.pkt_idx = c->at<uint32_t>(L.pkt_idx[0]);
-  a.pkt_val = c->at<float>(L.pkt_val[0]);
+  a.pkt_idx = c->at<uint32_t>(L.pkt_idx[slot]);
+  a.pkt_val = c->at<float>(L.pkt_val[slot]);
   a.pkt_count = (uint32_t)L.K[0];
   a.m = c->cfg.momentum;
   a.lr = c->cfg.lr;
@@ -483,7 +573,9 @@ int dgs_worker_push(dgs_ctx* c, uint32_t worker, const float* grad, dgs_packet* 
   rc = (c->cfg.flags & DGS_RESIDUAL_MODE) ? launch_select<kPushResidual>(c, a, worker, age)
                                           : launch_select<kPushSam>(c, a, worker, age);
   if (rc != DGS_OK) return rc;
+  DGS_CUDA(c, cudaEventRecord(c->ev_push[slot], c->st[0]));
   c->pushes[worker] += 1;
+  c->push_count += 1;
   if (out) {
     out->idx = a.pkt_idx;
     out->val = a.pkt_val;
@@ -497,14 +589,28 @@ int dgs_server_apply(dgs_ctx* c, uint32_t worker, const dgs_packet* pkt) {
   if (rc != DGS_OK) return rc;
   if (worker >= c->cfg.num_workers || !pkt) return DGS_EINVAL;
   if (pkt->count > 0 && (!pkt->idx || !pkt->val)) return DGS_EINVAL;
+  // whose packet is it?  one of the push slots: wait for that push; anything else: the caller's stream
+  int slot = -1;
+  for (int i = 0; i < kPushSlots; ++i)
+    if (pkt->idx == c->at<uint32_t>(c->lay.pkt_idx[i])) slot = i;
+  if (slot >= 0) {
+    DGS_CUDA(c, cudaStreamWaitEvent(c->st[1], c->ev_push[slot], 0));
+  } else {
+    rc = fork_from_user(c, 1);
+    if (rc != DGS_OK) return rc;
+  }
   if (pkt->count > 0) {
     const dim3 grid((pkt->count + kThreads - 1) / kThreads, c->cfg.num_workers + 1);
-    TimedLaunch t(c, DGS_KERNEL_SCATTER);
-    k_scatter_sub<<<grid, kThreads, 0, c->stream>>>(pkt->idx, pkt->val, pkt->count, c->at<float>(c->lay.theta),
-                                                    c->at<float>(c->lay.D), c->lay.n_pad, c->cfg.num_workers,
-                                                    c->cfg.n, c->ws.status);
+    TimedLaunch t(c, c->st[1], DGS_KERNEL_SCATTER);
+    k_scatter_sub<<<grid, kThreads, 0, c->st[1]>>>(pkt->idx, pkt->val, pkt->count, c->at<float>(c->lay.theta),
+                                                   c->at<float>(c->lay.D), c->lay.n_pad, c->cfg.num_workers,
+                                                   c->cfg.n, c->ws[1].status);
     DGS_CUDA(c, cudaGetLastError());
     c->launches += 1;
+  }
+  if (slot >= 0) {
+    DGS_CUDA(c, cudaEventRecord(c->ev_apply[slot], c->st[1]));
+    c->apply_pending[slot] = true;
   }
   c->timestamp += 1;  // t counts updates made to the server parameters
   return DGS_OK;
@@ -515,12 +621,14 @@ int dgs_worker_pull(dgs_ctx* c, uint32_t worker, dgs_packet* out) {
   if (rc != DGS_OK) return rc;
   if (worker >= c->cfg.num_workers) return DGS_EINVAL;
   const Layout& L = c->lay;
+  rc = fork_from_user(c, 1);  // the caller may still be reading the previous pull packet on its stream
+  if (rc != DGS_OK) return rc;
   SelArgs a;
   std::memset(&a, 0, sizeof(a));
   a.D = c->D_buf(worker);
   a.theta_local = (c->cfg.flags & DGS_KEEP_LOCAL_MODEL) ? c->theta_local_buf(worker) : nullptr;
-  a.pkt_idx = c->at<uint32_t>(L.pkt_idx[1]);
-  a.pkt_val = c->at<float>(L.pkt_val[1]);
+  a.pkt_idx = c->at<uint32_t>(L.pkt_idx[kPushSlots]);
+  a.pkt_val = c->at<float>(L.pkt_val[kPushSlots]);
   a.pkt_count = (uint32_t)L.K[1];
   a.m = c->cfg.momentum;
   a.lr = c->cfg.lr;
@@ -551,18 +659,29 @@ int dgs_event(dgs_ctx* c, uint32_t worker, const float* grad, dgs_packet* push_o
   return DGS_OK;
 }
 
+int dgs_flush(dgs_ctx* c) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  for (int i = 0; i < 2; ++i) {
+    DGS_CUDA(c, cudaEventRecord(c->ev_tail[i], c->st[i]));
+    DGS_CUDA(c, cudaStreamWaitEvent(c->user, c->ev_tail[i], 0));
+  }
+  return DGS_OK;
+}
+
 int dgs_event_host(dgs_ctx* c, uint32_t worker, const float* grad_host, uint32_t* out_idx, float* out_val) {
   int rc = live(c);
   if (rc != DGS_OK) return rc;
   if (!(c->cfg.flags & DGS_HOST_IO) || !grad_host || worker >= c->cfg.num_workers) return DGS_EINVAL;
   float* stage = c->at<float>(c->lay.grad_stage);
-  DGS_CUDA(c, cudaMemcpyAsync(stage, grad_host, c->cfg.n * 4, cudaMemcpyHostToDevice, c->stream));
+  // the staging buffer is read by pushes on the worker stream only, so the copy goes there too
+  DGS_CUDA(c, cudaMemcpyAsync(stage, grad_host, c->cfg.n * 4, cudaMemcpyHostToDevice, c->st[0]));
   dgs_packet g;
   rc = dgs_event(c, worker, stage, nullptr, &g);
   if (rc != DGS_OK) return rc;
-  if (out_idx) DGS_CUDA(c, cudaMemcpyAsync(out_idx, g.idx, (uint64_t)g.count * 4, cudaMemcpyDeviceToHost, c->stream));
-  if (out_val) DGS_CUDA(c, cudaMemcpyAsync(out_val, g.val, (uint64_t)g.count * 4, cudaMemcpyDeviceToHost, c->stream));
-  DGS_CUDA(c, cudaStreamSynchronize(c->stream));
+  if (out_idx) DGS_CUDA(c, cudaMemcpyAsync(out_idx, g.idx, (uint64_t)g.count * 4, cudaMemcpyDeviceToHost, c->st[1]));
+  if (out_val) DGS_CUDA(c, cudaMemcpyAsync(out_val, g.val, (uint64_t)g.count * 4, cudaMemcpyDeviceToHost, c->st[1]));
+  DGS_CUDA(c, cudaStreamSynchronize(c->st[1]));
   return DGS_OK;
 }
 
@@ -580,15 +699,15 @@ int dgs_state_ptr(dgs_ctx* c, int which, uint32_t worker, const float** out) {
       break;
     case DGS_U: {
       float* p = nullptr;
-      DGS_CUDA(c, cudaMemcpyAsync(&p, c->u_slot(worker), sizeof(p), cudaMemcpyDeviceToHost, c->stream));
-      DGS_CUDA(c, cudaStreamSynchronize(c->stream));
+      DGS_CUDA(c, cudaMemcpyAsync(&p, c->u_slot(worker), sizeof(p), cudaMemcpyDeviceToHost, c->st[0]));
+      rc = sync_all(c);
+      if (rc != DGS_OK) return rc;
       *out = p;
       return DGS_OK;
     }
     default: return DGS_EINVAL;
   }
-  DGS_CUDA(c, cudaStreamSynchronize(c->stream));
-  return DGS_OK;
+  return sync_all(c);
 }
 
 int dgs_state_load(dgs_ctx* c, int which, uint32_t worker, const float* src) {
@@ -596,9 +715,14 @@ int dgs_state_load(dgs_ctx* c, int which, uint32_t worker, const float* src) {
   if (rc != DGS_OK) return rc;
   if (!src) return DGS_EINVAL;
   const float* dst = nullptr;
-  rc = dgs_state_ptr(c, which, worker, &dst);
+  rc = dgs_state_ptr(c, which, worker, &dst);  // waits for all work in flight
   if (rc != DGS_OK) return rc;
-  DGS_CUDA(c, cudaMemcpyAsync(const_cast<float*>(dst), src, c->cfg.n * 4, cudaMemcpyDeviceToDevice, c->stream));
+  // velocities are only touched on the worker stream, everything else on the server stream
+  const int which_stream = which == DGS_U ? 0 : 1;
+  rc = fork_from_user(c, which_stream);
+  if (rc != DGS_OK) return rc;
+  DGS_CUDA(c, cudaMemcpyAsync(const_cast<float*>(dst), src, c->cfg.n * 4, cudaMemcpyDeviceToDevice,
+                              c->st[which_stream]));
   return DGS_OK;
 }
 
@@ -606,8 +730,9 @@ int dgs_status(dgs_ctx* c, int* device_status) {
   int rc = live(c);
   if (rc != DGS_OK) return rc;
   if (!device_status) return DGS_EINVAL;
-  DGS_CUDA(c, cudaMemcpyAsync(device_status, c->ws.status, 4, cudaMemcpyDeviceToHost, c->stream));
-  DGS_CUDA(c, cudaStreamSynchronize(c->stream));
+  rc = sync_all(c);
+  if (rc != DGS_OK) return rc;
+  DGS_CUDA(c, cudaMemcpy(device_status, c->ws[0].status, 4, cudaMemcpyDeviceToHost));
   return DGS_OK;
 }
 
@@ -616,8 +741,9 @@ int dgs_stats(dgs_ctx* c, uint64_t out[4]) {
   if (rc != DGS_OK) return rc;
   if (!out) return DGS_EINVAL;
   unsigned long long s[4] = {0, 0, 0, 0};
-  DGS_CUDA(c, cudaMemcpyAsync(s, c->ws.stats, sizeof(s), cudaMemcpyDeviceToHost, c->stream));
-  DGS_CUDA(c, cudaStreamSynchronize(c->stream));
+  rc = sync_all(c);
+  if (rc != DGS_OK) return rc;
+  DGS_CUDA(c, cudaMemcpy(s, c->ws[0].stats, sizeof(s), cudaMemcpyDeviceToHost));
   out[0] = s[0];
   out[1] = s[1];
   out[2] = c->timestamp;
@@ -652,7 +778,8 @@ int dgs_timing_read(dgs_ctx* c, double ms[DGS_NUM_KERNELS], uint64_t count[DGS_N
   int rc = live(c);
   if (rc != DGS_OK) return rc;
   if (!ms || !count) return DGS_EINVAL;
-  DGS_CUDA(c, cudaStreamSynchronize(c->stream));
+  rc = sync_all(c);
+  if (rc != DGS_OK) return rc;
   for (size_t i = 0; i < c->ev_kernel.size(); ++i) {
     float t = 0.f;
     DGS_CUDA(c, cudaEventElapsedTime(&t, c->ev_pool[2 * i], c->ev_pool[2 * i + 1]));
@@ -676,10 +803,10 @@ int dgs_last_cuda_error(dgs_ctx* c) {
 
 int dgs_free(dgs_ctx* c) {
   if (!c || c->magic != kMagic) return DGS_ESTATE;
-  cudaStreamSynchronize(c->stream);
-  for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
-  c->magic = 0;
-  delete c;
+  cudaStreamSynchronize(c->st[0]);
+  cudaStreamSynchronize(c->st[1]);
+  cudaStreamSynchronize(c->user);
+  destroy_ctx(c);
   return DGS_OK;
 }
 

@@ -190,8 +190,10 @@ def test_two_runs_are_bit_identical():
     outs = []
     for _ in range(2):
         ctx = dgs.Context.from_workload(wl)
+        # gradients must outlive the (asynchronous) events that read them
+        grads = [torch.from_numpy(wl.gradient(e)).to(DEV) for e in range(wl.num_events)]
         for e, w in enumerate(wl.schedule()):
-            ctx.event(int(w), torch.from_numpy(wl.gradient(e)).to(DEV))
+            ctx.event(int(w), grads[e])
         outs.append([ctx.state(dgs.DGS_THETA).clone()] +
                     [ctx.state(dgs.DGS_U, q).clone() for q in range(3)] +
                     [ctx.state(dgs.DGS_D, q).clone() for q in range(3)])
