@@ -82,7 +82,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -91,7 +91,15 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            self.rows.append((time.perf_counter(), [c.strip() for c in line.split(",")]))
+
+    def window(self, t0: float, t1: float) -> None:
+        """Keep the samples taken between two perf_counter readings (at least the nearest one)."""
+        inside = [r for t, r in self.rows if t0 <= t <= t1]
+        if not inside and self.rows:
+            mid = 0.5 * (t0 + t1)
+            inside = [min(self.rows, key=lambda tr: abs(tr[0] - mid))[1]]
+        self.rows = inside
 
     def __exit__(self, *a):
         if self.proc is not None:
@@ -244,19 +252,22 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    run_events(0, preroll)
-    run_events(preroll, Wm)
-    ctx.flush()
-    stats0 = ctx.stats()
-    launches0 = ctx.launch_count()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
     with ClockSampler(local_rank) as clocks:
+        run_events(0, preroll)
+        run_events(preroll, Wm)
+        ctx.flush()
+        stats0 = ctx.stats()
+        launches0 = ctx.launch_count()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        t_begin = time.perf_counter()
         ev0.record(stream)
         run_events(preroll + Wm, K)
         ctx.flush()
         ev1.record(stream)
         barrier()
+        t_end = time.perf_counter()
+    clocks.window(t_begin, t_end)
     elapsed = ev0.elapsed_time(ev1) * 1e-3
     launches = ctx.launch_count() - launches0
     stats1 = ctx.stats()
@@ -335,12 +346,12 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=128)
-    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--steps", type=int, default=512)
+    ap.add_argument("--warmup", type=int, default=32)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50", choices=sorted(W.BY_NAME))
     ap.add_argument("--seed", type=int, default=W.DEFAULT_SEED)
-    ap.add_argument("--grad-pool", type=int, default=192, help="distinct gradients kept in HBM (reused cyclically)")
+    ap.add_argument("--grad-pool", type=int, default=127, help="distinct gradients kept in HBM (reused cyclically)")
     ap.add_argument("--workers", type=int, default=0,
                     help="override the number of simulated workers (smaller state for profiler captures)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
