@@ -636,28 +636,23 @@ __device__ uint32_t block_pick(const uint32_t* hist, uint32_t k, uint32_t& bin, 
   return (uint32_t)total;
 }
 
-// Barrier among the first W CTAs of the grid (all resident: cooperative launch).
+// Barrier among the CTAs of finalize (all resident: cooperative launch).  One arrival
+// counter that only grows: the i-th barrier of a launch is passed when the counter has
+// reached i*W (the stream pass that precedes every finalize launch clears the counter).
 // Bounded: returns false, with the status word set, if the others do not arrive.
-__device__ bool worker_barrier(uint32_t* sync, uint32_t W, int* status, int* s_ok) {
+__device__ bool worker_barrier(uint32_t* sync, uint32_t W, int* status, int* s_ok, uint32_t& target) {
+  target += W;
   __syncthreads();
   if (threadIdx.x == 0) {
     int ok = 1;
     __threadfence();
-    const uint32_t gen = ld_volatile(sync + kBarGen);
-    const uint32_t prev = atomicAdd(sync + kBarCount, 1u);
-    if (prev == W - 1) {
-      atomicExch(sync + kBarCount, 0u);
-      __threadfence();
-      atomicAdd(sync + kBarGen, 1u);
-    } else {
-      uint32_t spins = 0;
-      while (ld_volatile(sync + kBarGen) == gen) {
-        if (++spins > kSpinLimit) {
-          ok = 0;
-          atomicMin(status, kStatusTimeout);
-          break;
-        }
-        __nanosleep(20);
+    atomicAdd(sync + kBarCount, 1u);
+    uint32_t spins = 0;
+    while ((int32_t)(ld_volatile(sync + kBarCount) - target) < 0) {
+      if (++spins > kSpinLimit) {
+        ok = 0;
+        atomicMin(status, kStatusTimeout);
+        break;
       }
     }
     __threadfence();
@@ -777,13 +772,18 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
   sv.S = S;
   __syncthreads();
 
+  // flat numbering of the candidates, and this thread's own candidates
+  uint32_t parts = 0, C = 0, per_thread = 0, my_lo = 0, my_hi = 0;
+  constexpr int kKeep = 8;            // candidates a thread keeps in registers between the phases
+  uint32_t rkey[kKeep], ridx[kKeep];  // valid when per_thread <= kKeep
+  uint32_t bar_target = 0;
   bool redo = false;
   for (int attempt = 0; attempt < 2; ++attempt) {
     if (redo) {
       // the guess was too high for some layer: take the bound that cannot fail from a histogram of
       // the whole input and repeat the stream pass, with the few CTAs this kernel has
       hist_all_tiles<MODE>(ws, a, in, cta, W, sh.stream.hist);
-      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
+      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
       for (uint32_t s = cta; s < S; s += W) {
         uint32_t bin, krem;
         uint32_t* h = ws.hist1 + (size_t)s * kBins1;
@@ -792,9 +792,55 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
         for (int b = threadIdx.x; b < kBins1; b += kThreads) h[b] = 0;
       }
       if (cta == 0 && threadIdx.x == 0) ws.sync[kFail] = 0;
-      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
+      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
       stream_tiles<MODE>(ws, a, ws.L_safe, in, out, cta, W, sh.stream);
-      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
+      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+    }
+    // flat numbering of the candidates (the stream pass is complete: an earlier kernel, or the barrier above)
+    parts = ld_volatile(ws.sync + kParts);
+    {
+      constexpr int PER = kMaxGrid / kThreads;   // parts <= kMaxGrid
+      uint32_t cnt[PER];
+#pragma unroll
+      for (int j = 0; j < PER; ++j) {
+        const uint32_t p = j * kThreads + threadIdx.x;
+        cnt[j] = p < parts ? __ldcg(ws.part_cands + p) : 0;
+        if (p < parts) sh.slot0[p] = __ldcg(ws.part_slot0 + p);
+      }
+      unsigned long long carry = 0;
+#pragma unroll
+      for (int j = 0; j < PER; ++j) {
+        if ((uint32_t)(j * kThreads) < parts) {   // CTA-uniform
+          const uint32_t p = j * kThreads + threadIdx.x;
+          unsigned long long total;
+          const unsigned long long ex = block_excl_scan(cnt[j], sh.warp_scan, total) + carry;
+          if (p < parts) sh.pre_cands[p] = (uint32_t)ex;
+          carry += total;
+        }
+      }
+      if (threadIdx.x == 0) sh.pre_cands[parts] = (uint32_t)carry;
+      __syncthreads();
+    }
+    C = sh.pre_cands[parts];
+    // every thread owns the flat candidates [my_lo, my_hi); when they are few it keeps them in registers
+    per_thread = (C + nthreads - 1) / nthreads;
+    my_lo = min(C, gthread * per_thread);
+    my_hi = min(C, my_lo + per_thread);
+    if (per_thread <= (uint32_t)kKeep && my_lo < my_hi) {
+      Cursor cur = cursor_at(sh, parts, my_lo);
+      float raw[kKeep];
+#pragma unroll
+      for (int u = 0; u < kKeep; ++u) {
+        raw[u] = 0.f;
+        ridx[u] = 0;
+        if (my_lo + u < my_hi) {
+          raw[u] = __ldcg(ws.cand_val + cur.slot);
+          ridx[u] = __ldcg(ws.cand_idx + cur.slot);
+          cursor_advance(sh, parts, cur, 1);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kKeep; ++u) rkey[u] = key_of(raw[u]);
     }
     // level 1: pick the bin of the k-th largest among the candidates; check the guess
     for (uint32_t s = cta; s < S; s += W) {
@@ -827,40 +873,10 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
       __syncthreads();
       for (int b = threadIdx.x; b < kBins1; b += kThreads) h[b] = 0;
     }
-    if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
+    if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
     if (redo || ld_volatile(ws.sync + kFail) == 0) break;
     redo = true;
   }
-
-  // flat numbering of the candidates
-  const uint32_t parts = ld_volatile(ws.sync + kParts);
-  {
-    constexpr int PER = kMaxGrid / kThreads;   // parts <= kMaxGrid
-    uint32_t cnt[PER];
-#pragma unroll
-    for (int j = 0; j < PER; ++j) {
-      const uint32_t p = j * kThreads + threadIdx.x;
-      cnt[j] = p < parts ? __ldcg(ws.part_cands + p) : 0;
-      if (p < parts) sh.slot0[p] = __ldcg(ws.part_slot0 + p);
-    }
-    unsigned long long carry = 0;
-#pragma unroll
-    for (int j = 0; j < PER; ++j) {
-      if ((uint32_t)(j * kThreads) < parts) {   // CTA-uniform
-        const uint32_t p = j * kThreads + threadIdx.x;
-        unsigned long long total;
-        const unsigned long long ex = block_excl_scan(cnt[j], sh.warp_scan, total) + carry;
-        if (p < parts) sh.pre_cands[p] = (uint32_t)ex;
-        carry += total;
-      }
-    }
-    if (threadIdx.x == 0) sh.pre_cands[parts] = (uint32_t)carry;
-    __syncthreads();
-  }
-  const uint32_t C = sh.pre_cands[parts];
-  // every thread owns the flat candidates [my_lo, my_hi)
-  const uint32_t per_thread = (C + nthreads - 1) / nthreads;
-  const uint32_t my_lo = min(C, gthread * per_thread), my_hi = min(C, my_lo + per_thread);
 
   // ---- levels 2 and 3 ----------------------------------------------------------------
 #pragma unroll 1
@@ -876,13 +892,26 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
       for (int b = threadIdx.x; b < B; b += kThreads) sh.stream.hist[b] = 0;
       __syncthreads();
     }
-    if (my_lo < my_hi) {
+    auto add_level = [&](uint32_t key, uint32_t idx) {
+      const uint32_t seg = S > 1 ? seg_of(sv, idx) : 0;
+      const uint32_t prefix = seg_smem ? sh.seg_a[seg] : __ldcg(&ws.sel[seg].prefix);
+      if ((key >> SH) == prefix) {
+        const uint32_t digit = (key >> (SH - 10)) & 1023u;
+        if (S == 1) atomicAdd(sh.stream.hist + digit, 1u);       // one layer: CTA-private histogram first
+        else atomicAdd(hist + (size_t)seg * B + digit, 1u);
+      }
+    };
+    if (per_thread <= (uint32_t)kKeep) {
+#pragma unroll
+      for (int u = 0; u < kKeep; ++u)
+        if (my_lo + u < my_hi) add_level(rkey[u], ridx[u]);
+    } else if (my_lo < my_hi) {
       Cursor cur = cursor_at(sh, parts, my_lo);
       for (uint32_t p = my_lo; p < my_hi; p += kBatch) {
         // all loads of the batch are issued before any loaded value is touched (a use right
         // after its load would make the loads wait for one another)
         float raw[kBatch];
-        uint32_t key[kBatch], idx[kBatch];
+        uint32_t idx[kBatch];
 #pragma unroll
         for (int u = 0; u < kBatch; ++u) {
           raw[u] = 0.f;
@@ -894,19 +923,8 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
           }
         }
 #pragma unroll
-        for (int u = 0; u < kBatch; ++u) key[u] = key_of(raw[u]);
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-          if (p + u < my_hi) {
-            const uint32_t seg = S > 1 ? seg_of(sv, idx[u]) : 0;
-            const uint32_t prefix = seg_smem ? sh.seg_a[seg] : __ldcg(&ws.sel[seg].prefix);
-            if ((key[u] >> SH) == prefix) {
-              const uint32_t digit = (key[u] >> (SH - 10)) & 1023u;
-              if (S == 1) atomicAdd(sh.stream.hist + digit, 1u);       // one layer: CTA-private histogram first
-              else atomicAdd(hist + (size_t)seg * B + digit, 1u);
-            }
-          }
-        }
+        for (int u = 0; u < kBatch; ++u)
+          if (p + u < my_hi) add_level(key_of(raw[u]), idx[u]);
       }
     }
     if (S == 1) {
@@ -916,7 +934,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
         if (v) atomicAdd(hist + b, v);
       }
     }
-    if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
+    if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
     for (uint32_t s = cta; s < S; s += W) {
       uint32_t bin, krem;
       uint32_t* h = hist + (size_t)s * B;
@@ -932,7 +950,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
       }
       for (int b = threadIdx.x; b < B; b += kThreads) h[b] = 0;
     }
-    if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
+    if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
   }
 
   // ---- count: per tile, how many candidates have key > T and key == T ----------------
@@ -944,37 +962,41 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
     }
     __syncthreads();
   }
-  if (my_lo < my_hi) {
-    Cursor cur = cursor_at(sh, parts, my_lo);
-    for (uint32_t p = my_lo; p < my_hi; p += kBatch) {
-      float raw[kBatch];
-      uint32_t key[kBatch], idx[kBatch];
-#pragma unroll
-      for (int u = 0; u < kBatch; ++u) {
-        raw[u] = 0.f;
-        idx[u] = 0;
-        if (p + u < my_hi) {
-          raw[u] = __ldcg(ws.cand_val + cur.slot);
-          idx[u] = __ldcg(ws.cand_idx + cur.slot);
-          cursor_advance(sh, parts, cur, 1);
-        }
+  {
+    auto add_count = [&](uint32_t key, uint32_t idx) {
+      const uint32_t seg = S > 1 ? seg_of(sv, idx) : 0;
+      const uint32_t T = seg_smem ? sh.seg_a[seg] : __ldcg(&ws.sel[seg].T);
+      if (key >= T) {
+        uint2* c = ws.tile_sel + tile_of(sv, seg, idx);
+        atomicAdd(key > T ? &c->x : &c->y, 1u);
       }
+    };
+    if (per_thread <= (uint32_t)kKeep) {
 #pragma unroll
-      for (int u = 0; u < kBatch; ++u) key[u] = key_of(raw[u]);
+      for (int u = 0; u < kKeep; ++u)
+        if (my_lo + u < my_hi) add_count(rkey[u], ridx[u]);
+    } else if (my_lo < my_hi) {
+      Cursor cur = cursor_at(sh, parts, my_lo);
+      for (uint32_t p = my_lo; p < my_hi; p += kBatch) {
+        float raw[kBatch];
+        uint32_t idx[kBatch];
 #pragma unroll
-      for (int u = 0; u < kBatch; ++u) {
-        if (p + u < my_hi) {
-          const uint32_t seg = S > 1 ? seg_of(sv, idx[u]) : 0;
-          const uint32_t T = seg_smem ? sh.seg_a[seg] : __ldcg(&ws.sel[seg].T);
-          if (key[u] >= T) {
-            uint2* c = ws.tile_sel + tile_of(sv, seg, idx[u]);
-            atomicAdd(key[u] > T ? &c->x : &c->y, 1u);
+        for (int u = 0; u < kBatch; ++u) {
+          raw[u] = 0.f;
+          idx[u] = 0;
+          if (p + u < my_hi) {
+            raw[u] = __ldcg(ws.cand_val + cur.slot);
+            idx[u] = __ldcg(ws.cand_idx + cur.slot);
+            cursor_advance(sh, parts, cur, 1);
           }
         }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u)
+          if (p + u < my_hi) add_count(key_of(raw[u]), idx[u]);
       }
     }
   }
-  if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
+  if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
 
   // ---- scan over the tiles in index order: CTA c owns tiles [c*chunk, (c+1)*chunk) ----
   const uint32_t chunk_tiles = (ws.num_tiles + W - 1) / W;
@@ -1006,7 +1028,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
     }
     if (threadIdx.x == 0) ws.cta_tot[cta] = make_uint2((uint32_t)(carry >> 32), (uint32_t)carry);
   }
-  if (!worker_barrier(ws.sync, W, ws.status, &sh.ok)) return;
+  if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
 
   // ---- emit: packet in index order, and the state updates that depend on selection ----
   {
@@ -1183,6 +1205,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_stream(Workspace ws, SelArgs a)
     in = *a.u_cur_slot;
     out = *a.u_spare_slot;
   }
+  if (blockIdx.x == 0 && threadIdx.x == 0) ws.sync[kBarCount] = 0;   // for the finalize launch that follows
   stream_tiles_tma<MODE>(ws, a, a.L_in, in, out, blockIdx.x, gridDim.x, sh, reinterpret_cast<float*>(dyn_smem), full,
                          &s_dead);
 }
