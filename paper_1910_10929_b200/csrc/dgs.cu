@@ -1,13 +1,16 @@
 // Host side of the C ABI declared in include/dgs.h: argument checks, the layout of
 // the caller's arena, and the kernel launches of one push / apply / pull event.
 //
-// Work runs on two streams of the library's own.  The worker stream takes the pushes
-// (stream pass + finalize), the server stream takes apply and pull.  A push touches only
-// the worker's velocity, the gradient and its own scratch, so the push of the next event
-// runs while the server side of the current one is still busy; the small, latency-bound
-// finalize kernels then share the GPU with the bandwidth-bound passes of the other stream.
-// Order between the two is kept with CUDA events: an apply waits for the push that made
-// its packet, and a push that reuses a packet slot waits for the apply that read it.
+// Work runs on a few streams of the library's own so that independent steps of consecutive
+// events overlap: pushes alternate between two worker streams, the apply runs on a stream
+// of its own, pulls alternate between two server streams.  A push touches only the worker's
+// velocity, the gradient and its own scratch; a pull touches one difference vector.  The
+// small, latency-bound finalize kernels thus share the GPU with the bandwidth-bound passes
+// of other events.  Order is kept by a small dependency tracker: every launch names the
+// buffers it reads and writes, and waits (cudaStreamWaitEvent) for the last writer of what
+// it reads and for the last writer and the readers of what it writes.  Per buffer the order
+// of operations is therefore the order of the calls, which keeps the results bit-identical
+// to a serial run.
 #include "dgs.h"
 
 #include <algorithm>
@@ -16,6 +19,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "dgs_kernels.cuh"
@@ -26,7 +30,11 @@ namespace {
 
 constexpr uint64_t kAlign = 256;
 constexpr uint32_t kMagic = 0x44475331u;  // "DGS1"
-constexpr int kPushSlots = 2;             // push packet slots, used alternately
+constexpr int kPushSlots = 3;             // push packet slots, used in turn
+constexpr int kPullSlots = 2;             // pull packet slots
+constexpr int kSets = 2;                  // scratch sets (and spare velocity buffers) per kind of selection
+constexpr int kWorkerStreams = 2, kServerStreams = 2;
+enum StreamId : int { kStW0 = 0, kStW1 = 1, kStApply = 2, kStRest = 3, kStS0 = 4, kStS1 = 5, kNumStreams = 6 };
 
 inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
@@ -43,9 +51,9 @@ struct Layout {
   uint64_t K[2] = {0, 0};
   // byte offsets into the arena
   uint64_t theta, u, D, theta_local, grad_stage;
-  uint64_t pkt_idx[kPushSlots + 1], pkt_val[kPushSlots + 1];  // push slots, then the pull slot
+  uint64_t pkt_idx[kPushSlots + kPullSlots], pkt_val[kPushSlots + kPullSlots];  // push slots, then pull slots
   uint64_t tiles, segs, seg_off, seg_tile0;
-  ScratchLayout sc[2];
+  ScratchLayout sc[2 * kSets];  // [kind * kSets + set]
   uint64_t L_next, u_slots, status, stats;
   uint64_t total = 0;
 };
@@ -126,11 +134,11 @@ void make_layout(const dgs_config* c, Layout* L) {
   };
   const uint64_t vec = L->n_pad * 4;
   L->theta = take(vec);
-  L->u = take(vec * (N + 1));  // N velocities and one spare that a push writes into
+  L->u = take(vec * (N + kSets));  // N velocities and the spares that pushes write into
   L->D = take(vec * N);
   L->theta_local = (c->flags & DGS_KEEP_LOCAL_MODEL) ? take(vec * N) : 0;
   L->grad_stage = (c->flags & DGS_HOST_IO) ? take(vec) : 0;
-  for (int p = 0; p <= kPushSlots; ++p) {
+  for (int p = 0; p < kPushSlots + kPullSlots; ++p) {
     const uint64_t K = L->K[p < kPushSlots ? 0 : 1];
     L->pkt_idx[p] = take(K * 4);
     L->pkt_val[p] = take(K * 4);
@@ -139,7 +147,7 @@ void make_layout(const dgs_config* c, Layout* L) {
   L->segs = take(S * sizeof(SegDesc));
   L->seg_off = take((S + 1) * 4);
   L->seg_tile0 = take(S * 4);
-  for (int k = 0; k < 2; ++k) {
+  for (int k = 0; k < 2 * kSets; ++k) {
     ScratchLayout& sc = L->sc[k];
     sc.cand_idx = take(vec);
     sc.cand_val = take(vec);
@@ -158,7 +166,7 @@ void make_layout(const dgs_config* c, Layout* L) {
     sc.zero_end = off;
   }
   L->L_next = take(2 * N * S * 4);
-  L->u_slots = take((N + 1) * sizeof(float*));
+  L->u_slots = take((N + kSets) * sizeof(float*));
   L->status = take(4);
   L->stats = take(32 * 8);
   L->total = off;
@@ -173,19 +181,28 @@ struct dgs_ctx {
   Layout lay;
   char* base;
   cudaStream_t user;       // the caller's stream: entry point of dependencies, target of dgs_flush
-  cudaStream_t st[2];      // [0] worker stream (push), [1] server stream (apply, pull)
+  cudaStream_t st[kNumStreams];
   cudaEvent_t ev_in;       // "everything the caller had enqueued when the call was made"
-  cudaEvent_t ev_push[kPushSlots];   // push packet in slot i is complete
-  cudaEvent_t ev_apply[kPushSlots];  // the apply that read slot i is done
-  bool apply_pending[kPushSlots];    // ev_apply[i] has been recorded since slot i was last written
-  cudaEvent_t ev_tail[2];  // for dgs_flush
-  uint64_t push_count;
-  Workspace ws[2];         // [0] push pipeline, [1] pull pipeline
+  bool forked[kNumStreams];  // stream already waits for ev_in of the current call
+  cudaEvent_t ev_tail[kNumStreams];  // for dgs_flush
+  // dependency tracker
+  struct Res {
+    cudaEvent_t last_write = nullptr;
+    int write_stream = -1;
+    std::vector<std::pair<cudaEvent_t, int>> reads;  // readers since the last write (event, stream)
+  };
+  std::vector<Res> res;
+  std::vector<cudaEvent_t> ev_ring;  // one "done" event per task, reused in turn
+  size_t ev_next;
+  uint64_t push_count, pull_count, event_count;
+  int prev_pull_worker;    // worker whose pull was enqueued last (-1: none): its D is left to a launch of its own
+  Workspace ws[2 * kSets]; // [kind * kSets + set]
   float inv_m;
   int stream_grid[3];    // CTAs of the stand-alone stream pass, per mode
   int hist_grid[3];      // CTAs of the whole-input histogram pass, per mode
   int finalize_grid[3];  // CTAs of the cooperative finalize kernel, per mode
   uint32_t select_seq;   // selections launched so far
+  uint64_t kind_seq[2];  // selections of each kind launched so far
   // Carried bounds: row (kind, worker) of L_next holds the bounds suggested by that worker's
   // latest selection of that kind ([0] push, [1] pull).  row_age says in which state it was
   // made: pushes the worker had done before (push), packets accumulated in D_w since its
@@ -218,6 +235,21 @@ struct dgs_ctx {
 };
 
 namespace {
+
+// resources of the dependency tracker
+struct ResIds {
+  uint32_t N;
+  uint32_t U(uint32_t w) const { return w; }
+  uint32_t D(uint32_t q) const { return N + q; }
+  uint32_t TL(uint32_t q) const { return 2 * N + q; }
+  uint32_t ROW(int kind, uint32_t w) const { return 3 * N + (uint32_t)kind * N + w; }
+  uint32_t THETA() const { return 5 * N; }
+  uint32_t SPARE(int j) const { return 5 * N + 1 + j; }
+  uint32_t SCR(int kind, int set) const { return 5 * N + 1 + kSets + kind * kSets + set; }
+  uint32_t PKT(int slot) const { return 5 * N + 1 + 3 * kSets + slot; }   // push slots, then pull slots
+  uint32_t STAGE() const { return 5 * N + 1 + 3 * kSets + kPushSlots + kPullSlots; }
+  uint32_t count() const { return STAGE() + 1; }
+};
 
 #define DGS_CUDA(ctx, call)                 \
   do {                                      \
@@ -260,36 +292,93 @@ struct TimedLaunch {
   }
 };
 
-// Makes internal stream `which` wait for everything the caller has enqueued on its stream so far.
-int fork_from_user(dgs_ctx* c, int which) {
+// Makes an internal stream wait for everything the caller had enqueued on its stream when the
+// current API call began (ev_in is recorded once per call by begin_call).
+int begin_call(dgs_ctx* c) {
   DGS_CUDA(c, cudaEventRecord(c->ev_in, c->user));
+  for (int i = 0; i < kNumStreams; ++i) c->forked[i] = false;
+  return DGS_OK;
+}
+int fork_from_user(dgs_ctx* c, int which) {
+  if (c->forked[which]) return DGS_OK;
   DGS_CUDA(c, cudaStreamWaitEvent(c->st[which], c->ev_in, 0));
+  c->forked[which] = true;
   return DGS_OK;
 }
 
-// Waits (on the host) for both internal streams and the caller's stream.
+// Waits (on the host) for all internal streams and the caller's stream.
 int sync_all(dgs_ctx* c) {
-  DGS_CUDA(c, cudaStreamSynchronize(c->st[0]));
-  DGS_CUDA(c, cudaStreamSynchronize(c->st[1]));
+  for (int i = 0; i < kNumStreams; ++i) DGS_CUDA(c, cudaStreamSynchronize(c->st[i]));
   DGS_CUDA(c, cudaStreamSynchronize(c->user));
   return DGS_OK;
 }
 
-// Most recent row of this kind made at an age <= `age`; -1 if there is none.
+// A task = the launches of one step on one stream.  task_begin makes the stream wait for
+// whatever the task depends on; task_end records the task's completion and files it with
+// the buffers it touched.
+struct Task {
+  int stream;
+  std::vector<uint32_t> reads, writes;
+};
+int task_begin(dgs_ctx* c, const Task& t) {
+  cudaEvent_t waited[64];
+  int nw = 0;
+  auto wait = [&](cudaEvent_t e, int s) -> int {
+    if (!e || s == t.stream) return DGS_OK;   // same stream: already ordered
+    for (int i = 0; i < nw; ++i)
+      if (waited[i] == e) return DGS_OK;
+    DGS_CUDA(c, cudaStreamWaitEvent(c->st[t.stream], e, 0));
+    if (nw < 64) waited[nw++] = e;
+    return DGS_OK;
+  };
+  for (uint32_t r : t.reads) {
+    const dgs_ctx::Res& x = c->res[r];
+    if (wait(x.last_write, x.write_stream) != DGS_OK) return DGS_ECUDA;
+  }
+  for (uint32_t w : t.writes) {
+    const dgs_ctx::Res& x = c->res[w];
+    if (wait(x.last_write, x.write_stream) != DGS_OK) return DGS_ECUDA;
+    for (const auto& rd : x.reads)
+      if (wait(rd.first, rd.second) != DGS_OK) return DGS_ECUDA;
+  }
+  return DGS_OK;
+}
+int task_end(dgs_ctx* c, const Task& t) {
+  cudaEvent_t e = c->ev_ring[c->ev_next];
+  c->ev_next = (c->ev_next + 1) % c->ev_ring.size();
+  DGS_CUDA(c, cudaEventRecord(e, c->st[t.stream]));
+  for (uint32_t r : t.reads) c->res[r].reads.push_back({e, t.stream});
+  for (uint32_t w : t.writes) {
+    dgs_ctx::Res& x = c->res[w];
+    x.last_write = e;
+    x.write_stream = t.stream;
+    x.reads.clear();
+  }
+  return DGS_OK;
+}
+
+// Row of carried bounds for a selection of this kind at this age: the most recent row made at
+// an age <= `age`, but preferably not the one written by the selection launched just before
+// (waiting for that one would chain consecutive selections together).  -1 if there is none.
 int pick_row(const dgs_ctx* c, int kind, uint64_t age) {
-  int best = -1;
+  int best = -1, best_old = -1;
+  const uint64_t newest = c->kind_seq[kind];
   for (uint32_t q = 0; q < c->cfg.num_workers; ++q) {
     if (!c->row_valid[kind][q] || c->row_age[kind][q] > age) continue;
     if (best < 0 || c->row_time[kind][q] > c->row_time[kind][best]) best = (int)q;
+    if (c->row_time[kind][q] < newest && (best_old < 0 || c->row_time[kind][q] > c->row_time[kind][best_old]))
+      best_old = (int)q;
   }
-  return best;
+  return best_old >= 0 ? best_old : best;
 }
 
 template <int MODE>
-int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age) {
+int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age, int stream_id, int set,
+                  Task& task) {
   constexpr int KIND = MODE == kPull ? 1 : 0;
-  cudaStream_t st = c->st[KIND];
-  Workspace& ws = c->ws[KIND];
+  const ResIds R{c->cfg.num_workers};
+  cudaStream_t st = c->st[stream_id];
+  Workspace& ws = c->ws[KIND * kSets + set];
   SelArgs a = a_in;
   a.speculate = (c->cfg.flags & DGS_NO_SPECULATION) ? 0 : 1;
   const int row = a.speculate ? pick_row(c, KIND, age) : -1;
@@ -298,11 +387,15 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age
   a.force_two_pass = single_pass ? 0 : 1;
   a.workers = (uint32_t)c->finalize_grid[MODE];
   a.seq = ++c->select_seq;
-  if (single_pass) {
-    a.L_in = c->L_next(KIND, (uint32_t)row);
-  } else {
+  a.L_in = single_pass ? c->L_next(KIND, (uint32_t)row) : ws.L_safe;
+  task.stream = stream_id;
+  if (single_pass && (uint32_t)row != worker) task.reads.push_back(R.ROW(KIND, (uint32_t)row));
+  if (a.speculate) task.writes.push_back(R.ROW(KIND, worker));
+  task.writes.push_back(R.SCR(KIND, set));
+  int rc = task_begin(c, task);
+  if (rc != DGS_OK) return rc;
+  if (!single_pass) {
     // nothing to go by: histogram of the whole input first, its bounds cannot fail
-    a.L_in = ws.L_safe;
     TimedLaunch t(c, st, MODE == kPull ? DGS_KERNEL_TWO_PASS_PULL : DGS_KERNEL_TWO_PASS_PUSH);
     k_hist_all<MODE><<<c->hist_grid[MODE], kThreads, 0, st>>>(ws, a);
     DGS_CUDA(c, cudaGetLastError());
@@ -325,9 +418,12 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age
                                             dim3(kThreads), args, 0, st));
     c->launches += 1;
   }
+  rc = task_end(c, task);
+  if (rc != DGS_OK) return rc;
+  c->kind_seq[KIND] += 1;
   if (a.speculate) {
     c->row_valid[KIND][worker] = 1;
-    c->row_time[KIND][worker] = c->select_seq;
+    c->row_time[KIND][worker] = c->kind_seq[KIND];
     c->row_age[KIND][worker] = age;
   }
   return DGS_OK;
@@ -356,15 +452,12 @@ int occupancy_grids(dgs_ctx* c, int sms) {
 }
 
 void destroy_ctx(dgs_ctx* c) {
-  for (int i = 0; i < 2; ++i) {
+  for (int i = 0; i < kNumStreams; ++i) {
     if (c->st[i]) cudaStreamDestroy(c->st[i]);
     if (c->ev_tail[i]) cudaEventDestroy(c->ev_tail[i]);
   }
-  for (int i = 0; i < kPushSlots; ++i) {
-    if (c->ev_push[i]) cudaEventDestroy(c->ev_push[i]);
-    if (c->ev_apply[i]) cudaEventDestroy(c->ev_apply[i]);
-  }
   if (c->ev_in) cudaEventDestroy(c->ev_in);
+  for (cudaEvent_t e : c->ev_ring) cudaEventDestroy(e);
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   c->magic = 0;
   delete c;
@@ -411,13 +504,17 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   c->segments.assign(cfg->segments, cfg->segments + cfg->num_segments);
   c->cfg.segments = c->segments.data();
   make_layout(&c->cfg, &c->lay);
-  c->st[0] = c->st[1] = nullptr;
-  c->ev_in = nullptr;
-  for (int i = 0; i < kPushSlots; ++i) {
-    c->ev_push[i] = c->ev_apply[i] = nullptr;
-    c->apply_pending[i] = false;
+  for (int i = 0; i < kNumStreams; ++i) {
+    c->st[i] = nullptr;
+    c->ev_tail[i] = nullptr;
+    c->forked[i] = false;
   }
-  c->ev_tail[0] = c->ev_tail[1] = nullptr;
+  c->ev_in = nullptr;
+  c->ev_next = 0;
+  c->pull_count = c->event_count = 0;
+  c->prev_pull_worker = -1;
+  c->kind_seq[0] = c->kind_seq[1] = 0;
+  c->res.assign(ResIds{cfg->num_workers}.count(), dgs_ctx::Res());
   if (c->lay.total > cfg->arena_bytes) {
     delete c;
     return DGS_ENOMEM;
@@ -462,15 +559,16 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   if (occupancy_grids<kPushSam>(c, sms) != DGS_OK || occupancy_grids<kPushResidual>(c, sms) != DGS_OK ||
       occupancy_grids<kPull>(c, sms) != DGS_OK)
     return fail(DGS_ECUDA);
-  for (int i = 0; i < 2; ++i) {
+  for (int i = 0; i < kNumStreams; ++i) {
     INIT_CUDA(cudaStreamCreateWithFlags(&c->st[i], cudaStreamNonBlocking));
     INIT_CUDA(cudaEventCreateWithFlags(&c->ev_tail[i], cudaEventDisableTiming));
   }
-  for (int i = 0; i < kPushSlots; ++i) {
-    INIT_CUDA(cudaEventCreateWithFlags(&c->ev_push[i], cudaEventDisableTiming));
-    INIT_CUDA(cudaEventCreateWithFlags(&c->ev_apply[i], cudaEventDisableTiming));
-  }
   INIT_CUDA(cudaEventCreateWithFlags(&c->ev_in, cudaEventDisableTiming));
+  for (int i = 0; i < 512; ++i) {
+    cudaEvent_t e;
+    INIT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    c->ev_ring.push_back(e);
+  }
 
   const Layout& L = c->lay;
   const uint64_t N = cfg->num_workers, vec = L.n_pad * 4;
@@ -481,7 +579,7 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   if (tiles.size() != L.num_tiles) return fail(DGS_EINVAL);
   cudaStream_t st = c->user;
   // state: u = 0, D = 0 (initialisation lines of Algorithm 3 and Algorithm 2), theta = theta_0
-  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.u), 0, vec * (N + 1), st));
+  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.u), 0, vec * (N + kSets), st));
   INIT_CUDA(cudaMemsetAsync(c->at<char>(L.D), 0, vec * N, st));
   INIT_CUDA(cudaMemsetAsync(c->at<char>(L.theta), 0, vec, st));
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.theta), cfg->theta0, cfg->n * 4, cudaMemcpyDeviceToDevice, st));
@@ -491,7 +589,7 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
       INIT_CUDA(cudaMemcpyAsync(c->theta_local_buf(q), cfg->theta0, cfg->n * 4, cudaMemcpyDeviceToDevice, st));
   }
   // scratch that kernels expect to find cleared, and the static tables
-  for (int k = 0; k < 2; ++k) {
+  for (int k = 0; k < 2 * kSets; ++k) {
     const ScratchLayout& sc = L.sc[k];
     INIT_CUDA(cudaMemsetAsync(c->at<char>(sc.zero_begin), 0, sc.zero_end - sc.zero_begin, st));
     INIT_CUDA(cudaMemsetAsync(c->at<char>(sc.part_cands), 0, (uint64_t)kMaxGrid * 4, st));
@@ -509,14 +607,14 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   seg_off[cfg->num_segments] = (uint32_t)cfg->n;  // n < 2^32
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.seg_off), seg_off.data(), seg_off.size() * 4, cudaMemcpyHostToDevice, st));
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.seg_tile0), seg_tile0.data(), seg_tile0.size() * 4, cudaMemcpyHostToDevice, st));
-  std::vector<float*> slots(N + 1);
-  for (uint32_t q = 0; q <= N; ++q) slots[q] = c->u_buf(q);
+  std::vector<float*> slots(N + kSets);
+  for (uint32_t q = 0; q < N + kSets; ++q) slots[q] = c->u_buf(q);
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.u_slots), slots.data(), slots.size() * sizeof(float*), cudaMemcpyHostToDevice, st));
   // the host vectors above go out of scope, and the library's own streams start from a ready arena
   INIT_CUDA(cudaStreamSynchronize(st));
 #undef INIT_CUDA
 
-  for (int k = 0; k < 2; ++k) {
+  for (int k = 0; k < 2 * kSets; ++k) {
     Workspace& w = c->ws[k];
     const ScratchLayout& sc = L.sc[k];
     w.tiles = c->at<Tile>(L.tiles);
@@ -545,35 +643,35 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   return DGS_OK;
 }
 
-int dgs_worker_push(dgs_ctx* c, uint32_t worker, const float* grad, dgs_packet* out) {
-  int rc = live(c);
-  if (rc != DGS_OK) return rc;
-  if (worker >= c->cfg.num_workers || !grad) return DGS_EINVAL;
-  if ((reinterpret_cast<uintptr_t>(grad) % 16) != 0) return DGS_EINVAL;
+namespace {
+
+int push_impl(dgs_ctx* c, uint32_t worker, const float* grad, dgs_packet* out, bool grad_is_stage) {
   const Layout& L = c->lay;
+  const ResIds R{c->cfg.num_workers};
   const int slot = (int)(c->push_count % kPushSlots);
-  rc = fork_from_user(c, 0);  // the gradient may have been produced on the caller's stream
+  const int set = (int)(c->push_count % kSets);
+  const int stream_id = kStW0 + (int)(c->push_count % kWorkerStreams);
+  int rc = fork_from_user(c, stream_id);  // the gradient may have been produced on the caller's stream
   if (rc != DGS_OK) return rc;
-  if (c->apply_pending[slot]) {  // the packet that lived in this slot must have been applied
-    DGS_CUDA(c, cudaStreamWaitEvent(c->st[0], c->ev_apply[slot], 0));
-    c->apply_pending[slot] = false;
-  }
   SelArgs a;
   std::memset(&a, 0, sizeof(a));
   a.grad = grad;
   a.u_cur_slot = c->u_slot(worker);
-  a.u_spare_slot = c->u_slot(c->cfg.num_workers);
+  a.u_spare_slot = c->u_slot(c->cfg.num_workers + set);
   a.pkt_idx = c->at<uint32_t>(L.pkt_idx[slot]);
   a.pkt_val = c->at<float>(L.pkt_val[slot]);
   a.pkt_count = (uint32_t)L.K[0];
   a.m = c->cfg.momentum;
   a.lr = c->cfg.lr;
   a.inv_m = c->inv_m;
+  Task task;
+  task.writes = {R.U(worker), R.SPARE(set), R.PKT(slot)};
+  if (grad_is_stage) task.reads.push_back(R.STAGE());
   const uint64_t age = c->pushes[worker];
-  rc = (c->cfg.flags & DGS_RESIDUAL_MODE) ? launch_select<kPushResidual>(c, a, worker, age)
-                                          : launch_select<kPushSam>(c, a, worker, age);
+  rc = (c->cfg.flags & DGS_RESIDUAL_MODE)
+           ? launch_select<kPushResidual>(c, a, worker, age, stream_id, set, task)
+           : launch_select<kPushSam>(c, a, worker, age, stream_id, set, task);
   if (rc != DGS_OK) return rc;
-  DGS_CUDA(c, cudaEventRecord(c->ev_push[slot], c->st[0]));
   c->pushes[worker] += 1;
   c->push_count += 1;
   if (out) {
@@ -584,60 +682,96 @@ int dgs_worker_push(dgs_ctx* c, uint32_t worker, const float* grad, dgs_packet* 
   return DGS_OK;
 }
 
-int dgs_server_apply(dgs_ctx* c, uint32_t worker, const dgs_packet* pkt) {
-  int rc = live(c);
-  if (rc != DGS_OK) return rc;
-  if (worker >= c->cfg.num_workers || !pkt) return DGS_EINVAL;
-  if (pkt->count > 0 && (!pkt->idx || !pkt->val)) return DGS_EINVAL;
-  // whose packet is it?  one of the push slots: wait for that push; anything else: the caller's stream
+int apply_impl(dgs_ctx* c, uint32_t worker, const dgs_packet* pkt) {
+  (void)worker;
+  const ResIds R{c->cfg.num_workers};
+  const uint32_t N = c->cfg.num_workers;
+  // whose packet is it?  one of the push slots: the tracker knows its writer; anything else: the caller's stream
   int slot = -1;
   for (int i = 0; i < kPushSlots; ++i)
     if (pkt->idx == c->at<uint32_t>(c->lay.pkt_idx[i])) slot = i;
-  if (slot >= 0) {
-    DGS_CUDA(c, cudaStreamWaitEvent(c->st[1], c->ev_push[slot], 0));
-  } else {
-    rc = fork_from_user(c, 1);
-    if (rc != DGS_OK) return rc;
-  }
   if (pkt->count > 0) {
-    const dim3 grid((pkt->count + kThreads - 1) / kThreads, c->cfg.num_workers + 1);
-    TimedLaunch t(c, c->st[1], DGS_KERNEL_SCATTER);
-    k_scatter_sub<<<grid, kThreads, 0, c->st[1]>>>(pkt->idx, pkt->val, pkt->count, c->at<float>(c->lay.theta),
-                                                   c->at<float>(c->lay.D), c->lay.n_pad, c->cfg.num_workers,
-                                                   c->cfg.n, c->ws[1].status);
-    DGS_CUDA(c, cudaGetLastError());
-    c->launches += 1;
-  }
-  if (slot >= 0) {
-    DGS_CUDA(c, cudaEventRecord(c->ev_apply[slot], c->st[1]));
-    c->apply_pending[slot] = true;
+    // The difference vector of the worker whose pull was enqueued last may still be in use by that
+    // pull: it gets its share of this packet in a launch of its own, so that the main launch (and
+    // with it the next pull) does not have to wait for that pull to finish.
+    const int skip = (N > 1 && c->prev_pull_worker >= 0) ? c->prev_pull_worker : -1;
+    const uint32_t gx = (pkt->count + kThreads - 1) / kThreads;
+    {
+      Task t;
+      t.stream = kStApply;
+      if (slot >= 0) t.reads.push_back(R.PKT(slot));
+      t.writes.push_back(R.THETA());
+      for (uint32_t q = 0; q < N; ++q)
+        if ((int)q != skip) t.writes.push_back(R.D(q));
+      int rc = slot >= 0 ? DGS_OK : fork_from_user(c, kStApply);
+      if (rc != DGS_OK) return rc;
+      rc = task_begin(c, t);
+      if (rc != DGS_OK) return rc;
+      {
+        TimedLaunch tl(c, c->st[kStApply], DGS_KERNEL_SCATTER);
+        const dim3 grid(gx, skip >= 0 ? N : N + 1);
+        k_scatter_sub<<<grid, kThreads, 0, c->st[kStApply]>>>(
+            pkt->idx, pkt->val, pkt->count, c->at<float>(c->lay.theta), c->at<float>(c->lay.D), c->lay.n_pad, N,
+            c->cfg.n, c->ws[0].status, 0u, skip >= 0 ? (uint32_t)skip : 0xFFFFFFFFu);
+        DGS_CUDA(c, cudaGetLastError());
+        c->launches += 1;
+      }
+      rc = task_end(c, t);
+      if (rc != DGS_OK) return rc;
+    }
+    if (skip >= 0) {
+      Task t;
+      t.stream = kStRest;
+      if (slot >= 0) t.reads.push_back(R.PKT(slot));
+      t.writes.push_back(R.D((uint32_t)skip));
+      int rc = slot >= 0 ? DGS_OK : fork_from_user(c, kStRest);
+      if (rc != DGS_OK) return rc;
+      rc = task_begin(c, t);
+      if (rc != DGS_OK) return rc;
+      {
+        TimedLaunch tl(c, c->st[kStRest], DGS_KERNEL_SCATTER);
+        k_scatter_sub<<<dim3(gx, 1), kThreads, 0, c->st[kStRest]>>>(
+            pkt->idx, pkt->val, pkt->count, c->at<float>(c->lay.theta), c->at<float>(c->lay.D), c->lay.n_pad, N,
+            c->cfg.n, c->ws[0].status, (uint32_t)skip, 0xFFFFFFFFu);
+        DGS_CUDA(c, cudaGetLastError());
+        c->launches += 1;
+      }
+      rc = task_end(c, t);
+      if (rc != DGS_OK) return rc;
+    }
   }
   c->timestamp += 1;  // t counts updates made to the server parameters
   return DGS_OK;
 }
 
-int dgs_worker_pull(dgs_ctx* c, uint32_t worker, dgs_packet* out) {
-  int rc = live(c);
-  if (rc != DGS_OK) return rc;
-  if (worker >= c->cfg.num_workers) return DGS_EINVAL;
+int pull_impl(dgs_ctx* c, uint32_t worker, dgs_packet* out) {
   const Layout& L = c->lay;
-  rc = fork_from_user(c, 1);  // the caller may still be reading the previous pull packet on its stream
+  const ResIds R{c->cfg.num_workers};
+  const int slot = kPushSlots + (int)(c->pull_count % kPullSlots);
+  const int set = (int)(c->pull_count % kSets);
+  const int stream_id = kStS0 + (int)(c->pull_count % kServerStreams);
+  int rc = fork_from_user(c, stream_id);  // the caller may still be reading an older pull packet on its stream
   if (rc != DGS_OK) return rc;
   SelArgs a;
   std::memset(&a, 0, sizeof(a));
   a.D = c->D_buf(worker);
   a.theta_local = (c->cfg.flags & DGS_KEEP_LOCAL_MODEL) ? c->theta_local_buf(worker) : nullptr;
-  a.pkt_idx = c->at<uint32_t>(L.pkt_idx[kPushSlots]);
-  a.pkt_val = c->at<float>(L.pkt_val[kPushSlots]);
+  a.pkt_idx = c->at<uint32_t>(L.pkt_idx[slot]);
+  a.pkt_val = c->at<float>(L.pkt_val[slot]);
   a.pkt_count = (uint32_t)L.K[1];
   a.m = c->cfg.momentum;
   a.lr = c->cfg.lr;
   a.inv_m = c->inv_m;
+  Task task;
+  task.writes = {R.D(worker), R.PKT(slot)};
+  if (a.theta_local) task.writes.push_back(R.TL(worker));
   // packets that entered D_worker since its previous pull
   const uint64_t age = c->timestamp - (c->prev[worker] < 0 ? 0 : (uint64_t)c->prev[worker]);
-  rc = launch_select<kPull>(c, a, worker, age);
+  rc = launch_select<kPull>(c, a, worker, age, stream_id, set, task);
   if (rc != DGS_OK) return rc;
   c->prev[worker] = (int64_t)c->timestamp;
+  c->pull_count += 1;
+  c->prev_pull_worker = (int)worker;
   if (out) {
     out->idx = a.pkt_idx;
     out->val = a.pkt_val;
@@ -646,13 +780,50 @@ int dgs_worker_pull(dgs_ctx* c, uint32_t worker, dgs_packet* out) {
   return DGS_OK;
 }
 
+}  // namespace
+
+int dgs_worker_push(dgs_ctx* c, uint32_t worker, const float* grad, dgs_packet* out) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (worker >= c->cfg.num_workers || !grad) return DGS_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(grad) % 16) != 0) return DGS_EINVAL;
+  rc = begin_call(c);
+  if (rc != DGS_OK) return rc;
+  return push_impl(c, worker, grad, out, false);
+}
+
+int dgs_server_apply(dgs_ctx* c, uint32_t worker, const dgs_packet* pkt) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (worker >= c->cfg.num_workers || !pkt) return DGS_EINVAL;
+  if (pkt->count > 0 && (!pkt->idx || !pkt->val)) return DGS_EINVAL;
+  rc = begin_call(c);
+  if (rc != DGS_OK) return rc;
+  return apply_impl(c, worker, pkt);
+}
+
+int dgs_worker_pull(dgs_ctx* c, uint32_t worker, dgs_packet* out) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (worker >= c->cfg.num_workers) return DGS_EINVAL;
+  rc = begin_call(c);
+  if (rc != DGS_OK) return rc;
+  return pull_impl(c, worker, out);
+}
+
 int dgs_event(dgs_ctx* c, uint32_t worker, const float* grad, dgs_packet* push_out, dgs_packet* pull_out) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (worker >= c->cfg.num_workers || !grad) return DGS_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(grad) % 16) != 0) return DGS_EINVAL;
+  rc = begin_call(c);
+  if (rc != DGS_OK) return rc;
   dgs_packet p, g;
-  int rc = dgs_worker_push(c, worker, grad, &p);
+  rc = push_impl(c, worker, grad, &p, false);
   if (rc != DGS_OK) return rc;
-  rc = dgs_server_apply(c, worker, &p);
+  rc = apply_impl(c, worker, &p);
   if (rc != DGS_OK) return rc;
-  rc = dgs_worker_pull(c, worker, &g);
+  rc = pull_impl(c, worker, &g);
   if (rc != DGS_OK) return rc;
   if (push_out) *push_out = p;
   if (pull_out) *pull_out = g;
@@ -662,7 +833,7 @@ int dgs_event(dgs_ctx* c, uint32_t worker, const float* grad, dgs_packet* push_o
 int dgs_flush(dgs_ctx* c) {
   int rc = live(c);
   if (rc != DGS_OK) return rc;
-  for (int i = 0; i < 2; ++i) {
+  for (int i = 0; i < kNumStreams; ++i) {
     DGS_CUDA(c, cudaEventRecord(c->ev_tail[i], c->st[i]));
     DGS_CUDA(c, cudaStreamWaitEvent(c->user, c->ev_tail[i], 0));
   }
@@ -673,15 +844,38 @@ int dgs_event_host(dgs_ctx* c, uint32_t worker, const float* grad_host, uint32_t
   int rc = live(c);
   if (rc != DGS_OK) return rc;
   if (!(c->cfg.flags & DGS_HOST_IO) || !grad_host || worker >= c->cfg.num_workers) return DGS_EINVAL;
-  float* stage = c->at<float>(c->lay.grad_stage);
-  // the staging buffer is read by pushes on the worker stream only, so the copy goes there too
-  DGS_CUDA(c, cudaMemcpyAsync(stage, grad_host, c->cfg.n * 4, cudaMemcpyHostToDevice, c->st[0]));
-  dgs_packet g;
-  rc = dgs_event(c, worker, stage, nullptr, &g);
+  rc = begin_call(c);
   if (rc != DGS_OK) return rc;
-  if (out_idx) DGS_CUDA(c, cudaMemcpyAsync(out_idx, g.idx, (uint64_t)g.count * 4, cudaMemcpyDeviceToHost, c->st[1]));
-  if (out_val) DGS_CUDA(c, cudaMemcpyAsync(out_val, g.val, (uint64_t)g.count * 4, cudaMemcpyDeviceToHost, c->st[1]));
-  DGS_CUDA(c, cudaStreamSynchronize(c->st[1]));
+  const ResIds R{c->cfg.num_workers};
+  float* stage = c->at<float>(c->lay.grad_stage);
+  {
+    // host -> staging buffer, on the stream of the push that will read it
+    Task t;
+    t.stream = kStW0 + (int)(c->push_count % kWorkerStreams);
+    t.writes.push_back(R.STAGE());
+    rc = fork_from_user(c, t.stream);
+    if (rc != DGS_OK) return rc;
+    rc = task_begin(c, t);
+    if (rc != DGS_OK) return rc;
+    DGS_CUDA(c, cudaMemcpyAsync(stage, grad_host, c->cfg.n * 4, cudaMemcpyHostToDevice, c->st[t.stream]));
+    rc = task_end(c, t);
+    if (rc != DGS_OK) return rc;
+  }
+  dgs_packet p, g;
+  rc = push_impl(c, worker, stage, &p, true);
+  if (rc != DGS_OK) return rc;
+  rc = apply_impl(c, worker, &p);
+  if (rc != DGS_OK) return rc;
+  const int pull_stream = kStS0 + (int)(c->pull_count % kServerStreams);
+  rc = pull_impl(c, worker, &g);
+  if (rc != DGS_OK) return rc;
+  cudaStream_t ps = c->st[pull_stream];
+  if (out_idx) DGS_CUDA(c, cudaMemcpyAsync(out_idx, g.idx, (uint64_t)g.count * 4, cudaMemcpyDeviceToHost, ps));
+  if (out_val) DGS_CUDA(c, cudaMemcpyAsync(out_val, g.val, (uint64_t)g.count * 4, cudaMemcpyDeviceToHost, ps));
+  // the event is complete when its pull is (the pull waited for the apply, the apply for the push),
+  // except for the share of the apply that runs on the side stream
+  DGS_CUDA(c, cudaStreamSynchronize(ps));
+  DGS_CUDA(c, cudaStreamSynchronize(c->st[kStRest]));
   return DGS_OK;
 }
 
@@ -699,9 +893,9 @@ int dgs_state_ptr(dgs_ctx* c, int which, uint32_t worker, const float** out) {
       break;
     case DGS_U: {
       float* p = nullptr;
-      DGS_CUDA(c, cudaMemcpyAsync(&p, c->u_slot(worker), sizeof(p), cudaMemcpyDeviceToHost, c->st[0]));
       rc = sync_all(c);
       if (rc != DGS_OK) return rc;
+      DGS_CUDA(c, cudaMemcpy(&p, c->u_slot(worker), sizeof(p), cudaMemcpyDeviceToHost));
       *out = p;
       return DGS_OK;
     }
@@ -717,13 +911,21 @@ int dgs_state_load(dgs_ctx* c, int which, uint32_t worker, const float* src) {
   const float* dst = nullptr;
   rc = dgs_state_ptr(c, which, worker, &dst);  // waits for all work in flight
   if (rc != DGS_OK) return rc;
-  // velocities are only touched on the worker stream, everything else on the server stream
-  const int which_stream = which == DGS_U ? 0 : 1;
-  rc = fork_from_user(c, which_stream);
+  rc = begin_call(c);
   if (rc != DGS_OK) return rc;
-  DGS_CUDA(c, cudaMemcpyAsync(const_cast<float*>(dst), src, c->cfg.n * 4, cudaMemcpyDeviceToDevice,
-                              c->st[which_stream]));
-  return DGS_OK;
+  const ResIds R{c->cfg.num_workers};
+  Task t;
+  t.stream = kStApply;
+  t.writes.push_back(which == DGS_THETA ? R.THETA()
+                     : which == DGS_U   ? R.U(worker)
+                     : which == DGS_D   ? R.D(worker)
+                                        : R.TL(worker));
+  rc = fork_from_user(c, t.stream);
+  if (rc != DGS_OK) return rc;
+  rc = task_begin(c, t);
+  if (rc != DGS_OK) return rc;
+  DGS_CUDA(c, cudaMemcpyAsync(const_cast<float*>(dst), src, c->cfg.n * 4, cudaMemcpyDeviceToDevice, c->st[t.stream]));
+  return task_end(c, t);
 }
 
 int dgs_status(dgs_ctx* c, int* device_status) {
@@ -803,8 +1005,7 @@ int dgs_last_cuda_error(dgs_ctx* c) {
 
 int dgs_free(dgs_ctx* c) {
   if (!c || c->magic != kMagic) return DGS_ESTATE;
-  cudaStreamSynchronize(c->st[0]);
-  cudaStreamSynchronize(c->st[1]);
+  for (int i = 0; i < kNumStreams; ++i) cudaStreamSynchronize(c->st[i]);
   cudaStreamSynchronize(c->user);
   destroy_ctx(c);
   return DGS_OK;

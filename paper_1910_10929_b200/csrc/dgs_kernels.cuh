@@ -1213,11 +1213,13 @@ __global__ void __launch_bounds__(kThreads, 2) k_stream(Workspace ws, SelArgs a)
 // ---- server apply ---------------------------------------------------------------
 // buffer q < N is D_q, buffer N is theta.  Indices of one packet are distinct, so every
 // (buffer, entry) pair is touched by exactly one thread: plain load / subtract / store.
+// One launch covers gridDim.y consecutive buffers starting at q_first, leaving out `skip`
+// (a difference vector that a pull is still working on gets its share in a launch of its own).
 __global__ void __launch_bounds__(kThreads) k_scatter_sub(const uint32_t* __restrict__ idx,
                                                           const float* __restrict__ val, uint32_t count,
                                                           float* __restrict__ theta, float* __restrict__ D,
                                                           uint64_t d_stride, uint32_t num_workers, uint64_t n,
-                                                          int* status) {
+                                                          int* status, uint32_t q_first, uint32_t skip) {
   const uint32_t j = blockIdx.x * kThreads + threadIdx.x;
   if (j >= count) return;
   const uint32_t i = idx[j];
@@ -1226,7 +1228,8 @@ __global__ void __launch_bounds__(kThreads) k_scatter_sub(const uint32_t* __rest
     atomicMin(status, -2000);
     return;
   }
-  const uint32_t q = blockIdx.y;
+  uint32_t q = q_first + blockIdx.y;
+  if (q >= skip) ++q;
   float* p = (q == num_workers ? theta : D + (uint64_t)q * d_stride) + i;
   *p = __fsub_rn(*p, v);
 }
