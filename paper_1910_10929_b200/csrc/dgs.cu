@@ -31,10 +31,14 @@ namespace {
 constexpr uint64_t kAlign = 256;
 constexpr uint32_t kMagic = 0x44475331u;  // "DGS1"
 constexpr int kPushSlots = 3;             // push packet slots, used in turn
-constexpr int kPullSlots = 2;             // pull packet slots
-constexpr int kSets = 2;                  // scratch sets (and spare velocity buffers) per kind of selection
-constexpr int kWorkerStreams = 2, kServerStreams = 2;
-enum StreamId : int { kStW0 = 0, kStW1 = 1, kStApply = 2, kStRest = 3, kStS0 = 4, kStS1 = 5, kNumStreams = 6 };
+constexpr int kPullSlots = 3;             // pull packet slots
+constexpr int kWorkerStreams = 2, kServerStreams = 3;
+constexpr int kPushSets = kWorkerStreams;  // scratch sets and spare velocity buffers of the pushes
+constexpr int kPullSets = kServerStreams;  // scratch sets of the pulls
+constexpr int kAllSets = kPushSets + kPullSets;
+constexpr int kMaxSkip = 3;               // difference vectors an apply may leave to side launches
+enum StreamId : int { kStW0 = 0, kStApply = kWorkerStreams, kStS0 = kWorkerStreams + 1,
+                      kNumStreams = kWorkerStreams + 1 + kServerStreams };
 
 inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
@@ -53,7 +57,7 @@ struct Layout {
   uint64_t theta, u, D, theta_local, grad_stage;
   uint64_t pkt_idx[kPushSlots + kPullSlots], pkt_val[kPushSlots + kPullSlots];  // push slots, then pull slots
   uint64_t tiles, segs, seg_off, seg_tile0;
-  ScratchLayout sc[2 * kSets];  // [kind * kSets + set]
+  ScratchLayout sc[kAllSets];  // push sets, then pull sets
   uint64_t L_next, u_slots, status, stats;
   uint64_t total = 0;
 };
@@ -134,7 +138,7 @@ void make_layout(const dgs_config* c, Layout* L) {
   };
   const uint64_t vec = L->n_pad * 4;
   L->theta = take(vec);
-  L->u = take(vec * (N + kSets));  // N velocities and the spares that pushes write into
+  L->u = take(vec * (N + kPushSets));  // N velocities and the spares that pushes write into
   L->D = take(vec * N);
   L->theta_local = (c->flags & DGS_KEEP_LOCAL_MODEL) ? take(vec * N) : 0;
   L->grad_stage = (c->flags & DGS_HOST_IO) ? take(vec) : 0;
@@ -147,7 +151,7 @@ void make_layout(const dgs_config* c, Layout* L) {
   L->segs = take(S * sizeof(SegDesc));
   L->seg_off = take((S + 1) * 4);
   L->seg_tile0 = take(S * 4);
-  for (int k = 0; k < 2 * kSets; ++k) {
+  for (int k = 0; k < kAllSets; ++k) {
     ScratchLayout& sc = L->sc[k];
     sc.cand_idx = take(vec);
     sc.cand_val = take(vec);
@@ -166,7 +170,7 @@ void make_layout(const dgs_config* c, Layout* L) {
     sc.zero_end = off;
   }
   L->L_next = take(2 * N * S * 4);
-  L->u_slots = take((N + kSets) * sizeof(float*));
+  L->u_slots = take((N + kPushSets) * sizeof(float*));
   L->status = take(4);
   L->stats = take(32 * 8);
   L->total = off;
@@ -195,8 +199,10 @@ struct dgs_ctx {
   std::vector<cudaEvent_t> ev_ring;  // one "done" event per task, reused in turn
   size_t ev_next;
   uint64_t push_count, pull_count, event_count;
-  int prev_pull_worker;    // worker whose pull was enqueued last (-1: none): its D is left to a launch of its own
-  Workspace ws[2 * kSets]; // [kind * kSets + set]
+  // workers whose pulls were enqueued last, newest first, and the stream each ran on: their difference
+  // vectors may still be in use, so an apply serves them with side launches on those streams
+  int recent_worker[kMaxSkip], recent_stream[kMaxSkip];
+  Workspace ws[kAllSets];  // push sets, then pull sets
   float inv_m;
   int stream_grid[3];    // CTAs of the stand-alone stream pass, per mode
   int hist_grid[3];      // CTAs of the whole-input histogram pass, per mode
@@ -245,9 +251,9 @@ struct ResIds {
   uint32_t ROW(int kind, uint32_t w) const { return 3 * N + (uint32_t)kind * N + w; }
   uint32_t THETA() const { return 5 * N; }
   uint32_t SPARE(int j) const { return 5 * N + 1 + j; }
-  uint32_t SCR(int kind, int set) const { return 5 * N + 1 + kSets + kind * kSets + set; }
-  uint32_t PKT(int slot) const { return 5 * N + 1 + 3 * kSets + slot; }   // push slots, then pull slots
-  uint32_t STAGE() const { return 5 * N + 1 + 3 * kSets + kPushSlots + kPullSlots; }
+  uint32_t SCR(int kind, int set) const { return 5 * N + 1 + kPushSets + (kind ? kPushSets : 0) + set; }
+  uint32_t PKT(int slot) const { return 5 * N + 1 + kPushSets + kAllSets + slot; }   // push slots, then pull slots
+  uint32_t STAGE() const { return PKT(kPushSlots + kPullSlots); }
   uint32_t count() const { return STAGE() + 1; }
 };
 
@@ -378,7 +384,7 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age
   constexpr int KIND = MODE == kPull ? 1 : 0;
   const ResIds R{c->cfg.num_workers};
   cudaStream_t st = c->st[stream_id];
-  Workspace& ws = c->ws[KIND * kSets + set];
+  Workspace& ws = c->ws[(KIND ? kPushSets : 0) + set];
   SelArgs a = a_in;
   a.speculate = (c->cfg.flags & DGS_NO_SPECULATION) ? 0 : 1;
   const int row = a.speculate ? pick_row(c, KIND, age) : -1;
@@ -512,7 +518,7 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   c->ev_in = nullptr;
   c->ev_next = 0;
   c->pull_count = c->event_count = 0;
-  c->prev_pull_worker = -1;
+  for (int i = 0; i < kMaxSkip; ++i) c->recent_worker[i] = c->recent_stream[i] = -1;
   c->kind_seq[0] = c->kind_seq[1] = 0;
   c->res.assign(ResIds{cfg->num_workers}.count(), dgs_ctx::Res());
   if (c->lay.total > cfg->arena_bytes) {
@@ -579,7 +585,7 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   if (tiles.size() != L.num_tiles) return fail(DGS_EINVAL);
   cudaStream_t st = c->user;
   // state: u = 0, D = 0 (initialisation lines of Algorithm 3 and Algorithm 2), theta = theta_0
-  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.u), 0, vec * (N + kSets), st));
+  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.u), 0, vec * (N + kPushSets), st));
   INIT_CUDA(cudaMemsetAsync(c->at<char>(L.D), 0, vec * N, st));
   INIT_CUDA(cudaMemsetAsync(c->at<char>(L.theta), 0, vec, st));
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.theta), cfg->theta0, cfg->n * 4, cudaMemcpyDeviceToDevice, st));
@@ -589,7 +595,7 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
       INIT_CUDA(cudaMemcpyAsync(c->theta_local_buf(q), cfg->theta0, cfg->n * 4, cudaMemcpyDeviceToDevice, st));
   }
   // scratch that kernels expect to find cleared, and the static tables
-  for (int k = 0; k < 2 * kSets; ++k) {
+  for (int k = 0; k < kAllSets; ++k) {
     const ScratchLayout& sc = L.sc[k];
     INIT_CUDA(cudaMemsetAsync(c->at<char>(sc.zero_begin), 0, sc.zero_end - sc.zero_begin, st));
     INIT_CUDA(cudaMemsetAsync(c->at<char>(sc.part_cands), 0, (uint64_t)kMaxGrid * 4, st));
@@ -607,14 +613,14 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   seg_off[cfg->num_segments] = (uint32_t)cfg->n;  // n < 2^32
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.seg_off), seg_off.data(), seg_off.size() * 4, cudaMemcpyHostToDevice, st));
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.seg_tile0), seg_tile0.data(), seg_tile0.size() * 4, cudaMemcpyHostToDevice, st));
-  std::vector<float*> slots(N + kSets);
-  for (uint32_t q = 0; q < N + kSets; ++q) slots[q] = c->u_buf(q);
+  std::vector<float*> slots(N + kPushSets);
+  for (uint32_t q = 0; q < N + kPushSets; ++q) slots[q] = c->u_buf(q);
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.u_slots), slots.data(), slots.size() * sizeof(float*), cudaMemcpyHostToDevice, st));
   // the host vectors above go out of scope, and the library's own streams start from a ready arena
   INIT_CUDA(cudaStreamSynchronize(st));
 #undef INIT_CUDA
 
-  for (int k = 0; k < 2 * kSets; ++k) {
+  for (int k = 0; k < kAllSets; ++k) {
     Workspace& w = c->ws[k];
     const ScratchLayout& sc = L.sc[k];
     w.tiles = c->at<Tile>(L.tiles);
@@ -649,7 +655,7 @@ int push_impl(dgs_ctx* c, uint32_t worker, const float* grad, dgs_packet* out, b
   const Layout& L = c->lay;
   const ResIds R{c->cfg.num_workers};
   const int slot = (int)(c->push_count % kPushSlots);
-  const int set = (int)(c->push_count % kSets);
+  const int set = (int)(c->push_count % kPushSets);
   const int stream_id = kStW0 + (int)(c->push_count % kWorkerStreams);
   int rc = fork_from_user(c, stream_id);  // the gradient may have been produced on the caller's stream
   if (rc != DGS_OK) return rc;
@@ -691,48 +697,67 @@ int apply_impl(dgs_ctx* c, uint32_t worker, const dgs_packet* pkt) {
   for (int i = 0; i < kPushSlots; ++i)
     if (pkt->idx == c->at<uint32_t>(c->lay.pkt_idx[i])) slot = i;
   if (pkt->count > 0) {
-    // The difference vector of the worker whose pull was enqueued last may still be in use by that
-    // pull: it gets its share of this packet in a launch of its own, so that the main launch (and
-    // with it the next pull) does not have to wait for that pull to finish.
-    const int skip = (N > 1 && c->prev_pull_worker >= 0) ? c->prev_pull_worker : -1;
+    // The difference vectors of the workers pulled last may still be in use by those pulls.  Each gets
+    // its share of this packet in a launch of its own, on the stream its pull ran on, so that the
+    // main launch (and with it the next pulls) does not have to wait for those pulls to finish.
+    uint32_t skip[kMaxSkip];
+    int skip_stream[kMaxSkip], ns = 0;
+    for (int i = 0; i < kMaxSkip && ns + 1 < (int)N; ++i) {
+      const int w = c->recent_worker[i];
+      if (w < 0) continue;
+      bool dup = false;
+      for (int j = 0; j < ns; ++j) dup = dup || skip[j] == (uint32_t)w;
+      if (dup) continue;
+      skip[ns] = (uint32_t)w;
+      skip_stream[ns] = c->recent_stream[i];
+      ++ns;
+    }
+    uint32_t sorted[kMaxSkip] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
+    for (int i = 0; i < ns; ++i) sorted[i] = skip[i];
+    std::sort(sorted, sorted + kMaxSkip);
+    // (the kernel finds the k-th buffer that is not skipped by bumping past the skipped ones in ascending order)
+    const uint32_t s0 = sorted[0], s1 = sorted[1], s2 = sorted[2];
     const uint32_t gx = (pkt->count + kThreads - 1) / kThreads;
     {
       Task t;
       t.stream = kStApply;
       if (slot >= 0) t.reads.push_back(R.PKT(slot));
       t.writes.push_back(R.THETA());
-      for (uint32_t q = 0; q < N; ++q)
-        if ((int)q != skip) t.writes.push_back(R.D(q));
+      for (uint32_t q = 0; q < N; ++q) {
+        bool skipped = false;
+        for (int j = 0; j < ns; ++j) skipped = skipped || skip[j] == q;
+        if (!skipped) t.writes.push_back(R.D(q));
+      }
       int rc = slot >= 0 ? DGS_OK : fork_from_user(c, kStApply);
       if (rc != DGS_OK) return rc;
       rc = task_begin(c, t);
       if (rc != DGS_OK) return rc;
       {
         TimedLaunch tl(c, c->st[kStApply], DGS_KERNEL_SCATTER);
-        const dim3 grid(gx, skip >= 0 ? N : N + 1);
+        const dim3 grid(gx, N + 1 - ns);
         k_scatter_sub<<<grid, kThreads, 0, c->st[kStApply]>>>(
             pkt->idx, pkt->val, pkt->count, c->at<float>(c->lay.theta), c->at<float>(c->lay.D), c->lay.n_pad, N,
-            c->cfg.n, c->ws[0].status, 0u, skip >= 0 ? (uint32_t)skip : 0xFFFFFFFFu);
+            c->cfg.n, c->ws[0].status, 0u, s0, s1, s2);
         DGS_CUDA(c, cudaGetLastError());
         c->launches += 1;
       }
       rc = task_end(c, t);
       if (rc != DGS_OK) return rc;
     }
-    if (skip >= 0) {
+    for (int i = 0; i < ns; ++i) {
       Task t;
-      t.stream = kStRest;
+      t.stream = skip_stream[i];
       if (slot >= 0) t.reads.push_back(R.PKT(slot));
-      t.writes.push_back(R.D((uint32_t)skip));
-      int rc = slot >= 0 ? DGS_OK : fork_from_user(c, kStRest);
+      t.writes.push_back(R.D(skip[i]));
+      int rc = slot >= 0 ? DGS_OK : fork_from_user(c, t.stream);
       if (rc != DGS_OK) return rc;
       rc = task_begin(c, t);
       if (rc != DGS_OK) return rc;
       {
-        TimedLaunch tl(c, c->st[kStRest], DGS_KERNEL_SCATTER);
-        k_scatter_sub<<<dim3(gx, 1), kThreads, 0, c->st[kStRest]>>>(
+        TimedLaunch tl(c, c->st[t.stream], DGS_KERNEL_SCATTER);
+        k_scatter_sub<<<dim3(gx, 1), kThreads, 0, c->st[t.stream]>>>(
             pkt->idx, pkt->val, pkt->count, c->at<float>(c->lay.theta), c->at<float>(c->lay.D), c->lay.n_pad, N,
-            c->cfg.n, c->ws[0].status, (uint32_t)skip, 0xFFFFFFFFu);
+            c->cfg.n, c->ws[0].status, skip[i], 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
         DGS_CUDA(c, cudaGetLastError());
         c->launches += 1;
       }
@@ -748,7 +773,7 @@ int pull_impl(dgs_ctx* c, uint32_t worker, dgs_packet* out) {
   const Layout& L = c->lay;
   const ResIds R{c->cfg.num_workers};
   const int slot = kPushSlots + (int)(c->pull_count % kPullSlots);
-  const int set = (int)(c->pull_count % kSets);
+  const int set = (int)(c->pull_count % kPullSets);
   const int stream_id = kStS0 + (int)(c->pull_count % kServerStreams);
   int rc = fork_from_user(c, stream_id);  // the caller may still be reading an older pull packet on its stream
   if (rc != DGS_OK) return rc;
@@ -771,7 +796,12 @@ int pull_impl(dgs_ctx* c, uint32_t worker, dgs_packet* out) {
   if (rc != DGS_OK) return rc;
   c->prev[worker] = (int64_t)c->timestamp;
   c->pull_count += 1;
-  c->prev_pull_worker = (int)worker;
+  for (int i = kMaxSkip - 1; i > 0; --i) {
+    c->recent_worker[i] = c->recent_worker[i - 1];
+    c->recent_stream[i] = c->recent_stream[i - 1];
+  }
+  c->recent_worker[0] = (int)worker;
+  c->recent_stream[0] = stream_id;
   if (out) {
     out->idx = a.pkt_idx;
     out->val = a.pkt_val;
@@ -873,9 +903,9 @@ int dgs_event_host(dgs_ctx* c, uint32_t worker, const float* grad_host, uint32_t
   if (out_idx) DGS_CUDA(c, cudaMemcpyAsync(out_idx, g.idx, (uint64_t)g.count * 4, cudaMemcpyDeviceToHost, ps));
   if (out_val) DGS_CUDA(c, cudaMemcpyAsync(out_val, g.val, (uint64_t)g.count * 4, cudaMemcpyDeviceToHost, ps));
   // the event is complete when its pull is (the pull waited for the apply, the apply for the push),
-  // except for the share of the apply that runs on the side stream
+  // except for the shares of the apply that run on the other server streams
   DGS_CUDA(c, cudaStreamSynchronize(ps));
-  DGS_CUDA(c, cudaStreamSynchronize(c->st[kStRest]));
+  for (int i = 0; i < kServerStreams; ++i) DGS_CUDA(c, cudaStreamSynchronize(c->st[kStS0 + i]));
   return DGS_OK;
 }
 

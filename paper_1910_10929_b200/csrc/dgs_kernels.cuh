@@ -1213,13 +1213,14 @@ __global__ void __launch_bounds__(kThreads, 2) k_stream(Workspace ws, SelArgs a)
 // ---- server apply ---------------------------------------------------------------
 // buffer q < N is D_q, buffer N is theta.  Indices of one packet are distinct, so every
 // (buffer, entry) pair is touched by exactly one thread: plain load / subtract / store.
-// One launch covers gridDim.y consecutive buffers starting at q_first, leaving out `skip`
-// (a difference vector that a pull is still working on gets its share in a launch of its own).
+// One launch covers gridDim.y buffers counted from q_first, leaving out up to three (a
+// difference vector that a pull is still working on gets its share in a launch of its own).
 __global__ void __launch_bounds__(kThreads) k_scatter_sub(const uint32_t* __restrict__ idx,
                                                           const float* __restrict__ val, uint32_t count,
                                                           float* __restrict__ theta, float* __restrict__ D,
                                                           uint64_t d_stride, uint32_t num_workers, uint64_t n,
-                                                          int* status, uint32_t q_first, uint32_t skip) {
+                                                          int* status, uint32_t q_first, uint32_t skip0,
+                                                          uint32_t skip1, uint32_t skip2) {
   const uint32_t j = blockIdx.x * kThreads + threadIdx.x;
   if (j >= count) return;
   const uint32_t i = idx[j];
@@ -1228,8 +1229,10 @@ __global__ void __launch_bounds__(kThreads) k_scatter_sub(const uint32_t* __rest
     atomicMin(status, -2000);
     return;
   }
-  uint32_t q = q_first + blockIdx.y;
-  if (q >= skip) ++q;
+  uint32_t q = q_first + blockIdx.y;   // the blockIdx.y-th buffer that is not skipped (skip0 <= skip1 <= skip2)
+  if (q >= skip0) ++q;
+  if (q >= skip1) ++q;
+  if (q >= skip2) ++q;
   float* p = (q == num_workers ? theta : D + (uint64_t)q * d_stride) + i;
   *p = __fsub_rn(*p, v);
 }
