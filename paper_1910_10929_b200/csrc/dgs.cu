@@ -45,7 +45,7 @@ inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 // Scratch of one selection pipeline ([0] push, on the worker stream; [1] pull, on the server stream)
 struct ScratchLayout {
   uint64_t cand_idx, cand_val, part_cands, part_slot0, tile_pre, cta_tot, tile_sel;
-  uint64_t hist1, hist2, hist3, sel, L_safe, sync;
+  uint64_t hist1, hist2, hist3, sel, L_safe, L_wide, sync;
   uint64_t zero_begin, zero_end;  // [tile_sel, end of sync): cleared at init
 };
 
@@ -166,6 +166,7 @@ void make_layout(const dgs_config* c, Layout* L) {
     sc.hist3 = take(S * kBins3 * 4);
     sc.sel = take(S * sizeof(SegSel));
     sc.L_safe = take(S * 4);
+    sc.L_wide = take(S * 4);
     sc.sync = take(kNumSyncWords * 4);
     sc.zero_end = off;
   }
@@ -274,7 +275,7 @@ inline int live(dgs_ctx* c) {
 }
 
 constexpr size_t kMaxTimedLaunches = 1 << 16;
-constexpr int kFinalizeWorkers = 64;  // CTAs of the finalize kernel
+constexpr int kFinalizeWorkers = 64;  // CTAs of the finalize kernel (more of them take SM slots from the stream passes)
 
 // Records an event before and after one launch when timing is on.
 struct TimedLaunch {
@@ -641,6 +642,7 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
     w.hist3 = c->at<uint32_t>(sc.hist3);
     w.sel = c->at<SegSel>(sc.sel);
     w.L_safe = c->at<uint32_t>(sc.L_safe);
+    w.L_wide = c->at<uint32_t>(sc.L_wide);
     w.sync = c->at<uint32_t>(sc.sync);
     w.status = c->at<int>(L.status);
     w.stats = c->at<unsigned long long>(L.stats);
@@ -1067,6 +1069,7 @@ struct StaticScratch {
   uint32_t seg_off[2];
   uint32_t seg_tile0[1];
   uint32_t L_safe[1];
+  uint32_t L_wide[1];
   uint32_t L_next[1];
   uint32_t sync[kNumSyncWords];
   int status;
@@ -1181,6 +1184,7 @@ extern "C" int dgs_topk_encode_static(const float* x, uint32_t n, uint32_t k, ui
   ws.hist3 = sc->hist3;
   ws.sel = &sc->sel;
   ws.L_safe = sc->L_safe;
+  ws.L_wide = sc->L_wide;
   ws.sync = sc->sync;
   ws.status = &sc->status;
   ws.stats = sc->stats;

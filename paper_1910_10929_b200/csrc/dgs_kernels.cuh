@@ -35,7 +35,7 @@ constexpr int kBins1 = 2048;        // key bits 30..20
 constexpr int kBins2 = 1024;        // key bits 19..10
 constexpr int kBins3 = 1024;        // key bits  9..0
 constexpr uint32_t kFull = 0xFFFFFFFFu;
-constexpr uint32_t kSpecFactor = 3; // aim for max(3k, k+64) candidates next time
+constexpr uint32_t kSpecFactor = 2; // aim for max(2k, k+64) candidates next time
 constexpr uint32_t kSpecSlack = 64;
 constexpr int kMaxGrid = 1024;      // upper bound on the grid of a stream pass (= parts of the candidate buffer)
 constexpr int kMaxWorkers = 128;    // upper bound on the grid of finalize
@@ -86,6 +86,7 @@ struct Workspace {
   uint32_t* hist3;        // [S][kBins3]
   SegSel* sel;            // [S]
   uint32_t* L_safe;       // [S] bound from the whole-input histogram (two-pass route)
+  uint32_t* L_wide;       // [S] from the same histogram: the bound that admits max(3k, k+64) entries
   uint32_t* sync;         // [kNumSyncWords]
   int* status;            // sticky device status word
   unsigned long long* stats;  // [0] single-pass selections, [1] two-pass selections, [2] candidates seen
@@ -787,8 +788,16 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
       for (uint32_t s = cta; s < S; s += W) {
         uint32_t bin, krem;
         uint32_t* h = ws.hist1 + (size_t)s * kBins1;
-        block_pick<kBins1>(h, ws.segs[s].k[PM], bin, krem, sh.warp_scan, sh.res);
-        if (threadIdx.x == 0) ws.L_safe[s] = bin << 20;
+        const uint32_t k = ws.segs[s].k[PM];
+        const uint32_t total = block_pick<kBins1>(h, k, bin, krem, sh.warp_scan, sh.res);
+        uint32_t wbin = 0, wrem;
+        const uint32_t want = max(k * kSpecFactor, k + kSpecSlack);
+        if (total >= want) block_pick<kBins1>(h, want, wbin, wrem, sh.warp_scan, sh.res);
+        if (threadIdx.x == 0) {
+          ws.L_safe[s] = bin << 20;
+          ws.L_wide[s] = wbin << 20;   // 0 (everything) when the layer has fewer than `want` entries
+        }
+        __syncthreads();
         for (int b = threadIdx.x; b < kBins1; b += kThreads) h[b] = 0;
       }
       if (cta == 0 && threadIdx.x == 0) ws.sync[kFail] = 0;
@@ -862,9 +871,12 @@ __global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs 
           uint32_t lbin, lrem;
           if (total >= want) {
             block_pick<kBins1>(h, want, lbin, lrem, sh.warp_scan, sh.res);
+          } else if (redo || a.force_two_pass) {
+            lbin = __ldcg(ws.L_wide + s) >> 20;   // known exactly from the histogram of the whole input
           } else {
-            const uint32_t used = (redo ? __ldcg(ws.L_safe + s) : a.L_in[s]) >> 20;
-            lbin = used > 0 ? used - 1 : 0;
+            // fewer candidates than wished for and nothing known below the bound: lower it by half an octave
+            const uint32_t used = a.L_in[s] >> 20;
+            lbin = used > 4 ? used - 4 : 0;
           }
           __syncthreads();
           if (threadIdx.x == 0) a.L_next[s] = lbin << 20;
@@ -1175,7 +1187,8 @@ __global__ void __launch_bounds__(kThreads, 4) k_hist_all(Workspace ws, SelArgs 
   hist_all_tiles<MODE>(ws, a, in, blockIdx.x, gridDim.x, s_hist);
 }
 
-// one CTA per layer (strided): L_safe = lower edge of the top-11-bit bin holding the k-th largest key
+// one CTA per layer (strided): L_safe = lower edge of the top-11-bit bin holding the k-th largest key,
+// L_wide = the same for the max(3k, k+64)-th largest (the bound suggested for later selections)
 template <int MODE>
 __global__ void __launch_bounds__(kThreads) k_pick_lower(Workspace ws) {
   __shared__ unsigned long long s_warp[kWarps];
@@ -1184,8 +1197,16 @@ __global__ void __launch_bounds__(kThreads) k_pick_lower(Workspace ws) {
   for (uint32_t s = blockIdx.x; s < ws.num_segs; s += gridDim.x) {
     uint32_t bin, krem;
     uint32_t* h = ws.hist1 + (size_t)s * kBins1;
-    block_pick<kBins1>(h, ws.segs[s].k[PM], bin, krem, s_warp, s_res);
-    if (threadIdx.x == 0) ws.L_safe[s] = bin << 20;
+    const uint32_t k = ws.segs[s].k[PM];
+    const uint32_t total = block_pick<kBins1>(h, k, bin, krem, s_warp, s_res);
+    uint32_t wbin = 0, wrem;
+    const uint32_t want = max(k * kSpecFactor, k + kSpecSlack);
+    if (total >= want) block_pick<kBins1>(h, want, wbin, wrem, s_warp, s_res);
+    if (threadIdx.x == 0) {
+      ws.L_safe[s] = bin << 20;
+      ws.L_wide[s] = wbin << 20;
+    }
+    __syncthreads();
     for (int b = threadIdx.x; b < kBins1; b += kThreads) h[b] = 0;
   }
 }
