@@ -361,6 +361,92 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
     return out
 
 
+
+def run_sweep(args) -> dict:
+    """Kernel sweep on one flat vector: n = 2^16 .. 2^28 in powers of 4, density 0.01 % .. 10 %,
+    values N(0,1) with 1 % of positions scaled by 100.  Times, per cell and cold (a 512 MB buffer
+    is rewritten between measurements): the selection + encoding of a pull on the two-pass
+    route (nothing carried over: histogram pass + stream pass + finalize) and on the single-pass
+    route (bound carried over from the previous selection), and the apply of the resulting
+    packet into 2 buffers (theta + 1 difference vector) and into 33 (theta + 32)."""
+    import torch
+
+    import paper_1910_10929_b200 as dgs
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, peak_kind = hbm_peak()
+    flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def timed(fn, ctx, reps=3):
+        out = []
+        for _ in range(reps):
+            flush_buf.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize(dev)
+            e0.record(stream)
+            fn()
+            ctx.flush()
+            e1.record(stream)
+            torch.cuda.synchronize(dev)
+            out.append(e0.elapsed_time(e1) * 1e3)
+        return statistics.median(out)
+
+    cells = []
+    for log2n in W.SWEEP_LOG2N:
+        if log2n > args.sweep_max_log2n:
+            continue
+        n = 1 << log2n
+        x = torch.from_numpy(W.sweep_values(n, args.seed, log2n)).to(dev)
+        for ppm in W.SWEEP_PPM:
+            k = W.k_of(n, ppm)
+            sel = dgs.Context(n, 1, 0.1, 0.9, [0], [n], [k], [k], torch.zeros(n, device=dev))
+
+            def pull_fresh():
+                sel.state_load(dgs.DGS_D, 0, x)
+                return sel.worker_pull(0)
+            # the first pull of a context has nothing to go by: two-pass route.  Time it on fresh contexts.
+            two_pass = []
+            for _ in range(3):
+                c2 = dgs.Context(n, 1, 0.1, 0.9, [0], [n], [k], [k], torch.zeros(n, device=dev))
+                c2.state_load(dgs.DGS_D, 0, x)
+                two_pass.append(timed(lambda: c2.worker_pull(0), c2, reps=1))
+                c2.close()
+            t_two = statistics.median(two_pass)
+            pull_fresh()                                   # leaves a carried bound behind
+            single = []
+            for _ in range(3):
+                sel.state_load(dgs.DGS_D, 0, x)
+                single.append(timed(lambda: sel.worker_pull(0), sel, reps=1))
+            t_single = statistics.median(single)
+            p = pull_fresh()
+            idx, val = sel.packet(p)
+            idx, val = idx.clone(), val.clone()
+            sel.close()
+            row = {"log2n": log2n, "density_ppm": ppm, "k": k,
+                   "select_two_pass_us": t_two, "select_single_pass_us": t_single,
+                   "select_two_pass_GBs": 4 * n / t_two / 1e3, "select_single_pass_GBs": 4 * n / t_single / 1e3,
+                   "select_single_pass_frac_of_peak": 4 * n / t_single / 1e3 / peak}
+            for nb_workers in (1, 32):
+                if (2 * nb_workers + 8) * 4 * n > 150e9:
+                    continue
+                ap = dgs.Context(n, nb_workers, 0.1, 0.9, [0], [n], [k], [k], torch.zeros(n, device=dev))
+                fp = dgs.dgs_packet(idx.data_ptr(), val.data_ptr(), k)
+                t_ap = timed(lambda: ap.server_apply(0, fp), ap)
+                ap.close()
+                bytes_alg = 8 * k * (nb_workers + 1) + 8 * k
+                row[f"scatter_{nb_workers + 1}buf_us"] = t_ap
+                row[f"scatter_{nb_workers + 1}buf_GBs"] = bytes_alg / t_ap / 1e3
+                row[f"scatter_{nb_workers + 1}buf_sector_GBs"] = 64 * k * (nb_workers + 1) / t_ap / 1e3
+            cells.append(row)
+            print(json.dumps(row), file=sys.stderr, flush=True)
+    return {"metric": "kernel sweep: select+compact and scatter GB/s", "unit": "GB/s", "peak_GB/s": peak,
+            "peak_kind": peak_kind, "data": "synthetic", "cells": cells,
+            "note": "select GB/s = 4n bytes (one read of the vector) / time; scatter GB/s = 8 bytes per "
+                    "(entry, buffer) + the packet / time, sector_GBs counts one 32-byte sector each way"}
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -374,6 +460,8 @@ def main() -> None:
                     help="override the number of simulated workers (smaller state for profiler captures)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="kernel sweep over vector sizes and densities")
+    ap.add_argument("--sweep-max-log2n", type=int, default=28)
     ap.add_argument("--traffic-bytes", type=float, default=None,
                     help="ncu dram bytes per launch of the dominant kernel, copied from profiles/")
     args = ap.parse_args()
@@ -383,6 +471,10 @@ def main() -> None:
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
 
+    if args.sweep:
+        if rank == 0:
+            print(json.dumps(run_sweep(args)), flush=True)
+        return
     if args.impl == "reference":
         if rank == 0:
             print(json.dumps(run_reference(args, make_workload(args.workload, args.seed, args.workers))), flush=True)

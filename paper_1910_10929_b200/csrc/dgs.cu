@@ -208,6 +208,7 @@ struct dgs_ctx {
   int stream_grid[3];    // CTAs of the stand-alone stream pass, per mode
   int hist_grid[3];      // CTAs of the whole-input histogram pass, per mode
   int finalize_grid[3];  // CTAs of the cooperative finalize kernel, per mode
+  int finalize_max[3];   // most CTAs of it that can be resident at once
   uint32_t select_seq;   // selections launched so far
   uint64_t kind_seq[2];  // selections of each kind launched so far
   // Carried bounds: row (kind, worker) of L_next holds the bounds suggested by that worker's
@@ -392,7 +393,9 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age
   const bool single_pass = row >= 0;
   a.L_next = c->L_next(KIND, worker);
   a.force_two_pass = single_pass ? 0 : 1;
-  a.workers = (uint32_t)c->finalize_grid[MODE];
+  // a selection of very many entries (dense packets) gets more CTAs: one more per 4096 entries
+  const int fin_grid = std::min(c->finalize_max[MODE], std::max(c->finalize_grid[MODE], (int)(a.pkt_count / 4096)));
+  a.workers = (uint32_t)fin_grid;
   a.seq = ++c->select_seq;
   a.L_in = single_pass ? c->L_next(KIND, (uint32_t)row) : ws.L_safe;
   task.stream = stream_id;
@@ -421,8 +424,8 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age
     // cooperative launch: the CTAs synchronise among themselves, so all must be resident
     TimedLaunch t(c, st, MODE == kPull ? DGS_KERNEL_FINALIZE_PULL : DGS_KERNEL_FINALIZE_PUSH);
     void* args[] = {(void*)&ws, (void*)&a};
-    DGS_CUDA(c, cudaLaunchCooperativeKernel((const void*)k_finalize<MODE>, dim3(c->finalize_grid[MODE]),
-                                            dim3(kThreads), args, 0, st));
+    DGS_CUDA(c, cudaLaunchCooperativeKernel((const void*)k_finalize<MODE>, dim3(fin_grid), dim3(kThreads), args, 0,
+                                            st));
     c->launches += 1;
   }
   rc = task_end(c, task);
@@ -454,7 +457,8 @@ int occupancy_grids(dgs_ctx* c, int sms) {
     c->broken = true;
     return DGS_ECUDA;
   }
-  c->finalize_grid[MODE] = std::min(std::min(sms * occ, kMaxWorkers), kFinalizeWorkers);
+  c->finalize_max[MODE] = std::min(sms * occ, kMaxWorkers);
+  c->finalize_grid[MODE] = std::min(c->finalize_max[MODE], kFinalizeWorkers);
   return DGS_OK;
 }
 

@@ -38,7 +38,7 @@ constexpr uint32_t kFull = 0xFFFFFFFFu;
 constexpr uint32_t kSpecFactor = 2; // aim for max(2k, k+64) candidates next time
 constexpr uint32_t kSpecSlack = 64;
 constexpr int kMaxGrid = 1024;      // upper bound on the grid of a stream pass (= parts of the candidate buffer)
-constexpr int kMaxWorkers = 128;    // upper bound on the grid of finalize
+constexpr int kMaxWorkers = 320;    // upper bound on the grid of finalize
 constexpr uint32_t kSpinLimit = 1u << 22;  // bounded waits: give up and report after this many polls
 constexpr int kStatusTimeout = -4;  // = DGS_ETIMEOUT
 
