@@ -84,3 +84,33 @@ def compare_state(ctx, orc, num_workers: int, keep_local: bool) -> None:
         same(dgs.DGS_D, oracle.D, q, "D")
         if keep_local:
             same(dgs.DGS_THETA_LOCAL, oracle.THETA_LOCAL, q, "theta_local")
+
+
+def replay_async_and_compare(wl, *, flags: int = 0, num_events=None, device: str = "cuda:0"):
+    """Enqueues all events back to back without ever waiting (the library's streams overlap
+    consecutive events), then replays the same events on the CPU checker and compares the
+    whole final state and the last packets bit for bit.  Any missing dependency between the
+    overlapped steps shows up as a difference."""
+    keep_local = bool(flags & dgs.DGS_KEEP_LOCAL_MODEL)
+    residual = bool(flags & dgs.DGS_RESIDUAL_MODE)
+    theta0 = wl.theta0()
+    sched = wl.schedule()
+    E = len(sched) if num_events is None else num_events
+    sched = np.resize(sched, E)
+    grads_host = [wl.gradient(e) for e in range(E)]
+    grads = [torch.from_numpy(g).to(device) for g in grads_host]      # alive until the end
+    ctx = dgs.Context.from_workload(wl, theta0=torch.from_numpy(theta0).to(device), flags=flags)
+    torch.cuda.synchronize()
+    last = None
+    for e in range(E):
+        last = ctx.event(int(sched[e]), grads[e])
+    pi, pv = packet_to_numpy(ctx, last[0])
+    gi, gv = packet_to_numpy(ctx, last[1])
+    assert ctx.status() == 0
+    orc = oracle.Oracle.from_workload(wl, keep_local=keep_local, residual_mode=residual, theta0=theta0)
+    for e in range(E):
+        (oi, ov), (qi, qv) = orc.event(int(sched[e]), grads_host[e])
+    assert np.array_equal(pi, oi) and np.array_equal(bits(pv), bits(ov)), "last push packet differs"
+    assert np.array_equal(gi, qi) and np.array_equal(bits(gv), bits(qv)), "last pull packet differs"
+    compare_state(ctx, orc, wl.num_workers, keep_local)
+    return ctx, orc

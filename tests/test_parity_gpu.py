@@ -11,7 +11,7 @@ import torch
 import oracle
 import paper_1910_10929_b200 as dgs
 import workloads as W
-from _replay import bits, key, packet_to_numpy, replay_and_compare
+from _replay import bits, key, packet_to_numpy, replay_and_compare, replay_async_and_compare
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -112,6 +112,26 @@ def test_trajectory_resnet18_per_layer():
 def test_trajectory_resnet50_global():
     wl = W.resnet50(num_workers=32, num_events=36)
     replay_and_compare(wl)
+
+
+@pytest.mark.parametrize("flags", [0, dgs.DGS_KEEP_LOCAL_MODEL, dgs.DGS_RESIDUAL_MODE])
+def test_overlapped_events_random_arrivals(flags):
+    # i.i.d. arrivals: the same worker often comes twice in a row, ages vary, bounds fail now and then
+    wl = W.custom("async", [150_000, 517, 90_000, 64, 70_001], 5, 150, 5_000, grad_kind="laplace",
+                  schedule_kind="uniform")
+    ctx, _ = replay_async_and_compare(wl, flags=flags)
+    assert ctx.stats()[0] > 0
+
+
+def test_overlapped_events_resnet50_32_workers():
+    # the benchmark's configuration, three rounds of the 32 workers, nothing waited for in between
+    wl = W.resnet50(num_workers=32, num_events=96)
+    replay_async_and_compare(wl)
+
+
+def test_overlapped_events_resnet18_per_layer():
+    wl = W.resnet18(num_workers=32, num_events=80)
+    replay_async_and_compare(wl)
 
 
 def test_trajectory_gpt2_small_few_workers():
