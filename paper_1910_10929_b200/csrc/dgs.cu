@@ -30,9 +30,9 @@ namespace {
 
 constexpr uint64_t kAlign = 256;
 constexpr uint32_t kMagic = 0x44475331u;  // "DGS1"
-constexpr int kPushSlots = 3;             // push packet slots, used in turn
+constexpr int kPushSlots = 4;             // push packet slots, used in turn
 constexpr int kPullSlots = 3;             // pull packet slots
-constexpr int kWorkerStreams = 2, kServerStreams = 3;
+constexpr int kWorkerStreams = 3, kServerStreams = 3;
 constexpr int kPushSets = kWorkerStreams;  // scratch sets and spare velocity buffers of the pushes
 constexpr int kPullSets = kServerStreams;  // scratch sets of the pulls
 constexpr int kAllSets = kPushSets + kPullSets;
