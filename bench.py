@@ -315,14 +315,15 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
     kernel_bytes = {
         "stream_push": 12 * wl.n, "finalize_push": None, "two_pass_push": 8 * wl.n,
         "scatter": None, "stream_pull": 4 * wl.n, "finalize_pull": None, "two_pass_pull": 4 * wl.n,
+        "catch_up": None,
     }
     achieved = kernel_bytes[dom] / (dom_ms * 1e-3 / max(dom_cnt, 1)) / 1e9
 
     def kernel_gbs(k, ms, cnt):
         if not cnt or ms <= 0:
             return None
-        if k == "scatter":          # several launches per event (main + side launches): bytes per event
-            return ab["apply"] * K / (ms * 1e-3) / 1e9
+        if k == "catch_up":         # the apply's bytes of an event (N + 1 buffers) over scatter + catch-up time
+            return ab["apply"] * K / ((ms + ktimes["scatter"][0]) * 1e-3) / 1e9
         return kernel_bytes[k] / (ms * 1e-3 / cnt) / 1e9 if kernel_bytes[k] else None
 
     traffic = args.traffic_bytes

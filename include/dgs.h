@@ -183,7 +183,8 @@ enum {
   DGS_KERNEL_STREAM_PULL = 4,
   DGS_KERNEL_FINALIZE_PULL = 5,
   DGS_KERNEL_TWO_PASS_PULL = 6,
-  DGS_NUM_KERNELS = 7
+  DGS_KERNEL_CATCH_UP = 7,      /* pull: applied packets folded into the worker's difference vector   */
+  DGS_NUM_KERNELS = 8
 };
 
 /* Measurement aid (no counterpart in the paper).  While on, every kernel launch of

@@ -27,9 +27,9 @@ EXPORTS = (
 )
 DGS_ELIMIT = -6
 DGS_STATIC_MAX_N = 1 << 20
-DGS_NUM_KERNELS = 7
+DGS_NUM_KERNELS = 8
 KERNEL_NAMES = ("stream_push", "finalize_push", "two_pass_push", "scatter", "stream_pull", "finalize_pull",
-                "two_pass_pull")
+                "two_pass_pull", "catch_up")
 
 
 class dgs_segment(C.Structure):

@@ -30,13 +30,13 @@ namespace {
 
 constexpr uint64_t kAlign = 256;
 constexpr uint32_t kMagic = 0x44475331u;  // "DGS1"
-constexpr int kPushSlots = 4;             // push packet slots, used in turn
-constexpr int kPullSlots = 3;             // pull packet slots
-constexpr int kWorkerStreams = 3, kServerStreams = 3;
+constexpr int kPushSlots = 5;             // push packet slots, used in turn
+constexpr int kPullSlots = 4;             // pull packet slots
+constexpr int kWorkerStreams = 4, kServerStreams = 4;
 constexpr int kPushSets = kWorkerStreams;  // scratch sets and spare velocity buffers of the pushes
 constexpr int kPullSets = kServerStreams;  // scratch sets of the pulls
 constexpr int kAllSets = kPushSets + kPullSets;
-constexpr int kMaxSkip = 3;               // difference vectors an apply may leave to side launches
+constexpr int kLogRingMax = 64;           // most packets the apply log keeps (k_catch_up holds two ranges per lane)
 enum StreamId : int { kStW0 = 0, kStApply = kWorkerStreams, kStS0 = kWorkerStreams + 1,
                       kNumStreams = kWorkerStreams + 1 + kServerStreams };
 
@@ -59,6 +59,8 @@ struct Layout {
   uint64_t tiles, segs, seg_off, seg_tile0;
   ScratchLayout sc[kAllSets];  // push sets, then pull sets
   uint64_t L_next, u_slots, status, stats;
+  uint64_t log_idx, log_val;  // ring of applied packets not yet folded into every D_q
+  uint32_t log_ring = 0, log_stride = 0;
   uint64_t total = 0;
 };
 
@@ -170,6 +172,10 @@ void make_layout(const dgs_config* c, Layout* L) {
     sc.sync = take(kNumSyncWords * 4);
     sc.zero_end = off;
   }
+  L->log_ring = (uint32_t)std::min<uint64_t>(kLogRingMax, std::max<uint64_t>(N + 8, 16));
+  L->log_stride = (uint32_t)align_up(L->K[0], 64);
+  L->log_idx = take((uint64_t)L->log_ring * L->log_stride * 4);
+  L->log_val = take((uint64_t)L->log_ring * L->log_stride * 4);
   L->L_next = take(2 * N * S * 4);
   L->u_slots = take((N + kPushSets) * sizeof(float*));
   L->status = take(4);
@@ -191,18 +197,28 @@ struct dgs_ctx {
   bool forked[kNumStreams];  // stream already waits for ev_in of the current call
   cudaEvent_t ev_tail[kNumStreams];  // for dgs_flush
   // dependency tracker
+  struct Dep {
+    cudaEvent_t ev = nullptr;
+    int stream = -1;
+    uint64_t seq = 0;  // position of the task in the order of all tasks (0: none)
+  };
   struct Res {
-    cudaEvent_t last_write = nullptr;
-    int write_stream = -1;
-    std::vector<std::pair<cudaEvent_t, int>> reads;  // readers since the last write (event, stream)
+    Dep last_write;
+    std::vector<Dep> reads;  // readers since the last write
   };
   std::vector<Res> res;
-  std::vector<cudaEvent_t> ev_ring;  // one "done" event per task, reused in turn
-  size_t ev_next;
+  // one "done" event per task, reused in turn; a ring per stream, so that an event is only ever
+  // re-recorded later on the same stream and waiting for a reused one still covers the older task
+  std::vector<cudaEvent_t> ev_ring[kNumStreams];
+  size_t ev_next[kNumStreams];
+  uint64_t task_seq;                               // tasks filed so far
+  uint64_t waited_seq[kNumStreams][kNumStreams];   // [waiting stream][stream]: newest task already waited for
   uint64_t push_count, pull_count, event_count;
-  // workers whose pulls were enqueued last, newest first, and the stream each ran on: their difference
-  // vectors may still be in use, so an apply serves them with side launches on those streams
-  int recent_worker[kMaxSkip], recent_stream[kMaxSkip];
+  // Lazy difference vectors: packet number p (counted from 0) of the library's own pushes sits in slot
+  // p % ring of the log from its apply on; applied[q] packets have been folded into D_q so far.
+  PacketLog log;
+  uint64_t log_head;              // packets filed so far
+  std::vector<uint64_t> applied;  // per worker
   Workspace ws[kAllSets];  // push sets, then pull sets
   float inv_m;
   int stream_grid[3];    // CTAs of the stand-alone stream pass, per mode
@@ -256,7 +272,8 @@ struct ResIds {
   uint32_t SCR(int kind, int set) const { return 5 * N + 1 + kPushSets + (kind ? kPushSets : 0) + set; }
   uint32_t PKT(int slot) const { return 5 * N + 1 + kPushSets + kAllSets + slot; }   // push slots, then pull slots
   uint32_t STAGE() const { return PKT(kPushSlots + kPullSlots); }
-  uint32_t count() const { return STAGE() + 1; }
+  uint32_t LOG(uint32_t slot) const { return STAGE() + 1 + slot; }
+  uint32_t count() const { return LOG(kLogRingMax); }
 };
 
 #define DGS_CUDA(ctx, call)                 \
@@ -329,53 +346,87 @@ struct Task {
   std::vector<uint32_t> reads, writes;
 };
 int task_begin(dgs_ctx* c, const Task& t) {
-  cudaEvent_t waited[64];
-  int nw = 0;
-  auto wait = [&](cudaEvent_t e, int s) -> int {
-    if (!e || s == t.stream) return DGS_OK;   // same stream: already ordered
-    for (int i = 0; i < nw; ++i)
-      if (waited[i] == e) return DGS_OK;
-    DGS_CUDA(c, cudaStreamWaitEvent(c->st[t.stream], e, 0));
-    if (nw < 64) waited[nw++] = e;
-    return DGS_OK;
+  // Tasks of one stream complete in order, so per stream only the newest task that this one depends
+  // on matters, and only if the stream has not already waited for that task or a newer one.
+  dgs_ctx::Dep need[kNumStreams];
+  auto want = [&](const dgs_ctx::Dep& d) {
+    if (!d.ev || d.stream == t.stream) return;   // same stream: already ordered
+    if (d.seq > need[d.stream].seq) need[d.stream] = d;
   };
-  for (uint32_t r : t.reads) {
-    const dgs_ctx::Res& x = c->res[r];
-    if (wait(x.last_write, x.write_stream) != DGS_OK) return DGS_ECUDA;
-  }
+  for (uint32_t r : t.reads) want(c->res[r].last_write);
   for (uint32_t w : t.writes) {
     const dgs_ctx::Res& x = c->res[w];
-    if (wait(x.last_write, x.write_stream) != DGS_OK) return DGS_ECUDA;
-    for (const auto& rd : x.reads)
-      if (wait(rd.first, rd.second) != DGS_OK) return DGS_ECUDA;
+    want(x.last_write);
+    for (const dgs_ctx::Dep& rd : x.reads) want(rd);
+  }
+  for (int s = 0; s < kNumStreams; ++s) {
+    if (!need[s].ev || need[s].seq <= c->waited_seq[t.stream][s]) continue;
+    DGS_CUDA(c, cudaStreamWaitEvent(c->st[t.stream], need[s].ev, 0));
+    c->waited_seq[t.stream][s] = need[s].seq;
   }
   return DGS_OK;
 }
 int task_end(dgs_ctx* c, const Task& t) {
-  cudaEvent_t e = c->ev_ring[c->ev_next];
-  c->ev_next = (c->ev_next + 1) % c->ev_ring.size();
-  DGS_CUDA(c, cudaEventRecord(e, c->st[t.stream]));
-  for (uint32_t r : t.reads) c->res[r].reads.push_back({e, t.stream});
+  dgs_ctx::Dep d;
+  d.ev = c->ev_ring[t.stream][c->ev_next[t.stream]];
+  d.stream = t.stream;
+  d.seq = ++c->task_seq;
+  c->ev_next[t.stream] = (c->ev_next[t.stream] + 1) % c->ev_ring[t.stream].size();
+  DGS_CUDA(c, cudaEventRecord(d.ev, c->st[t.stream]));
+  for (uint32_t r : t.reads) c->res[r].reads.push_back(d);
   for (uint32_t w : t.writes) {
     dgs_ctx::Res& x = c->res[w];
-    x.last_write = e;
-    x.write_stream = t.stream;
+    x.last_write = d;
     x.reads.clear();
   }
   return DGS_OK;
 }
 
+// Dependencies of folding the filed packets that D_q has not seen yet into it.
+void catch_up_deps(const dgs_ctx* c, uint32_t q, Task* t) {
+  const ResIds R{c->cfg.num_workers};
+  for (uint64_t p = c->applied[q]; p < c->log_head; ++p) t->reads.push_back(R.LOG((uint32_t)(p % c->log.ring)));
+  t->writes.push_back(R.D(q));
+}
+// The launch itself, on a stream that task_begin has prepared with those dependencies.
+int catch_up_launch(dgs_ctx* c, uint32_t q, cudaStream_t st) {
+  const uint64_t first = c->applied[q];
+  const uint32_t count = (uint32_t)(c->log_head - first);
+  if (count > 0) {
+    TimedLaunch tl(c, st, DGS_KERNEL_CATCH_UP);
+    k_catch_up<<<kCatchGrid, kThreads, 0, st>>>(c->log, first, count, c->D_buf(q), c->cfg.n);
+    DGS_CUDA(c, cudaGetLastError());
+    c->launches += 1;
+  }
+  c->applied[q] = c->log_head;
+  return DGS_OK;
+}
+// Both, as a task of its own on the apply stream.
+int catch_up_now(dgs_ctx* c, uint32_t q) {
+  if (c->applied[q] == c->log_head) return DGS_OK;
+  Task t;
+  t.stream = kStApply;
+  catch_up_deps(c, q, &t);
+  int rc = task_begin(c, t);
+  if (rc != DGS_OK) return rc;
+  rc = catch_up_launch(c, q, c->st[kStApply]);
+  if (rc != DGS_OK) return rc;
+  return task_end(c, t);
+}
+
 // Row of carried bounds for a selection of this kind at this age: the most recent row made at
-// an age <= `age`, but preferably not the one written by the selection launched just before
-// (waiting for that one would chain consecutive selections together).  -1 if there is none.
+// an age <= `age`, but preferably not one written by the selections that the other streams of
+// this kind are still working on (waiting for those would chain the streams together; the row
+// before them was written on this selection's own stream).  -1 if there is none.
 int pick_row(const dgs_ctx* c, int kind, uint64_t age) {
   int best = -1, best_old = -1;
+  const uint64_t in_flight = (uint64_t)(kind ? kServerStreams : kWorkerStreams) - 1;
   const uint64_t newest = c->kind_seq[kind];
   for (uint32_t q = 0; q < c->cfg.num_workers; ++q) {
     if (!c->row_valid[kind][q] || c->row_age[kind][q] > age) continue;
-    if (best < 0 || c->row_time[kind][q] > c->row_time[kind][best]) best = (int)q;
-    if (c->row_time[kind][q] < newest && (best_old < 0 || c->row_time[kind][q] > c->row_time[kind][best_old]))
-      best_old = (int)q;
+    const uint64_t t = c->row_time[kind][q];
+    if (best < 0 || t > c->row_time[kind][best]) best = (int)q;
+    if (t + in_flight <= newest && (best_old < 0 || t > c->row_time[kind][best_old])) best_old = (int)q;
   }
   return best_old >= 0 ? best_old : best;
 }
@@ -404,6 +455,10 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age
   task.writes.push_back(R.SCR(KIND, set));
   int rc = task_begin(c, task);
   if (rc != DGS_OK) return rc;
+  if (MODE == kPull) {
+    rc = catch_up_launch(c, worker, st);
+    if (rc != DGS_OK) return rc;
+  }
   if (!single_pass) {
     // nothing to go by: histogram of the whole input first, its bounds cannot fail
     TimedLaunch t(c, st, MODE == kPull ? DGS_KERNEL_TWO_PASS_PULL : DGS_KERNEL_TWO_PASS_PUSH);
@@ -468,7 +523,8 @@ void destroy_ctx(dgs_ctx* c) {
     if (c->ev_tail[i]) cudaEventDestroy(c->ev_tail[i]);
   }
   if (c->ev_in) cudaEventDestroy(c->ev_in);
-  for (cudaEvent_t e : c->ev_ring) cudaEventDestroy(e);
+  for (int i = 0; i < kNumStreams; ++i)
+    for (cudaEvent_t e : c->ev_ring[i]) cudaEventDestroy(e);
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   c->magic = 0;
   delete c;
@@ -521,9 +577,14 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
     c->forked[i] = false;
   }
   c->ev_in = nullptr;
-  c->ev_next = 0;
+  c->task_seq = 0;
+  for (int i = 0; i < kNumStreams; ++i) {
+    c->ev_next[i] = 0;
+    for (int j = 0; j < kNumStreams; ++j) c->waited_seq[i][j] = 0;
+  }
   c->pull_count = c->event_count = 0;
-  for (int i = 0; i < kMaxSkip; ++i) c->recent_worker[i] = c->recent_stream[i] = -1;
+  c->log_head = 0;
+  c->applied.assign(cfg->num_workers, 0);
   c->kind_seq[0] = c->kind_seq[1] = 0;
   c->res.assign(ResIds{cfg->num_workers}.count(), dgs_ctx::Res());
   if (c->lay.total > cfg->arena_bytes) {
@@ -575,11 +636,12 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
     INIT_CUDA(cudaEventCreateWithFlags(&c->ev_tail[i], cudaEventDisableTiming));
   }
   INIT_CUDA(cudaEventCreateWithFlags(&c->ev_in, cudaEventDisableTiming));
-  for (int i = 0; i < 512; ++i) {
-    cudaEvent_t e;
-    INIT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
-    c->ev_ring.push_back(e);
-  }
+  for (int s = 0; s < kNumStreams; ++s)
+    for (int i = 0; i < 256; ++i) {
+      cudaEvent_t e;
+      INIT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+      c->ev_ring[s].push_back(e);
+    }
 
   const Layout& L = c->lay;
   const uint64_t N = cfg->num_workers, vec = L.n_pad * 4;
@@ -651,6 +713,11 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
     w.status = c->at<int>(L.status);
     w.stats = c->at<unsigned long long>(L.stats);
   }
+  c->log.idx = c->at<uint32_t>(L.log_idx);
+  c->log.val = c->at<float>(L.log_val);
+  c->log.stride = L.log_stride;
+  c->log.cap = (uint32_t)L.K[0];
+  c->log.ring = L.log_ring;
   *out = c;
   return DGS_OK;
 }
@@ -702,74 +769,63 @@ int apply_impl(dgs_ctx* c, uint32_t worker, const dgs_packet* pkt) {
   int slot = -1;
   for (int i = 0; i < kPushSlots; ++i)
     if (pkt->idx == c->at<uint32_t>(c->lay.pkt_idx[i])) slot = i;
-  if (pkt->count > 0) {
-    // The difference vectors of the workers pulled last may still be in use by those pulls.  Each gets
-    // its share of this packet in a launch of its own, on the stream its pull ran on, so that the
-    // main launch (and with it the next pulls) does not have to wait for those pulls to finish.
-    uint32_t skip[kMaxSkip];
-    int skip_stream[kMaxSkip], ns = 0;
-    for (int i = 0; i < kMaxSkip && ns + 1 < (int)N; ++i) {
-      const int w = c->recent_worker[i];
-      if (w < 0) continue;
-      bool dup = false;
-      for (int j = 0; j < ns; ++j) dup = dup || skip[j] == (uint32_t)w;
-      if (dup) continue;
-      skip[ns] = (uint32_t)w;
-      skip_stream[ns] = c->recent_stream[i];
-      ++ns;
+  const uint32_t gx = (pkt->count + kThreads - 1) / kThreads;
+  if (pkt->count == 0) {
+    // nothing to subtract
+  } else if (slot >= 0 && pkt->val == c->at<float>(c->lay.pkt_val[slot]) && pkt->count == c->log.cap) {
+    // One of the library's own packets (sorted by index, of the fixed size): theta now, the D_q lazily.
+    // Its slot of the log still holds the packet filed `ring` applies ago; whoever has not folded that
+    // one in yet does so first.
+    const uint32_t lslot = (uint32_t)(c->log_head % c->log.ring);
+    if (c->log_head >= c->log.ring) {
+      const uint64_t oldest = c->log_head - c->log.ring;
+      for (uint32_t q = 0; q < N; ++q)
+        if (c->applied[q] <= oldest) {
+          const int rc = catch_up_now(c, q);
+          if (rc != DGS_OK) return rc;
+        }
     }
-    uint32_t sorted[kMaxSkip] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
-    for (int i = 0; i < ns; ++i) sorted[i] = skip[i];
-    std::sort(sorted, sorted + kMaxSkip);
-    // (the kernel finds the k-th buffer that is not skipped by bumping past the skipped ones in ascending order)
-    const uint32_t s0 = sorted[0], s1 = sorted[1], s2 = sorted[2];
-    const uint32_t gx = (pkt->count + kThreads - 1) / kThreads;
+    Task t;
+    t.stream = kStApply;
+    t.reads.push_back(R.PKT(slot));
+    t.writes = {R.THETA(), R.LOG(lslot)};
+    int rc = task_begin(c, t);
+    if (rc != DGS_OK) return rc;
     {
-      Task t;
-      t.stream = kStApply;
-      if (slot >= 0) t.reads.push_back(R.PKT(slot));
-      t.writes.push_back(R.THETA());
-      for (uint32_t q = 0; q < N; ++q) {
-        bool skipped = false;
-        for (int j = 0; j < ns; ++j) skipped = skipped || skip[j] == q;
-        if (!skipped) t.writes.push_back(R.D(q));
-      }
-      int rc = slot >= 0 ? DGS_OK : fork_from_user(c, kStApply);
-      if (rc != DGS_OK) return rc;
-      rc = task_begin(c, t);
-      if (rc != DGS_OK) return rc;
-      {
-        TimedLaunch tl(c, c->st[kStApply], DGS_KERNEL_SCATTER);
-        const dim3 grid(gx, N + 1 - ns);
-        k_scatter_sub<<<grid, kThreads, 0, c->st[kStApply]>>>(
-            pkt->idx, pkt->val, pkt->count, c->at<float>(c->lay.theta), c->at<float>(c->lay.D), c->lay.n_pad, N,
-            c->cfg.n, c->ws[0].status, 0u, s0, s1, s2);
-        DGS_CUDA(c, cudaGetLastError());
-        c->launches += 1;
-      }
-      rc = task_end(c, t);
+      TimedLaunch tl(c, c->st[kStApply], DGS_KERNEL_SCATTER);
+      k_apply_log<<<gx, kThreads, 0, c->st[kStApply]>>>(pkt->idx, pkt->val, pkt->count, c->at<float>(c->lay.theta),
+                                                        c->cfg.n, c->ws[0].status, c->log, lslot);
+      DGS_CUDA(c, cudaGetLastError());
+      c->launches += 1;
+    }
+    rc = task_end(c, t);
+    if (rc != DGS_OK) return rc;
+    c->log_head += 1;
+  } else {
+    // Any other packet: bring every D_q up to date, then subtract from theta and all of them at once.
+    for (uint32_t q = 0; q < N; ++q) {
+      const int rc = catch_up_now(c, q);
       if (rc != DGS_OK) return rc;
     }
-    for (int i = 0; i < ns; ++i) {
-      Task t;
-      t.stream = skip_stream[i];
-      if (slot >= 0) t.reads.push_back(R.PKT(slot));
-      t.writes.push_back(R.D(skip[i]));
-      int rc = slot >= 0 ? DGS_OK : fork_from_user(c, t.stream);
-      if (rc != DGS_OK) return rc;
-      rc = task_begin(c, t);
-      if (rc != DGS_OK) return rc;
-      {
-        TimedLaunch tl(c, c->st[t.stream], DGS_KERNEL_SCATTER);
-        k_scatter_sub<<<dim3(gx, 1), kThreads, 0, c->st[t.stream]>>>(
-            pkt->idx, pkt->val, pkt->count, c->at<float>(c->lay.theta), c->at<float>(c->lay.D), c->lay.n_pad, N,
-            c->cfg.n, c->ws[0].status, skip[i], 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
-        DGS_CUDA(c, cudaGetLastError());
-        c->launches += 1;
-      }
-      rc = task_end(c, t);
-      if (rc != DGS_OK) return rc;
+    Task t;
+    t.stream = kStApply;
+    if (slot >= 0) t.reads.push_back(R.PKT(slot));
+    t.writes.push_back(R.THETA());
+    for (uint32_t q = 0; q < N; ++q) t.writes.push_back(R.D(q));
+    int rc = slot >= 0 ? DGS_OK : fork_from_user(c, kStApply);
+    if (rc != DGS_OK) return rc;
+    rc = task_begin(c, t);
+    if (rc != DGS_OK) return rc;
+    {
+      TimedLaunch tl(c, c->st[kStApply], DGS_KERNEL_SCATTER);
+      k_scatter_sub<<<dim3(gx, N + 1), kThreads, 0, c->st[kStApply]>>>(
+          pkt->idx, pkt->val, pkt->count, c->at<float>(c->lay.theta), c->at<float>(c->lay.D), c->lay.n_pad, N,
+          c->cfg.n, c->ws[0].status);
+      DGS_CUDA(c, cudaGetLastError());
+      c->launches += 1;
     }
+    rc = task_end(c, t);
+    if (rc != DGS_OK) return rc;
   }
   c->timestamp += 1;  // t counts updates made to the server parameters
   return DGS_OK;
@@ -794,7 +850,8 @@ int pull_impl(dgs_ctx* c, uint32_t worker, dgs_packet* out) {
   a.lr = c->cfg.lr;
   a.inv_m = c->inv_m;
   Task task;
-  task.writes = {R.D(worker), R.PKT(slot)};
+  task.writes = {R.PKT(slot)};
+  catch_up_deps(c, worker, &task);  // D_worker is brought up to date first, on the same stream
   if (a.theta_local) task.writes.push_back(R.TL(worker));
   // packets that entered D_worker since its previous pull
   const uint64_t age = c->timestamp - (c->prev[worker] < 0 ? 0 : (uint64_t)c->prev[worker]);
@@ -802,12 +859,6 @@ int pull_impl(dgs_ctx* c, uint32_t worker, dgs_packet* out) {
   if (rc != DGS_OK) return rc;
   c->prev[worker] = (int64_t)c->timestamp;
   c->pull_count += 1;
-  for (int i = kMaxSkip - 1; i > 0; --i) {
-    c->recent_worker[i] = c->recent_worker[i - 1];
-    c->recent_stream[i] = c->recent_stream[i - 1];
-  }
-  c->recent_worker[0] = (int)worker;
-  c->recent_stream[0] = stream_id;
   if (out) {
     out->idx = a.pkt_idx;
     out->val = a.pkt_val;
@@ -922,7 +973,11 @@ int dgs_state_ptr(dgs_ctx* c, int which, uint32_t worker, const float** out) {
   if (which != DGS_THETA && worker >= c->cfg.num_workers) return DGS_EINVAL;
   switch (which) {
     case DGS_THETA: *out = c->at<float>(c->lay.theta); break;
-    case DGS_D: *out = c->D_buf(worker); break;
+    case DGS_D:
+      rc = catch_up_now(c, worker);
+      if (rc != DGS_OK) return rc;
+      *out = c->D_buf(worker);
+      break;
     case DGS_THETA_LOCAL:
       if (!(c->cfg.flags & DGS_KEEP_LOCAL_MODEL)) return DGS_EINVAL;
       *out = c->theta_local_buf(worker);

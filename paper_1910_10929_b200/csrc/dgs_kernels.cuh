@@ -742,7 +742,7 @@ __device__ __forceinline__ void cursor_advance(const FinalizeShared& sh, uint32_
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(kThreads, 2) k_finalize(Workspace ws, SelArgs a) {
+__global__ void __maxnreg__(96) k_finalize(Workspace ws, SelArgs a) {
   __shared__ FinalizeShared sh;
 
   constexpr int PM = MODE == kPull ? 1 : 0;
@@ -1213,7 +1213,7 @@ __global__ void __launch_bounds__(kThreads) k_pick_lower(Workspace ws) {
 
 // ---- stand-alone stream pass with the carried bound -------------------------------
 template <int MODE>
-__global__ void __launch_bounds__(kThreads, 2) k_stream(Workspace ws, SelArgs a) {
+__global__ void __maxnreg__(64) k_stream(Workspace ws, SelArgs a) {
   extern __shared__ __align__(128) unsigned char dyn_smem[];   // the ring of stages
   __shared__ StreamShared sh;
   __shared__ __align__(8) uint64_t full[StreamRing<MODE>::kStages];
@@ -1232,16 +1232,154 @@ __global__ void __launch_bounds__(kThreads, 2) k_stream(Workspace ws, SelArgs a)
 }
 
 // ---- server apply ---------------------------------------------------------------
-// buffer q < N is D_q, buffer N is theta.  Indices of one packet are distinct, so every
+// Algorithm 2 lowers theta and every D_q by the decoded packet.  D_q is read only by worker
+// q's pull, so the library keeps D_q lazily: an apply lowers theta at once and files the
+// packet in a ring of recent packets; a pull of worker q first folds into D_q, in arrival
+// order, the packets filed since D_q was last brought up to date.  Every D_q[i] sees the
+// same subtractions in the same order as with an eager update, so the result is the same
+// bit for bit, and each packet is folded into D_q while the entries it touches are hot
+// instead of being scattered into all N vectors at once.
+//
+constexpr int kCatchGrid = 128;                             // CTAs of k_catch_up
+constexpr uint32_t kCatchWarps = kCatchGrid * (kThreads / 32);
+constexpr int kCatchBatch = 2;                              // entries per lane in flight per packet
+
+struct PacketLog {
+  uint32_t* idx;   // [ring][stride], each packet sorted by index
+  float* val;      // [ring][stride]
+  uint32_t stride; // entries between slots
+  uint32_t cap;    // entries per packet
+  uint32_t ring;   // slots
+};
+
+// theta -= packet, and a copy of the packet into slot `slot` of the log.
+__global__ void __launch_bounds__(kThreads) k_apply_log(const uint32_t* __restrict__ idx,
+                                                        const float* __restrict__ val, uint32_t count,
+                                                        float* __restrict__ theta, uint64_t n, int* status,
+                                                        PacketLog lg, uint32_t slot) {
+  const uint32_t j = blockIdx.x * kThreads + threadIdx.x;
+  if (j >= count) return;
+  const uint32_t i = idx[j];
+  const float v = val[j];
+  lg.idx[(uint64_t)slot * lg.stride + j] = i;
+  lg.val[(uint64_t)slot * lg.stride + j] = v;
+  if (i >= n) {
+    atomicMin(status, -2000);
+    return;
+  }
+  theta[i] = __fsub_rn(theta[i], v);
+}
+
+// D -= packets first .. first + count - 1 of the log, in that order (count <= 64).  The index
+// space is cut into kCatchWarps ranges holding equally many entries of the newest packet (the
+// others are spread much alike); a warp owns one range, finds its part of every packet by
+// binary search (packets are sorted), and takes the packets one after the other.  No two
+// warps touch the same entry of D, so no atomics and no block-wide barriers are needed.
+__global__ void __maxnreg__(32) k_catch_up(PacketLog lg, uint64_t first, uint32_t count,
+                                                       float* __restrict__ D, uint64_t n) {
+  const uint32_t lane = threadIdx.x & 31;
+  const uint32_t w = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+  if (w >= kCatchWarps || count == 0) return;
+  const uint32_t* ref = lg.idx + ((first + count - 1) % lg.ring) * (uint64_t)lg.stride;
+  const uint32_t key_lo = w == 0 ? 0u : __ldcg(ref + (uint64_t)w * lg.cap / kCatchWarps);
+  const uint32_t key_hi = w + 1 == kCatchWarps ? 0xFFFFFFFFu : __ldcg(ref + (uint64_t)(w + 1) * lg.cap / kCatchWarps);
+  // positions of [key_lo, key_hi) in packet `lane` and in packet `lane + 32`
+  uint32_t lo_r[2] = {0, 0}, hi_r[2] = {0, 0};
+  {
+    const uint32_t* a[2];
+    uint32_t l0[2], r0[2], l1[2], r1[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const uint32_t p = lane + 32 * h;
+      a[h] = lg.idx + ((first + min(p, count - 1)) % lg.ring) * (uint64_t)lg.stride;
+      l0[h] = l1[h] = 0;
+      r0[h] = r1[h] = p < count ? lg.cap : 0;
+    }
+    for (uint32_t span = lg.cap; span > 0; span >>= 1) {  // enough halvings for a range of cap entries
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        if (l0[h] < r0[h]) {
+          const uint32_t mid = (l0[h] + r0[h]) >> 1;
+          if (__ldcg(a[h] + mid) < key_lo) l0[h] = mid + 1; else r0[h] = mid;
+        }
+        if (l1[h] < r1[h]) {
+          const uint32_t mid = (l1[h] + r1[h]) >> 1;
+          if (__ldcg(a[h] + mid) < key_hi) l1[h] = mid + 1; else r1[h] = mid;
+        }
+      }
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      lo_r[h] = l0[h];
+      hi_r[h] = l1[h];
+    }
+  }
+  uint32_t ci[kCatchBatch], ni[kCatchBatch];
+  float cv[kCatchBatch], nv[kCatchBatch];
+  uint32_t lo = 0, hi = 0, nlo = 0, nhi = 0;
+  const uint32_t* pi = nullptr;
+  const float* pv = nullptr;
+  const uint32_t* npi = nullptr;
+  const float* npv = nullptr;
+  auto fetch = [&](uint32_t p, uint32_t& flo, uint32_t& fhi, const uint32_t*& fpi, const float*& fpv,
+                   uint32_t (&fi)[kCatchBatch], float (&fv)[kCatchBatch]) {
+    const uint32_t a0 = __shfl_sync(0xFFFFFFFFu, lo_r[0], p & 31), a1 = __shfl_sync(0xFFFFFFFFu, lo_r[1], p & 31);
+    const uint32_t b0 = __shfl_sync(0xFFFFFFFFu, hi_r[0], p & 31), b1 = __shfl_sync(0xFFFFFFFFu, hi_r[1], p & 31);
+    flo = p < 32 ? a0 : a1;
+    fhi = p < 32 ? b0 : b1;
+    const uint64_t at = ((first + p) % lg.ring) * (uint64_t)lg.stride;
+    fpi = lg.idx + at;
+    fpv = lg.val + at;
+#pragma unroll
+    for (int e = 0; e < kCatchBatch; ++e) {
+      const uint32_t j = flo + lane + 32 * e;
+      const bool in = j < fhi;
+      fi[e] = in ? __ldcg(fpi + j) : 0xFFFFFFFFu;
+      fv[e] = in ? __ldcg(fpv + j) : 0.0f;
+    }
+  };
+  fetch(0, lo, hi, pi, pv, ci, cv);
+  for (uint32_t p = 0; p < count; ++p) {
+    if (p + 1 < count) fetch(p + 1, nlo, nhi, npi, npv, ni, nv);
+    for (uint32_t base = lo;;) {
+      float d[kCatchBatch];
+#pragma unroll
+      for (int e = 0; e < kCatchBatch; ++e)
+        if (ci[e] < n) d[e] = __ldcg(D + ci[e]);
+#pragma unroll
+      for (int e = 0; e < kCatchBatch; ++e)
+        if (ci[e] < n) __stcg(D + ci[e], __fsub_rn(d[e], cv[e]));
+      base += 32 * kCatchBatch;
+      if (base >= hi) break;
+#pragma unroll
+      for (int e = 0; e < kCatchBatch; ++e) {  // a range with more entries than one batch
+        const uint32_t j = base + lane + 32 * e;
+        const bool in = j < hi;
+        ci[e] = in ? __ldcg(pi + j) : 0xFFFFFFFFu;
+        cv[e] = in ? __ldcg(pv + j) : 0.0f;
+      }
+    }
+    __syncwarp();  // orders this packet's stores before the next packet's loads within the warp
+    lo = nlo;
+    hi = nhi;
+    pi = npi;
+    pv = npv;
+#pragma unroll
+    for (int e = 0; e < kCatchBatch; ++e) {
+      ci[e] = ni[e];
+      cv[e] = nv[e];
+    }
+  }
+}
+
+// Eager form, for a packet that is not one of the library's own (any order of indices, any
+// count): buffer q < N is D_q, buffer N is theta.  Indices of one packet are distinct, so every
 // (buffer, entry) pair is touched by exactly one thread: plain load / subtract / store.
-// One launch covers gridDim.y buffers counted from q_first, leaving out up to three (a
-// difference vector that a pull is still working on gets its share in a launch of its own).
 __global__ void __launch_bounds__(kThreads) k_scatter_sub(const uint32_t* __restrict__ idx,
                                                           const float* __restrict__ val, uint32_t count,
                                                           float* __restrict__ theta, float* __restrict__ D,
                                                           uint64_t d_stride, uint32_t num_workers, uint64_t n,
-                                                          int* status, uint32_t q_first, uint32_t skip0,
-                                                          uint32_t skip1, uint32_t skip2) {
+                                                          int* status) {
   const uint32_t j = blockIdx.x * kThreads + threadIdx.x;
   if (j >= count) return;
   const uint32_t i = idx[j];
@@ -1250,10 +1388,7 @@ __global__ void __launch_bounds__(kThreads) k_scatter_sub(const uint32_t* __rest
     atomicMin(status, -2000);
     return;
   }
-  uint32_t q = q_first + blockIdx.y;   // the blockIdx.y-th buffer that is not skipped (skip0 <= skip1 <= skip2)
-  if (q >= skip0) ++q;
-  if (q >= skip1) ++q;
-  if (q >= skip2) ++q;
+  const uint32_t q = blockIdx.y;
   float* p = (q == num_workers ? theta : D + (uint64_t)q * d_stride) + i;
   *p = __fsub_rn(*p, v);
 }

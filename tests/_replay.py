@@ -86,7 +86,7 @@ def compare_state(ctx, orc, num_workers: int, keep_local: bool) -> None:
             same(dgs.DGS_THETA_LOCAL, oracle.THETA_LOCAL, q, "theta_local")
 
 
-def replay_async_and_compare(wl, *, flags: int = 0, num_events=None, device: str = "cuda:0"):
+def replay_async_and_compare(wl, *, flags: int = 0, num_events=None, schedule=None, device: str = "cuda:0"):
     """Enqueues all events back to back without ever waiting (the library's streams overlap
     consecutive events), then replays the same events on the CPU checker and compares the
     whole final state and the last packets bit for bit.  Any missing dependency between the
@@ -94,7 +94,7 @@ def replay_async_and_compare(wl, *, flags: int = 0, num_events=None, device: str
     keep_local = bool(flags & dgs.DGS_KEEP_LOCAL_MODEL)
     residual = bool(flags & dgs.DGS_RESIDUAL_MODE)
     theta0 = wl.theta0()
-    sched = wl.schedule()
+    sched = wl.schedule() if schedule is None else np.asarray(schedule)
     E = len(sched) if num_events is None else num_events
     sched = np.resize(sched, E)
     grads_host = [wl.gradient(e) for e in range(E)]

@@ -134,6 +134,20 @@ def test_overlapped_events_resnet18_per_layer():
     replay_async_and_compare(wl)
 
 
+def test_starved_worker_sees_every_packet_it_missed():
+    # worker 2 arrives once, stays away for 50 events (more than the library keeps packets for), comes back
+    wl = W.custom("starved", [40_000, 700, 9_001], 3, 60, 10_000, grad_kind="laplace")
+    sched = [2] + [0, 1] * 25 + [2, 0, 2, 1, 2, 2, 0, 1, 2]
+    replay_and_compare(wl, schedule=sched, compare_state_every=20)
+    replay_async_and_compare(wl, schedule=sched, flags=dgs.DGS_KEEP_LOCAL_MODEL)
+
+
+def test_more_workers_than_packets_kept():
+    # 70 workers in a fixed cycle: every difference vector is 70 packets behind when its worker returns
+    wl = W.custom("many", [30_000, 301, 2_048], 70, 180, 10_000, grad_kind="normal", schedule_kind="cyclic")
+    replay_async_and_compare(wl)
+
+
 def test_trajectory_gpt2_small_few_workers():
     wl = W.gpt2_small(num_workers=3, num_events=7)
     replay_and_compare(wl)
