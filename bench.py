@@ -29,6 +29,9 @@ from concurrent.futures import ThreadPoolExecutor
 
 import numpy as np
 
+# hardware queues for the library's streams (read when the CUDA context is created; see the package)
+os.environ.setdefault("CUDA_DEVICE_MAX_CONNECTIONS", "32")
+
 ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
@@ -261,6 +264,7 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
         run_events(preroll, Wm)
         ctx.flush()
         stats0 = ctx.stats()
+        reads0 = ctx.pull_read_stats()
         launches0 = ctx.launch_count()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
@@ -275,6 +279,7 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
     elapsed = ev0.elapsed_time(ev1) * 1e-3
     launches = ctx.launch_count() - launches0
     stats1 = ctx.stats()
+    reads1 = ctx.pull_read_stats()
     assert ctx.status() == 0, "device status word is not clean"
     elapsed_max, events_all = reduce_max_time(elapsed, K, dist)
 
@@ -337,12 +342,14 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
                    "segments": wl.num_segments, "lr": wl.lr, "momentum": wl.momentum, "seed": wl.seed,
                    "preroll_events": preroll, "distinct_gradients": pool,
                    "l2": "inputs larger than L2: every event reads a different gradient, velocity and "
-                         "difference vector", "replicas": world},
+                         "difference vector", "replicas": world,
+                   "cuda_device_max_connections": os.environ.get("CUDA_DEVICE_MAX_CONNECTIONS")},
         "effective_hbm": {"algorithmic_bytes_per_event": ab, "GB/s": eff_gbs,
                           "frac_of_nominal_8TBs": eff_gbs / NOMINAL_HBM_GBS, "frac_of_peak": eff_gbs / peak,
                           "peak_GB/s": peak, "peak_kind": peak_kind},
         "selection_routes": {"single_pass": stats1[0] - stats0[0], "two_pass": stats1[1] - stats0[1],
-                             "candidates_per_selection": (stats1[3] - stats0[3]) / max(1, 2 * K)},
+                             "candidates_per_selection": (stats1[3] - stats0[3]) / max(1, 2 * K),
+                             "pull_chunks_read_fraction": (reads1[1] - reads0[1]) / max(1, reads1[0] - reads0[0])},
         "kernels": {k: {"ms_total": ms, "launches": c, "us_per_launch": (1e3 * ms / c if c else None),
                         "share": ms / tot_ms,
                         "GB/s": kernel_gbs(k, ms, c)}

@@ -168,6 +168,14 @@ int dgs_status(dgs_ctx* ctx, int* device_status);
  * steps have examined in total (the k selected ones included). */
 int dgs_stats(dgs_ctx* ctx, uint64_t out[4]);
 
+/* Waits for all work in flight and reports how much of the difference vectors the pulls'
+ * stream passes had to read: out[0] stage-sized chunks (4096 elements) of whole tiles that
+ * the passes covered, out[1] those of them that were actually read.  The library keeps,
+ * per 512 elements of every D_q, an upper bound on the magnitudes in it; a chunk whose
+ * bounds are all below the selection's lower bound cannot hold a selected entry (Eq. 6a
+ * takes the largest magnitudes) and is not read.  The selection stays exact. */
+int dgs_pull_read_stats(dgs_ctx* ctx, uint64_t out[2]);
+
 /* prev(worker): the server timestamp at that worker's last pull, -1 before it. */
 int dgs_prev(dgs_ctx* ctx, uint32_t worker, int64_t* out);
 

@@ -12,6 +12,12 @@ import ctypes as C
 import os
 from typing import Optional, Sequence, Tuple
 
+# The library spreads its kernels over eleven CUDA streams.  The driver maps streams onto a fixed
+# number of hardware queues (8 unless told otherwise) and streams that share a queue run one after
+# the other; the variable is read when the process creates its CUDA context, so it has to be in
+# place before that.  A value the user has set is left alone.
+os.environ.setdefault("CUDA_DEVICE_MAX_CONNECTIONS", "32")
+
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libdgs.so")
 
@@ -21,7 +27,7 @@ DGS_THETA, DGS_U, DGS_D, DGS_THETA_LOCAL = 0, 1, 2, 3
 
 EXPORTS = (
     "dgs_arena_bytes", "dgs_init", "dgs_worker_push", "dgs_server_apply", "dgs_worker_pull",
-    "dgs_event", "dgs_flush", "dgs_event_host", "dgs_state_ptr", "dgs_state_load", "dgs_status", "dgs_stats",
+    "dgs_event", "dgs_flush", "dgs_event_host", "dgs_state_ptr", "dgs_state_load", "dgs_status", "dgs_stats", "dgs_pull_read_stats",
     "dgs_prev", "dgs_launch_count", "dgs_last_cuda_error", "dgs_free", "dgs_error_string",
     "dgs_timing_enable", "dgs_timing_read", "dgs_topk_encode_static",
 )
@@ -76,6 +82,7 @@ def lib() -> C.CDLL:
         L.dgs_state_load.argtypes = [vp, i32, u32, vp]
         L.dgs_status.argtypes = [vp, C.POINTER(i32)]
         L.dgs_stats.argtypes = [vp, C.POINTER(C.c_uint64)]
+        L.dgs_pull_read_stats.argtypes = [vp, C.POINTER(C.c_uint64)]
         L.dgs_prev.argtypes = [vp, u32, C.POINTER(C.c_int64)]
         L.dgs_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
         L.dgs_last_cuda_error.argtypes = [vp]
@@ -174,6 +181,13 @@ def dgs_stats(ctx: int) -> Tuple[int, int, int, int]:
     out = (C.c_uint64 * 4)()
     _check(lib().dgs_stats(ctx, out), "dgs_stats")
     return tuple(int(v) for v in out)
+
+
+def dgs_pull_read_stats(ctx: int) -> Tuple[int, int]:
+    """(chunks of D covered by the pulls' stream passes, chunks actually read)."""
+    out = (C.c_uint64 * 2)()
+    _check(lib().dgs_pull_read_stats(ctx, out), "dgs_pull_read_stats")
+    return int(out[0]), int(out[1])
 
 
 def dgs_prev(ctx: int, worker: int) -> int:

@@ -97,6 +97,9 @@ class Context:
     def stats(self):
         return dgs.dgs_stats(self.handle)
 
+    def pull_read_stats(self):
+        return dgs.dgs_pull_read_stats(self.handle)
+
     def launch_count(self) -> int:
         return dgs.dgs_launch_count(self.handle)
 

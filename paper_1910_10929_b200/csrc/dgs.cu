@@ -31,8 +31,8 @@ namespace {
 constexpr uint64_t kAlign = 256;
 constexpr uint32_t kMagic = 0x44475331u;  // "DGS1"
 constexpr int kPushSlots = 5;             // push packet slots, used in turn
-constexpr int kPullSlots = 4;             // pull packet slots
-constexpr int kWorkerStreams = 4, kServerStreams = 4;
+constexpr int kPullSlots = 6;             // pull packet slots
+constexpr int kWorkerStreams = 4, kServerStreams = 6;
 constexpr int kPushSets = kWorkerStreams;  // scratch sets and spare velocity buffers of the pushes
 constexpr int kPullSets = kServerStreams;  // scratch sets of the pulls
 constexpr int kAllSets = kPushSets + kPullSets;
@@ -59,7 +59,9 @@ struct Layout {
   uint64_t tiles, segs, seg_off, seg_tile0;
   ScratchLayout sc[kAllSets];  // push sets, then pull sets
   uint64_t L_next, u_slots, status, stats;
-  uint64_t log_idx, log_val;  // ring of applied packets not yet folded into every D_q
+  uint64_t log_idx, log_val;
+  uint64_t blk_max;      // [N][blk_stride]: per block of kWarpTile elements, an upper bound on the keys of D_q in it
+  uint64_t blk_stride = 0;  // ring of applied packets not yet folded into every D_q
   uint32_t log_ring = 0, log_stride = 0;
   uint64_t total = 0;
 };
@@ -176,6 +178,8 @@ void make_layout(const dgs_config* c, Layout* L) {
   L->log_stride = (uint32_t)align_up(L->K[0], 64);
   L->log_idx = take((uint64_t)L->log_ring * L->log_stride * 4);
   L->log_val = take((uint64_t)L->log_ring * L->log_stride * 4);
+  L->blk_stride = align_up((c->n + kWarpTile - 1) / kWarpTile, 64);
+  L->blk_max = take(N * L->blk_stride * 4);
   L->L_next = take(2 * N * S * 4);
   L->u_slots = take((N + kPushSets) * sizeof(float*));
   L->status = take(4);
@@ -252,6 +256,7 @@ struct dgs_ctx {
   float* u_buf(uint32_t q) const { return at<float>(lay.u) + (uint64_t)q * lay.n_pad; }
   float* D_buf(uint32_t q) const { return at<float>(lay.D) + (uint64_t)q * lay.n_pad; }
   float* theta_local_buf(uint32_t q) const { return at<float>(lay.theta_local) + (uint64_t)q * lay.n_pad; }
+  uint32_t* blk_max(uint32_t q) const { return at<uint32_t>(lay.blk_max) + (uint64_t)q * lay.blk_stride; }
   float** u_slot(uint32_t q) const { return at<float*>(lay.u_slots) + q; }
   uint32_t* L_next(int pm, uint32_t w) const {
     return at<uint32_t>(lay.L_next) + ((uint64_t)pm * cfg.num_workers + w) * cfg.num_segments;
@@ -394,7 +399,7 @@ int catch_up_launch(dgs_ctx* c, uint32_t q, cudaStream_t st) {
   const uint32_t count = (uint32_t)(c->log_head - first);
   if (count > 0) {
     TimedLaunch tl(c, st, DGS_KERNEL_CATCH_UP);
-    k_catch_up<<<kCatchGrid, kThreads, 0, st>>>(c->log, first, count, c->D_buf(q), c->cfg.n);
+    k_catch_up<<<kCatchGrid, kThreads, 0, st>>>(c->log, first, count, c->D_buf(q), c->blk_max(q), c->cfg.n);
     DGS_CUDA(c, cudaGetLastError());
     c->launches += 1;
   }
@@ -425,7 +430,7 @@ int pick_row(const dgs_ctx* c, int kind, uint64_t age) {
   for (uint32_t q = 0; q < c->cfg.num_workers; ++q) {
     if (!c->row_valid[kind][q] || c->row_age[kind][q] > age) continue;
     const uint64_t t = c->row_time[kind][q];
-    if (best < 0 || t > c->row_time[kind][best]) best = (int)q;
+    if (best < 0 || t < c->row_time[kind][best]) best = (int)q;   // else the oldest: the likeliest to be complete
     if (t + in_flight <= newest && (best_old < 0 || t > c->row_time[kind][best_old])) best_old = (int)q;
   }
   return best_old >= 0 ? best_old : best;
@@ -631,8 +636,13 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   if (occupancy_grids<kPushSam>(c, sms) != DGS_OK || occupancy_grids<kPushResidual>(c, sms) != DGS_OK ||
       occupancy_grids<kPull>(c, sms) != DGS_OK)
     return fail(DGS_ECUDA);
+  int prio_low = 0, prio_high = 0;
+  INIT_CUDA(cudaDeviceGetStreamPriorityRange(&prio_low, &prio_high));
   for (int i = 0; i < kNumStreams; ++i) {
-    INIT_CUDA(cudaStreamCreateWithFlags(&c->st[i], cudaStreamNonBlocking));
+    // The push passes move most of the bytes and fill every SM; the short kernels of the server side sit on
+    // the longer chain (apply -> catch-up -> pull), so their blocks go first whenever an SM has room.
+    const int prio = i < kStApply ? prio_low : prio_high;
+    INIT_CUDA(cudaStreamCreateWithPriority(&c->st[i], cudaStreamNonBlocking, prio));
     INIT_CUDA(cudaEventCreateWithFlags(&c->ev_tail[i], cudaEventDisableTiming));
   }
   INIT_CUDA(cudaEventCreateWithFlags(&c->ev_in, cudaEventDisableTiming));
@@ -668,6 +678,7 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
     INIT_CUDA(cudaMemsetAsync(c->at<char>(sc.part_cands), 0, (uint64_t)kMaxGrid * 4, st));
     INIT_CUDA(cudaMemsetAsync(c->at<char>(sc.part_slot0), 0, (uint64_t)kMaxGrid * 4, st));
   }
+  INIT_CUDA(cudaMemsetAsync(c->at<char>(L.blk_max), 0, N * L.blk_stride * 4, st));   // D = 0
   INIT_CUDA(cudaMemsetAsync(c->at<char>(L.L_next), 0xFF, 2 * N * cfg->num_segments * 4, st));
   INIT_CUDA(cudaMemsetAsync(c->at<char>(L.status), 0, L.total - L.status, st));
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.tiles), tiles.data(), tiles.size() * sizeof(Tile), cudaMemcpyHostToDevice, st));
@@ -820,7 +831,7 @@ int apply_impl(dgs_ctx* c, uint32_t worker, const dgs_packet* pkt) {
       TimedLaunch tl(c, c->st[kStApply], DGS_KERNEL_SCATTER);
       k_scatter_sub<<<dim3(gx, N + 1), kThreads, 0, c->st[kStApply]>>>(
           pkt->idx, pkt->val, pkt->count, c->at<float>(c->lay.theta), c->at<float>(c->lay.D), c->lay.n_pad, N,
-          c->cfg.n, c->ws[0].status);
+          c->cfg.n, c->ws[0].status, c->blk_max(0), c->lay.blk_stride);
       DGS_CUDA(c, cudaGetLastError());
       c->launches += 1;
     }
@@ -842,6 +853,7 @@ int pull_impl(dgs_ctx* c, uint32_t worker, dgs_packet* out) {
   SelArgs a;
   std::memset(&a, 0, sizeof(a));
   a.D = c->D_buf(worker);
+  a.blk_max = c->blk_max(worker);
   a.theta_local = (c->cfg.flags & DGS_KEEP_LOCAL_MODEL) ? c->theta_local_buf(worker) : nullptr;
   a.pkt_idx = c->at<uint32_t>(L.pkt_idx[slot]);
   a.pkt_val = c->at<float>(L.pkt_val[slot]);
@@ -1016,6 +1028,8 @@ int dgs_state_load(dgs_ctx* c, int which, uint32_t worker, const float* src) {
   rc = task_begin(c, t);
   if (rc != DGS_OK) return rc;
   DGS_CUDA(c, cudaMemcpyAsync(const_cast<float*>(dst), src, c->cfg.n * 4, cudaMemcpyDeviceToDevice, c->st[t.stream]));
+  if (which == DGS_D)   // nothing is known about the new contents: every block may hold anything
+    DGS_CUDA(c, cudaMemsetAsync(c->blk_max(worker), 0xFF, c->lay.blk_stride * 4, c->st[t.stream]));
   return task_end(c, t);
 }
 
@@ -1041,6 +1055,19 @@ int dgs_stats(dgs_ctx* c, uint64_t out[4]) {
   out[1] = s[1];
   out[2] = c->timestamp;
   out[3] = s[2];
+  return DGS_OK;
+}
+
+int dgs_pull_read_stats(dgs_ctx* c, uint64_t out[2]) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (!out) return DGS_EINVAL;
+  unsigned long long s[2] = {0, 0};
+  rc = sync_all(c);
+  if (rc != DGS_OK) return rc;
+  DGS_CUDA(c, cudaMemcpy(s, c->ws[0].stats + 3, sizeof(s), cudaMemcpyDeviceToHost));
+  out[0] = s[0];
+  out[1] = s[1];
   return DGS_OK;
 }
 

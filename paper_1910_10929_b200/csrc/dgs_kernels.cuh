@@ -98,6 +98,7 @@ struct SelArgs {
   float** u_spare_slot;   // push: device slot holding the spare buffer pointer
   float* D;               // pull: D_w
   float* theta_local;     // pull: theta_w or null
+  uint32_t* blk_max;      // pull: per block of kWarpTile elements, an upper bound on the keys of D_w in it (or null)
   const uint32_t* L_in;   // [S] lower bounds guessed for this selection (single-pass route)
   uint32_t* L_next;       // [S] receives the bounds this selection suggests for a later, similar one
   uint32_t* pkt_idx;
@@ -169,9 +170,11 @@ __device__ __forceinline__ void load_tile_vec(const float* __restrict__ a, const
 }
 
 // ---- stream pass ----------------------------------------------------------------
+constexpr int kLiveWords = 128;     // one bit per stage-sized chunk of a CTA's share of a layer
 struct StreamShared {
   uint32_t hist[kBins1];  // top 11 key bits of the candidates of the layer being processed
   uint32_t cursor;        // candidates appended by this CTA so far
+  uint32_t live[kLiveWords];  // pull: chunks that may hold a candidate (the others are not read)
 };
 
 __device__ __forceinline__ void flush_hist(uint32_t* s_hist, uint32_t* g_hist) {
@@ -343,9 +346,11 @@ __device__ __forceinline__ void finish_full_tile_smem(const Workspace& ws, const
   const float4* pu = reinterpret_cast<const float4*>(su) + lane;
   const float4* pg = reinterpret_cast<const float4*>(sg) + lane;
   uint32_t mask = 0;
+  uint32_t top = 0;       // pull: largest key of this lane's elements
 #pragma unroll
   for (int j = 0; j < kVecIters; ++j) {
     float4 x = pu[j * 32];
+    if (MODE == kPull) top = max(max(top, max(key_of(x.x), key_of(x.y))), max(key_of(x.z), key_of(x.w)));
     if (MODE != kPull) {
       const float4 g = pg[j * 32];
       x.x = combine<MODE>(x.x, g.x, a.m, a.lr);
@@ -363,6 +368,11 @@ __device__ __forceinline__ void finish_full_tile_smem(const Workspace& ws, const
       o.w = c3 ? x.w : unsent<MODE>(x.w, a.inv_m);
       __stcs(reinterpret_cast<float4*>(out + tile_start) + lane + j * 32, o);
     }
+  }
+  if (MODE == kPull && a.blk_max != nullptr) {
+    // the tile is a whole block: its bound becomes exact again (entries sent later only lower it)
+    top = __reduce_max_sync(kFull, top);
+    if (lane == 0) a.blk_max[tile_start / kWarpTile] = top;
   }
   if (!__any_sync(kFull, mask != 0)) return;
   // per-j candidate counts of this lane, one per byte
@@ -408,7 +418,7 @@ constexpr int kStageTiles = kWarps;                        // one tile per warp 
 constexpr int kStageFloats = kStageTiles * kWarpTile;      // per input array
 template <int MODE> struct StreamRing {
   static constexpr int kInputs = MODE == kPull ? 1 : 2;
-  static constexpr int kStages = MODE == kPull ? 5 : 3;
+  static constexpr int kStages = MODE == kPull ? 3 : 2;
   static constexpr int kStageBytes = kInputs * kStageFloats * 4;
   static constexpr int kBytes = kStages * kStageBytes;     // 80 KB (pull) / 96 KB (push)
 };
@@ -490,10 +500,51 @@ __device__ void stream_tiles_tma(const Workspace& ws, const SelArgs& a, const ui
       bulk_load(dst, in + elem, bytes, full + st);
       if (MODE != kPull) bulk_load(dst + kStageFloats, a.grad + elem, bytes, full + st);
     };
-    if (threadIdx.x == 0)
-      for (uint32_t c = 0; c < min(nchunks, (uint32_t)R::kStages); ++c) issue(c, uses + c);
-    for (uint32_t c = 0; c < nchunks; ++c) {
-      const uint32_t use = uses + c, st = use % R::kStages;
+    // Pull: a chunk all of whose blocks have a bound below L holds no candidate and is not read.
+    const bool can_skip = MODE == kPull && a.blk_max != nullptr && L > 0 && nchunks <= kLiveWords * 32;
+    if (can_skip) {
+      for (uint32_t base = warp * 32; base < nchunks; base += kWarps * 32) {
+        const uint32_t c = base + lane;
+        bool live = false;
+        if (c < nchunks) {
+          const uint32_t tiles_here = min((uint32_t)kStageTiles, nfull - c * kStageTiles);
+          const uint32_t* bm = a.blk_max + e0 / kWarpTile + c * kStageTiles;
+          uint32_t top = 0;
+          for (uint32_t j = 0; j < tiles_here; ++j) top = max(top, __ldcg(bm + j));
+          live = top >= L;
+        }
+        const uint32_t word = __ballot_sync(kFull, live);
+        if (lane == 0) sh.live[base / 32] = word;
+      }
+      __syncthreads();
+    }
+    auto next_live = [&](uint32_t c) -> uint32_t {       // first chunk >= c that is read, nchunks if none
+      if constexpr (MODE == kPull) {
+        while (can_skip && c < nchunks) {
+          const uint32_t w = sh.live[c >> 5] >> (c & 31);
+          if (w) return c + __ffs(w) - 1;
+          c = (c | 31u) + 1;
+        }
+      }
+      return min(c, nchunks);
+    };
+    if (MODE == kPull && threadIdx.x == 0 && nchunks) {     // bookkeeping: chunks of D_w that exist / that are read
+      uint32_t read = nchunks;
+      if (can_skip) {
+        read = 0;
+        for (uint32_t w = 0; w * 32 < nchunks; ++w) read += __popc(sh.live[w]);
+      }
+      atomicAdd(ws.stats + 3, (unsigned long long)nchunks);
+      atomicAdd(ws.stats + 4, (unsigned long long)read);
+    }
+    uint32_t pc = 0, issued = 0;                          // thread 0: next chunk to ask for, chunks asked for
+    if (threadIdx.x == 0) {
+      pc = next_live(0);
+      for (; issued < (uint32_t)R::kStages && pc < nchunks; ++issued, pc = next_live(pc + 1)) issue(pc, uses + issued);
+    }
+    uint32_t done = 0;
+    for (uint32_t c = next_live(0); c < nchunks; c = next_live(c + 1), ++done) {
+      const uint32_t use = uses + done, st = use % R::kStages;
       if (!mbar_wait(full + st, (use / R::kStages) & 1u)) *s_dead = 1;
       const uint32_t tl = c * kStageTiles + warp;          // this warp's tile among the full ones
       if (tl < nfull && !*s_dead) {
@@ -502,10 +553,14 @@ __device__ void stream_tiles_tma(const Workspace& ws, const SelArgs& a, const ui
       }
       __syncthreads();                                     // every warp is done reading this stage
       if (*s_dead) break;
-      if (threadIdx.x == 0 && c + R::kStages < nchunks) issue(c + R::kStages, use + R::kStages);
+      if (threadIdx.x == 0 && pc < nchunks) {
+        issue(pc, uses + issued);
+        ++issued;
+        pc = next_live(pc + 1);
+      }
     }
     if (*s_dead) break;
-    uses += nchunks;
+    uses += done;
     __syncthreads();
     flush_hist(sh.hist, ws.hist1 + (size_t)s * kBins1);
     __syncthreads();
@@ -1275,8 +1330,9 @@ __global__ void __launch_bounds__(kThreads) k_apply_log(const uint32_t* __restri
 // others are spread much alike); a warp owns one range, finds its part of every packet by
 // binary search (packets are sorted), and takes the packets one after the other.  No two
 // warps touch the same entry of D, so no atomics and no block-wide barriers are needed.
-__global__ void __maxnreg__(32) k_catch_up(PacketLog lg, uint64_t first, uint32_t count,
-                                                       float* __restrict__ D, uint64_t n) {
+__global__ void __launch_bounds__(kThreads) k_catch_up(PacketLog lg, uint64_t first, uint32_t count,
+                                                       float* __restrict__ D, uint32_t* __restrict__ blk_max,
+                                                       uint64_t n) {
   const uint32_t lane = threadIdx.x & 31;
   const uint32_t w = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
   if (w >= kCatchWarps || count == 0) return;
@@ -1348,7 +1404,11 @@ __global__ void __maxnreg__(32) k_catch_up(PacketLog lg, uint64_t first, uint32_
         if (ci[e] < n) d[e] = __ldcg(D + ci[e]);
 #pragma unroll
       for (int e = 0; e < kCatchBatch; ++e)
-        if (ci[e] < n) __stcg(D + ci[e], __fsub_rn(d[e], cv[e]));
+        if (ci[e] < n) {
+          const float r = __fsub_rn(d[e], cv[e]);
+          __stcg(D + ci[e], r);
+          atomicMax(blk_max + ci[e] / kWarpTile, key_of(r));   // keeps the block's bound an upper bound
+        }
       base += 32 * kCatchBatch;
       if (base >= hi) break;
 #pragma unroll
@@ -1379,7 +1439,8 @@ __global__ void __launch_bounds__(kThreads) k_scatter_sub(const uint32_t* __rest
                                                           const float* __restrict__ val, uint32_t count,
                                                           float* __restrict__ theta, float* __restrict__ D,
                                                           uint64_t d_stride, uint32_t num_workers, uint64_t n,
-                                                          int* status) {
+                                                          int* status, uint32_t* __restrict__ blk_max,
+                                                          uint64_t blk_stride) {
   const uint32_t j = blockIdx.x * kThreads + threadIdx.x;
   if (j >= count) return;
   const uint32_t i = idx[j];
@@ -1390,7 +1451,9 @@ __global__ void __launch_bounds__(kThreads) k_scatter_sub(const uint32_t* __rest
   }
   const uint32_t q = blockIdx.y;
   float* p = (q == num_workers ? theta : D + (uint64_t)q * d_stride) + i;
-  *p = __fsub_rn(*p, v);
+  const float r = __fsub_rn(*p, v);
+  *p = r;
+  if (q < num_workers) atomicMax(blk_max + (uint64_t)q * blk_stride + i / kWarpTile, key_of(r));
 }
 
 }  // namespace dgs
