@@ -142,6 +142,31 @@ def test_starved_worker_sees_every_packet_it_missed():
     replay_async_and_compare(wl, schedule=sched, flags=dgs.DGS_KEEP_LOCAL_MODEL)
 
 
+def test_pull_skips_cold_chunks_and_notices_when_they_heat_up():
+    # gradients live in one third of the vector at a time and move on with growing size, so chunks of the
+    # difference vectors that the pulls had stopped reading come back into the selection
+    n, third = 3 * 262_144, 262_144
+    wl = W.custom("moving_heat", [n], 3, 36, 2_000, grad_kind="normal", grad_scale=1e-3)
+    base = wl.gradient
+
+    def moving(e, out=None):
+        g = base(e)
+        phase = (e // 9) % 3
+        keep = np.zeros(n, dtype=np.float32)
+        keep[phase * third:(phase + 1) * third] = np.float32(1 + e // 9)
+        g *= keep
+        if out is not None:
+            out[:] = g
+            return out
+        return g
+
+    wl.gradient = moving
+    ctx, _ = replay_and_compare(wl, compare_state_every=9)
+    covered, read = ctx.pull_read_stats()
+    assert 0 < read < covered            # some chunks were skipped, and the packets still agreed throughout
+    replay_async_and_compare(wl, flags=dgs.DGS_KEEP_LOCAL_MODEL)
+
+
 def test_more_workers_than_packets_kept():
     # 70 workers in a fixed cycle: every difference vector is 70 packets behind when its worker returns
     wl = W.custom("many", [30_000, 301, 2_048], 70, 180, 10_000, grad_kind="normal", schedule_kind="cyclic")
