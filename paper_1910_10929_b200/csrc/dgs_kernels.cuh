@@ -934,7 +934,12 @@ __global__ void __maxnreg__(96) k_finalize(Workspace ws, SelArgs a) {
             lbin = used > 4 ? used - 4 : 0;
           }
           __syncthreads();
-          if (threadIdx.x == 0) a.L_next[s] = lbin << 20;
+          // A bound of zero makes every element of the layer a candidate (zeros included).  That is fine for a
+          // layer not much larger than the wished-for number of candidates; for a large one, no bound at all is
+          // the better advice: the next selection finds nothing, notices, and takes its bound from a histogram.
+          const uint32_t layer_cap = (ws.segs[s].tile_end - ws.segs[s].tile_begin) * (uint32_t)kWarpTile;
+          const bool flood = lbin == 0 && layer_cap / 8 > want;
+          if (threadIdx.x == 0) a.L_next[s] = flood ? 0xFFFFFFFFu : lbin << 20;
         }
       }
       __syncthreads();
