@@ -83,7 +83,9 @@ enum {
   DGS_RESIDUAL_MODE = 1u << 1,    /* worker rule of Algorithm 1 instead of Algorithm 3: v <- v + eta*grad,
                                      sent entries leave v, the rest stay (no momentum, no 1/m rescale) */
   DGS_HOST_IO = 1u << 2,          /* reserve staging buffers for dgs_event_host */
-  DGS_NO_SPECULATION = 1u << 3    /* always take the two-pass selection (histogram pass, then stream pass) */
+  DGS_NO_SPECULATION = 1u << 3,   /* always take the two-pass selection (histogram pass, then stream pass) */
+  DGS_SINGLE_STREAM = 1u << 4     /* enqueue every step on ONE internal stream: kernels run one after the other in
+                                     call order (same results; for debugging and for timing a kernel on its own) */
 };
 
 typedef struct {
@@ -204,6 +206,16 @@ int dgs_timing_enable(dgs_ctx* ctx, int on);
  * milliseconds and the number of recorded launches of kernel i since the last
  * read, and the accumulators restart from zero. */
 int dgs_timing_read(dgs_ctx* ctx, double ms[DGS_NUM_KERNELS], uint64_t count[DGS_NUM_KERNELS]);
+
+/* Measurement aid (no counterpart in the paper): the launches recorded since the last read as
+ * a timeline instead of sums.  Waits for all work in flight.  For the first min(cap, recorded)
+ * launches, in the order they were enqueued: start_ms / stop_ms (HOST f32[cap]) receive the
+ * device times of the two events around the launch, in milliseconds after the first recorded
+ * launch began; kernel[i] one of DGS_KERNEL_*; stream[i] the index of the library stream it
+ * ran on.  *count receives how many entries were written.  The record restarts empty (the sums
+ * of dgs_timing_read do not include these launches). */
+int dgs_timing_trace(dgs_ctx* ctx, uint32_t cap, float* start_ms, float* stop_ms, int32_t* kernel, int32_t* stream,
+                     uint32_t* count);
 
 /* The cudaError_t of the last failed runtime call of this context (0 if none). */
 int dgs_last_cuda_error(dgs_ctx* ctx);

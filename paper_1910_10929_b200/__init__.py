@@ -22,14 +22,14 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libdgs.so")
 
 DGS_OK, DGS_EINVAL, DGS_ENOMEM, DGS_ECUDA, DGS_ETIMEOUT, DGS_ESTATE = 0, -1, -2, -3, -4, -5
-DGS_KEEP_LOCAL_MODEL, DGS_RESIDUAL_MODE, DGS_HOST_IO, DGS_NO_SPECULATION = 1, 2, 4, 8
+DGS_KEEP_LOCAL_MODEL, DGS_RESIDUAL_MODE, DGS_HOST_IO, DGS_NO_SPECULATION, DGS_SINGLE_STREAM = 1, 2, 4, 8, 16
 DGS_THETA, DGS_U, DGS_D, DGS_THETA_LOCAL = 0, 1, 2, 3
 
 EXPORTS = (
     "dgs_arena_bytes", "dgs_init", "dgs_worker_push", "dgs_server_apply", "dgs_worker_pull",
     "dgs_event", "dgs_flush", "dgs_event_host", "dgs_state_ptr", "dgs_state_load", "dgs_status", "dgs_stats", "dgs_pull_read_stats",
     "dgs_prev", "dgs_launch_count", "dgs_last_cuda_error", "dgs_free", "dgs_error_string",
-    "dgs_timing_enable", "dgs_timing_read", "dgs_topk_encode_static",
+    "dgs_timing_enable", "dgs_timing_read", "dgs_timing_trace", "dgs_topk_encode_static",
 )
 DGS_ELIMIT = -6
 DGS_STATIC_MAX_N = 1 << 20
@@ -89,6 +89,8 @@ def lib() -> C.CDLL:
         L.dgs_topk_encode_static.argtypes = [vp, u32, u32, vp, vp, vp]
         L.dgs_timing_enable.argtypes = [vp, i32]
         L.dgs_timing_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
+        L.dgs_timing_trace.argtypes = [vp, u32, C.POINTER(C.c_float), C.POINTER(C.c_float), C.POINTER(C.c_int32),
+                                       C.POINTER(C.c_int32), C.POINTER(u32)]
         L.dgs_free.argtypes = [vp]
         L.dgs_error_string.argtypes = [i32]
         L.dgs_error_string.restype = C.c_char_p
@@ -212,6 +214,15 @@ def dgs_timing_read(ctx: int):
     cnt = (C.c_uint64 * DGS_NUM_KERNELS)()
     _check(lib().dgs_timing_read(ctx, ms, cnt), "dgs_timing_read")
     return {KERNEL_NAMES[i]: (float(ms[i]), int(cnt[i])) for i in range(DGS_NUM_KERNELS)}
+
+
+def dgs_timing_trace(ctx: int, cap: int = 65536):
+    """[(start_ms, stop_ms, kernel name, stream index)] of the launches recorded since the last read."""
+    a, b = (C.c_float * cap)(), (C.c_float * cap)()
+    k, s = (C.c_int32 * cap)(), (C.c_int32 * cap)()
+    cnt = C.c_uint32(0)
+    _check(lib().dgs_timing_trace(ctx, cap, a, b, k, s, C.byref(cnt)), "dgs_timing_trace")
+    return [(float(a[i]), float(b[i]), KERNEL_NAMES[k[i]], int(s[i])) for i in range(cnt.value)]
 
 
 def dgs_topk_encode_static(x_ptr: int, n: int, k: int, out_idx_ptr: int, out_val_ptr: int, stream: int = 0) -> None:

@@ -32,11 +32,17 @@ constexpr uint64_t kAlign = 256;
 constexpr uint32_t kMagic = 0x44475331u;  // "DGS1"
 constexpr int kPushSlots = 5;             // push packet slots, used in turn
 constexpr int kPullSlots = 6;             // pull packet slots
-constexpr int kWorkerStreams = 4, kServerStreams = 6;
+#ifndef DGS_WORKER_STREAMS
+#define DGS_WORKER_STREAMS 4
+#endif
+#ifndef DGS_SERVER_STREAMS
+#define DGS_SERVER_STREAMS 6
+#endif
+constexpr int kWorkerStreams = DGS_WORKER_STREAMS, kServerStreams = DGS_SERVER_STREAMS;
 constexpr int kPushSets = kWorkerStreams;  // scratch sets and spare velocity buffers of the pushes
 constexpr int kPullSets = kServerStreams;  // scratch sets of the pulls
 constexpr int kAllSets = kPushSets + kPullSets;
-constexpr int kLogRingMax = 64;           // most packets the apply log keeps (k_catch_up holds two ranges per lane)
+constexpr int kLogRingMax = kCatchMaxPackets;  // most packets the apply log keeps (one k_catch_up launch folds them all)
 enum StreamId : int { kStW0 = 0, kStApply = kWorkerStreams, kStS0 = kWorkerStreams + 1,
                       kNumStreams = kWorkerStreams + 1 + kServerStreams };
 
@@ -44,9 +50,9 @@ inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
 // Scratch of one selection pipeline ([0] push, on the worker stream; [1] pull, on the server stream)
 struct ScratchLayout {
-  uint64_t cand_idx, cand_val, part_cands, part_slot0, tile_pre, cta_tot, tile_sel;
+  uint64_t cand_idx, cand_val, part_cands, part_slot0, cta_tot, seg_start;
   uint64_t hist1, hist2, hist3, sel, L_safe, L_wide, sync;
-  uint64_t zero_begin, zero_end;  // [tile_sel, end of sync): cleared at init
+  uint64_t zero_begin, zero_end;  // [hist1, end of sync): cleared at init
 };
 
 struct Layout {
@@ -59,7 +65,8 @@ struct Layout {
   uint64_t tiles, segs, seg_off, seg_tile0;
   ScratchLayout sc[kAllSets];  // push sets, then pull sets
   uint64_t L_next, u_slots, status, stats;
-  uint64_t log_idx, log_val;
+  uint64_t log_idx, log_val, log_bnd, log_pos;
+  uint32_t log_ranges = 0;
   uint64_t blk_max;      // [N][blk_stride]: per block of kWarpTile elements, an upper bound on the keys of D_q in it
   uint64_t blk_stride = 0;  // ring of applied packets not yet folded into every D_q
   uint32_t log_ring = 0, log_stride = 0;
@@ -161,11 +168,10 @@ void make_layout(const dgs_config* c, Layout* L) {
     sc.cand_val = take(vec);
     sc.part_cands = take((uint64_t)kMaxGrid * 4);
     sc.part_slot0 = take((uint64_t)kMaxGrid * 4);
-    sc.tile_pre = take((uint64_t)L->num_tiles * sizeof(uint2));
     sc.cta_tot = take((uint64_t)kMaxWorkers * sizeof(uint2));
-    sc.tile_sel = take((uint64_t)L->num_tiles * sizeof(uint2));
-    sc.zero_begin = sc.tile_sel;
+    sc.seg_start = take(S * sizeof(uint2));
     sc.hist1 = take(S * kBins1 * 4);
+    sc.zero_begin = sc.hist1;
     sc.hist2 = take(S * kBins2 * 4);
     sc.hist3 = take(S * kBins3 * 4);
     sc.sel = take(S * sizeof(SegSel));
@@ -178,6 +184,15 @@ void make_layout(const dgs_config* c, Layout* L) {
   L->log_stride = (uint32_t)align_up(L->K[0], 64);
   L->log_idx = take((uint64_t)L->log_ring * L->log_stride * 4);
   L->log_val = take((uint64_t)L->log_ring * L->log_stride * 4);
+  {
+    // ranges of the log = CTAs of a catch-up: about kCatchTarget entries each when a worker has missed
+    // as many packets as there are workers, and no more ranges than a packet has entries
+    const uint64_t entries = std::min<uint64_t>(N, L->log_ring) * L->K[0];
+    L->log_ranges = (uint32_t)std::min<uint64_t>(std::min<uint64_t>(kCatchMaxGrid, L->K[0]),
+                                                 std::max<uint64_t>(1, (entries + kCatchTarget - 1) / kCatchTarget));
+  }
+  L->log_bnd = take((uint64_t)L->log_ranges * 4);
+  L->log_pos = take((uint64_t)L->log_ring * (L->log_ranges + 1) * 4);
   L->blk_stride = align_up((c->n + kWarpTile - 1) / kWarpTile, 64);
   L->blk_max = take(N * L->blk_stride * 4);
   L->L_next = take(2 * N * S * 4);
@@ -248,6 +263,7 @@ struct dgs_ctx {
   bool timing;
   std::vector<cudaEvent_t> ev_pool;   // pairs: [2i] start, [2i+1] stop
   std::vector<int> ev_kernel;         // kernel id of each recorded pair
+  std::vector<int> ev_stream;         // index of the library stream it ran on
   double time_ms[DGS_NUM_KERNELS];
   uint64_t time_count[DGS_NUM_KERNELS];
 
@@ -278,7 +294,8 @@ struct ResIds {
   uint32_t PKT(int slot) const { return 5 * N + 1 + kPushSets + kAllSets + slot; }   // push slots, then pull slots
   uint32_t STAGE() const { return PKT(kPushSlots + kPullSlots); }
   uint32_t LOG(uint32_t slot) const { return STAGE() + 1 + slot; }
-  uint32_t count() const { return LOG(kLogRingMax); }
+  uint32_t RANGES() const { return LOG(kLogRingMax); }   // the ranges of the log
+  uint32_t count() const { return RANGES() + 1; }
 };
 
 #define DGS_CUDA(ctx, call)                 \
@@ -298,7 +315,10 @@ inline int live(dgs_ctx* c) {
 }
 
 constexpr size_t kMaxTimedLaunches = 1 << 16;
-constexpr int kFinalizeWorkers = 64;  // CTAs of the finalize kernel (more of them take SM slots from the stream passes)
+#ifndef DGS_FINALIZE_WORKERS
+#define DGS_FINALIZE_WORKERS 64
+#endif
+constexpr int kFinalizeWorkers = DGS_FINALIZE_WORKERS;  // CTAs of the finalize kernel (more of them take SM slots from the stream passes)
 
 // Records an event before and after one launch when timing is on.
 struct TimedLaunch {
@@ -316,6 +336,10 @@ struct TimedLaunch {
     if (cudaEventRecord(c->ev_pool[2 * i], st) != cudaSuccess) return;
     stop = c->ev_pool[2 * i + 1];
     c->ev_kernel.push_back(kernel_id);
+    int which = -1;
+    for (int j = 0; j < kNumStreams; ++j)
+      if (c->st[j] == st) which = j;
+    c->ev_stream.push_back(which);
   }
   ~TimedLaunch() {
     if (stop) cudaEventRecord(stop, st);
@@ -391,6 +415,7 @@ int task_end(dgs_ctx* c, const Task& t) {
 void catch_up_deps(const dgs_ctx* c, uint32_t q, Task* t) {
   const ResIds R{c->cfg.num_workers};
   for (uint64_t p = c->applied[q]; p < c->log_head; ++p) t->reads.push_back(R.LOG((uint32_t)(p % c->log.ring)));
+  if (c->applied[q] < c->log_head) t->reads.push_back(R.RANGES());
   t->writes.push_back(R.D(q));
 }
 // The launch itself, on a stream that task_begin has prepared with those dependencies.
@@ -399,7 +424,7 @@ int catch_up_launch(dgs_ctx* c, uint32_t q, cudaStream_t st) {
   const uint32_t count = (uint32_t)(c->log_head - first);
   if (count > 0) {
     TimedLaunch tl(c, st, DGS_KERNEL_CATCH_UP);
-    k_catch_up<<<kCatchGrid, kThreads, 0, st>>>(c->log, first, count, c->D_buf(q), c->blk_max(q), c->cfg.n);
+    k_catch_up<<<c->log.ranges, kCatchThreads, 0, st>>>(c->log, first, count, c->D_buf(q), c->blk_max(q), c->cfg.n);
     DGS_CUDA(c, cudaGetLastError());
     c->launches += 1;
   }
@@ -484,8 +509,8 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age
     // cooperative launch: the CTAs synchronise among themselves, so all must be resident
     TimedLaunch t(c, st, MODE == kPull ? DGS_KERNEL_FINALIZE_PULL : DGS_KERNEL_FINALIZE_PUSH);
     void* args[] = {(void*)&ws, (void*)&a};
-    DGS_CUDA(c, cudaLaunchCooperativeKernel((const void*)k_finalize<MODE>, dim3(fin_grid), dim3(kThreads), args, 0,
-                                            st));
+    DGS_CUDA(c, cudaLaunchCooperativeKernel((const void*)k_finalize<MODE>, dim3(fin_grid), dim3(kThreads), args,
+                                            finalize_dyn_bytes(c->cfg.num_segments), st));
     c->launches += 1;
   }
   rc = task_end(c, task);
@@ -508,10 +533,14 @@ int occupancy_grids(dgs_ctx* c, int sms) {
                                                             StreamRing<MODE>::kBytes));
   if (occ < 1) occ = 1;
   c->stream_grid[MODE] = std::min(sms * occ, kMaxGrid);
+#ifdef DGS_PULL_GRID
+  if (MODE == kPull) c->stream_grid[MODE] = std::min(c->stream_grid[MODE], DGS_PULL_GRID);
+#endif
   DGS_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_hist_all<MODE>, kThreads, 0));
   if (occ < 1) occ = 1;
   c->hist_grid[MODE] = std::min(sms * occ, kMaxGrid);
-  DGS_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_finalize<MODE>, kThreads, 0));
+  DGS_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_finalize<MODE>, kThreads,
+                                                            finalize_dyn_bytes(c->cfg.num_segments)));
   if (occ < 1) {
     c->last_cuda = (int)cudaErrorCooperativeLaunchTooLarge;
     c->broken = true;
@@ -524,7 +553,7 @@ int occupancy_grids(dgs_ctx* c, int sms) {
 
 void destroy_ctx(dgs_ctx* c) {
   for (int i = 0; i < kNumStreams; ++i) {
-    if (c->st[i]) cudaStreamDestroy(c->st[i]);
+    if (c->st[i] && (i == 0 || c->st[i] != c->st[0])) cudaStreamDestroy(c->st[i]);
     if (c->ev_tail[i]) cudaEventDestroy(c->ev_tail[i]);
   }
   if (c->ev_in) cudaEventDestroy(c->ev_in);
@@ -642,7 +671,10 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
     // The push passes move most of the bytes and fill every SM; the short kernels of the server side sit on
     // the longer chain (apply -> catch-up -> pull), so their blocks go first whenever an SM has room.
     const int prio = i < kStApply ? prio_low : prio_high;
-    INIT_CUDA(cudaStreamCreateWithPriority(&c->st[i], cudaStreamNonBlocking, prio));
+    if (i > 0 && (cfg->flags & DGS_SINGLE_STREAM))
+      c->st[i] = c->st[0];   // every step on one stream: kernels run one after the other, in call order
+    else
+      INIT_CUDA(cudaStreamCreateWithPriority(&c->st[i], cudaStreamNonBlocking, prio));
     INIT_CUDA(cudaEventCreateWithFlags(&c->ev_tail[i], cudaEventDisableTiming));
   }
   INIT_CUDA(cudaEventCreateWithFlags(&c->ev_in, cudaEventDisableTiming));
@@ -711,9 +743,8 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
     w.cand_val = c->at<float>(sc.cand_val);
     w.part_cands = c->at<uint32_t>(sc.part_cands);
     w.part_slot0 = c->at<uint32_t>(sc.part_slot0);
-    w.tile_pre = c->at<uint2>(sc.tile_pre);
-    w.tile_sel = c->at<uint2>(sc.tile_sel);
     w.cta_tot = c->at<uint2>(sc.cta_tot);
+    w.seg_start = c->at<uint2>(sc.seg_start);
     w.hist1 = c->at<uint32_t>(sc.hist1);
     w.hist2 = c->at<uint32_t>(sc.hist2);
     w.hist3 = c->at<uint32_t>(sc.hist3);
@@ -729,6 +760,9 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   c->log.stride = L.log_stride;
   c->log.cap = (uint32_t)L.K[0];
   c->log.ring = L.log_ring;
+  c->log.bnd = c->at<uint32_t>(L.log_bnd);
+  c->log.pos = c->at<uint32_t>(L.log_pos);
+  c->log.ranges = L.log_ranges;
   *out = c;
   return DGS_OK;
 }
@@ -788,6 +822,15 @@ int apply_impl(dgs_ctx* c, uint32_t worker, const dgs_packet* pkt) {
     // Its slot of the log still holds the packet filed `ring` applies ago; whoever has not folded that
     // one in yet does so first.
     const uint32_t lslot = (uint32_t)(c->log_head % c->log.ring);
+    // The ranges of the log are taken from the first packet filed, again from packet N (velocities have
+    // built up by then) and then every 16 N packets, so that they follow a drifting distribution.  The
+    // positions filed with older packets refer to the old ranges: nobody may still need those packets.
+    const bool new_ranges = c->log_head == 0 || c->log_head == N || c->log_head % (16ull * N) == 0;
+    if (new_ranges)
+      for (uint32_t q = 0; q < N; ++q) {
+        const int rc = catch_up_now(c, q);
+        if (rc != DGS_OK) return rc;
+      }
     if (c->log_head >= c->log.ring) {
       const uint64_t oldest = c->log_head - c->log.ring;
       for (uint32_t q = 0; q < N; ++q)
@@ -800,12 +843,20 @@ int apply_impl(dgs_ctx* c, uint32_t worker, const dgs_packet* pkt) {
     t.stream = kStApply;
     t.reads.push_back(R.PKT(slot));
     t.writes = {R.THETA(), R.LOG(lslot)};
+    if (new_ranges) t.writes.push_back(R.RANGES());
     int rc = task_begin(c, t);
     if (rc != DGS_OK) return rc;
     {
       TimedLaunch tl(c, c->st[kStApply], DGS_KERNEL_SCATTER);
-      k_apply_log<<<gx, kThreads, 0, c->st[kStApply]>>>(pkt->idx, pkt->val, pkt->count, c->at<float>(c->lay.theta),
-                                                        c->cfg.n, c->ws[0].status, c->log, lslot);
+      if (new_ranges) {
+        k_log_ranges<<<(c->log.ranges + kThreads - 1) / kThreads, kThreads, 0, c->st[kStApply]>>>(pkt->idx, c->log);
+        DGS_CUDA(c, cudaGetLastError());
+        c->launches += 1;
+      }
+      const uint32_t pos_ctas = (c->log.ranges + 1 + kThreads - 1) / kThreads;
+      k_apply_log<<<gx + pos_ctas, kThreads, 0, c->st[kStApply]>>>(pkt->idx, pkt->val, pkt->count,
+                                                                   c->at<float>(c->lay.theta), c->cfg.n,
+                                                                   c->ws[0].status, c->log, lslot, gx);
       DGS_CUDA(c, cudaGetLastError());
       c->launches += 1;
     }
@@ -1107,12 +1158,33 @@ int dgs_timing_read(dgs_ctx* c, double ms[DGS_NUM_KERNELS], uint64_t count[DGS_N
     c->time_count[c->ev_kernel[i]] += 1;
   }
   c->ev_kernel.clear();
+  c->ev_stream.clear();
   for (int i = 0; i < DGS_NUM_KERNELS; ++i) {
     ms[i] = c->time_ms[i];
     count[i] = c->time_count[i];
     c->time_ms[i] = 0.0;
     c->time_count[i] = 0;
   }
+  return DGS_OK;
+}
+
+int dgs_timing_trace(dgs_ctx* c, uint32_t cap, float* start_ms, float* stop_ms, int32_t* kernel, int32_t* stream,
+                     uint32_t* count) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (!start_ms || !stop_ms || !kernel || !stream || !count) return DGS_EINVAL;
+  rc = sync_all(c);
+  if (rc != DGS_OK) return rc;
+  const size_t m = std::min<size_t>(cap, c->ev_kernel.size());
+  for (size_t i = 0; i < m; ++i) {
+    DGS_CUDA(c, cudaEventElapsedTime(start_ms + i, c->ev_pool[0], c->ev_pool[2 * i]));
+    DGS_CUDA(c, cudaEventElapsedTime(stop_ms + i, c->ev_pool[0], c->ev_pool[2 * i + 1]));
+    kernel[i] = c->ev_kernel[i];
+    stream[i] = c->ev_stream[i];
+  }
+  *count = (uint32_t)m;
+  c->ev_kernel.clear();
+  c->ev_stream.clear();
   return DGS_OK;
 }
 
@@ -1142,11 +1214,10 @@ struct StaticScratch {
   uint32_t cand_idx[kStaticMaxN];
   float cand_val[kStaticMaxN];
   Tile tiles[kStaticMaxTiles];
-  uint2 tile_sel[kStaticMaxTiles];
-  uint2 tile_pre[kStaticMaxTiles];
   uint32_t part_cands[kMaxGrid];
   uint32_t part_slot0[kMaxGrid];
   uint2 cta_tot[kMaxWorkers];
+  uint2 seg_start[1];
   uint32_t hist1[kBins1];
   uint32_t hist2[kBins2];
   uint32_t hist3[kBins3];
@@ -1175,7 +1246,6 @@ __global__ void k_static_prepare(StaticScratch* sc, uint32_t n, uint32_t k, uint
     t.len = (uint16_t)min((uint32_t)kWarpTile, n - i * kWarpTile);
     t.seg = 0;
     sc->tiles[i] = t;
-    sc->tile_sel[i] = make_uint2(0, 0);
   }
   if (i < kBins1) sc->hist1[i] = 0;
   if (i < kBins2) sc->hist2[i] = 0;
@@ -1226,7 +1296,9 @@ int static_setup(int dev, StaticDevice** out) {
     d.stream_grid = std::min(sms * std::max(occ, 1), kMaxGrid);
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_hist_all<kPull>, kThreads, 0) != cudaSuccess) return DGS_ECUDA;
     d.hist_grid = std::min(sms * std::max(occ, 1), kMaxGrid);
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_finalize<kPull>, kThreads, 0) != cudaSuccess || occ < 1)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_finalize<kPull>, kThreads, finalize_dyn_bytes(1)) !=
+            cudaSuccess ||
+        occ < 1)
       return DGS_ECUDA;
     d.finalize_grid = std::min(std::min(sms * occ, kMaxWorkers), kFinalizeWorkers);
     d.scratch = static_cast<StaticScratch*>(p);
@@ -1262,9 +1334,8 @@ extern "C" int dgs_topk_encode_static(const float* x, uint32_t n, uint32_t k, ui
   ws.part_slot0 = sc->part_slot0;
   ws.seg_off = sc->seg_off;
   ws.seg_tile0 = sc->seg_tile0;
-  ws.tile_sel = sc->tile_sel;
-  ws.tile_pre = sc->tile_pre;
   ws.cta_tot = sc->cta_tot;
+  ws.seg_start = sc->seg_start;
   ws.hist1 = sc->hist1;
   ws.hist2 = sc->hist2;
   ws.hist3 = sc->hist3;
@@ -1298,8 +1369,8 @@ extern "C" int dgs_topk_encode_static(const float* x, uint32_t n, uint32_t k, ui
   k_stream<kPull><<<d->stream_grid, kThreads, StreamRing<kPull>::kBytes, st>>>(ws, a);
   if (cudaGetLastError() != cudaSuccess) return DGS_ECUDA;
   void* args[] = {(void*)&ws, (void*)&a};
-  if (cudaLaunchCooperativeKernel((const void*)k_finalize<kPull>, dim3(d->finalize_grid), dim3(kThreads), args, 0,
-                                  st) != cudaSuccess)
+  if (cudaLaunchCooperativeKernel((const void*)k_finalize<kPull>, dim3(d->finalize_grid), dim3(kThreads), args,
+                                  finalize_dyn_bytes(1), st) != cudaSuccess)
     return DGS_ECUDA;
   return DGS_OK;
 }

@@ -37,7 +37,7 @@ constexpr int kBins3 = 1024;        // key bits  9..0
 constexpr uint32_t kFull = 0xFFFFFFFFu;
 constexpr uint32_t kSpecFactor = 2; // aim for max(2k, k+64) candidates next time
 constexpr uint32_t kSpecSlack = 64;
-constexpr int kMaxGrid = 1024;      // upper bound on the grid of a stream pass (= parts of the candidate buffer)
+constexpr int kMaxGrid = 512;       // upper bound on the grid of a stream pass (= parts of the candidate buffer)
 constexpr int kMaxWorkers = 320;    // upper bound on the grid of finalize
 constexpr uint32_t kSpinLimit = 1u << 22;  // bounded waits: give up and report after this many polls
 constexpr int kStatusTimeout = -4;  // = DGS_ETIMEOUT
@@ -61,6 +61,7 @@ struct SegSel {        // per-layer selection state of the selection in flight
   uint32_t krem;       // entries still to take at or below the fixed prefix
   uint32_t T;          // k-th largest key
   uint32_t r;          // entries with key == T that are taken (lowest indices)
+  uint32_t neq;        // candidates with key == T
 };
 
 // word indices in Workspace::sync
@@ -78,9 +79,8 @@ struct Workspace {
   uint32_t* part_slot0;   // [kMaxGrid] first slot of each part
   const uint32_t* seg_off;   // [S+1] first element of each layer, and n
   const uint32_t* seg_tile0; // [S]   first tile of each layer
-  uint2* tile_sel;        // [num_tiles] (#key > T, #key == T) per tile; all zero between selections
-  uint2* tile_pre;        // [num_tiles] exclusive prefix of tile_sel inside the scanning CTA's chunk
-  uint2* cta_tot;         // [kMaxWorkers]
+  uint2* cta_tot;         // [kMaxWorkers] (#key > T, #key == T) among the candidates of each CTA of finalize
+  uint2* seg_start;       // [S] the same counted over all earlier layers
   uint32_t* hist1;        // [S][kBins1]
   uint32_t* hist2;        // [S][kBins2]
   uint32_t* hist3;        // [S][kBins3]
@@ -170,10 +170,18 @@ __device__ __forceinline__ void load_tile_vec(const float* __restrict__ a, const
 }
 
 // ---- stream pass ----------------------------------------------------------------
+// Candidates are appended in INDEX ORDER: a CTA owns a contiguous range of tiles and a region
+// of the candidate buffer; it takes its tiles in rounds of kWarps consecutive tiles (one per
+// warp).  In a round every warp first counts the candidates of its tile, the counts are
+// exchanged through shared memory, and each warp then writes its candidates behind those of the
+// warps holding earlier tiles.  Read part after part, the candidate buffer therefore lists all
+// candidates of the vector in ascending index order, which is what lets the finalize kernel
+// number the selected ones with a plain prefix sum.
 constexpr int kLiveWords = 128;     // one bit per stage-sized chunk of a CTA's share of a layer
 struct StreamShared {
-  uint32_t hist[kBins1];  // top 11 key bits of the candidates of the layer being processed
-  uint32_t cursor;        // candidates appended by this CTA so far
+  uint32_t hist[kBins1];      // top 11 key bits of the candidates of the layer being processed
+  uint32_t cursor;            // candidates appended by this CTA so far
+  uint32_t wcnt[2][kWarps];   // candidates per warp of the current round (two rounds alternate)
   uint32_t live[kLiveWords];  // pull: chunks that may hold a candidate (the others are not read)
 };
 
@@ -187,13 +195,25 @@ __device__ __forceinline__ void flush_hist(uint32_t* s_hist, uint32_t* g_hist) {
   }
 }
 
-// What follows the loads of a full tile: x[16] holds this lane's values (4 float4 at
-// elements j*128 + lane*4 + c of the tile).  Writes the new velocity (push), appends the
-// tile's candidates in index order to the CTA's region, histograms their top key bits.
+// candidates of warps 0 .. warp-1 in this round, and of all warps
+__device__ __forceinline__ uint32_t round_offset(const uint32_t* wcnt, int warp, uint32_t& total) {
+  uint32_t before = 0, tot = 0;
+#pragma unroll
+  for (int w = 0; w < kWarps; ++w) {
+    const uint32_t c = wcnt[w];
+    if (w < warp) before += c;
+    tot += c;
+  }
+  total = tot;
+  return before;
+}
+
+// A full tile held in registers: x[16] are this lane's values (4 float4 at elements
+// j*128 + lane*4 + c of the tile).  Returns the candidate mask; writes the new velocity (push).
 template <int MODE>
-__device__ __forceinline__ void finish_full_tile(const Workspace& ws, const SelArgs& a, StreamShared& sh,
-                                                 uint32_t tile_start, const float (&x)[4 * kVecIters], uint32_t L,
-                                                 uint32_t slot0, int lane, uint32_t lt, float* __restrict__ out) {
+__device__ __forceinline__ uint32_t tile_mask_regs(const SelArgs& a, uint32_t tile_start,
+                                                   const float (&x)[4 * kVecIters], uint32_t L, int lane,
+                                                   float* __restrict__ out) {
   uint32_t mask = 0;
 #pragma unroll
   for (int e = 0; e < 4 * kVecIters; ++e)
@@ -210,40 +230,55 @@ __device__ __forceinline__ void finish_full_tile(const Workspace& ws, const SelA
       __stcs(po + j * 32, o);
     }
   }
-  const uint32_t total = __reduce_add_sync(kFull, (uint32_t)__popc(mask));
-  if (total) {
-    uint32_t base = 0;
-    if (lane == 0) base = slot0 + atomicAdd(&sh.cursor, total);
-    base = __shfl_sync(kFull, base, 0);
+  return mask;
+}
+
+// Writes the candidates of a full tile (mask from tile_mask_*) from slot `base` on, in index
+// order, and histograms their top key bits.  The cost is proportional to the candidates: one
+// packed warp scan gives every lane the rank of its candidates (lane l holds elements
+// j*128 + l*4 + c, order is j-major, so the four per-j counts travel as four bytes of one
+// word), and a lane that has candidates walks its set bits.  value(off) returns element `off`.
+template <typename ValueFn>
+__device__ __forceinline__ void tile_emit(const Workspace& ws, StreamShared& sh, uint32_t tile_start, uint32_t mask,
+                                          uint32_t base, int lane, ValueFn value) {
+  if (!__any_sync(kFull, mask != 0)) return;
+  // per-j candidate counts of this lane, one per byte
+  uint32_t t = mask - ((mask >> 1) & 0x5555u);
+  t = (t & 0x3333u) + ((t >> 2) & 0x3333u);                       // nibble j = count of nibble j of mask
+  const uint32_t packed = (t & 0xFu) | ((t & 0xF0u) << 4) | ((t & 0xF00u) << 8) | ((t & 0xF000u) << 12);
+  uint32_t incl = packed;                                          // byte j: inclusive prefix over lanes (<= 128)
 #pragma unroll
-    for (int j = 0; j < kVecIters; ++j) {
-      const uint32_t mj = (mask >> (j * 4)) & 0xFu;
-      if (!__any_sync(kFull, mj != 0)) continue;
-      const uint32_t b0 = __ballot_sync(kFull, mj & 1u), b1 = __ballot_sync(kFull, mj & 2u);
-      const uint32_t b2 = __ballot_sync(kFull, mj & 4u), b3 = __ballot_sync(kFull, mj & 8u);
-      uint32_t pos = base + __popc(b0 & lt) + __popc(b1 & lt) + __popc(b2 & lt) + __popc(b3 & lt);
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        if ((mj >> c) & 1u) {
-          const float v = x[4 * j + c];
-          ws.cand_idx[pos] = tile_start + j * 128 + lane * 4 + c;
-          ws.cand_val[pos] = v;
-          atomicAdd(sh.hist + (key_of(v) >> 20), 1u);
-          ++pos;
-        }
-      }
-      base += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t o = __shfl_up_sync(kFull, incl, d);
+    if (lane >= d) incl += o;
+  }
+  const uint32_t tot = __shfl_sync(kFull, incl, 31);
+  const uint32_t t0 = tot & 0xFFu, t1 = (tot >> 8) & 0xFFu, t2 = (tot >> 16) & 0xFFu;
+  if (mask) {
+    const uint32_t excl = incl - packed;                           // byte j: candidates of lower lanes at step j
+    uint32_t m = mask;
+    while (m) {
+      const int e = __ffs(m) - 1;
+      m &= m - 1;
+      const int j = e >> 2, c = e & 3;
+      const uint32_t before_j = j == 0 ? 0u : (j == 1 ? t0 : (j == 2 ? t0 + t1 : t0 + t1 + t2));
+      const uint32_t in_lane = __popc((mask >> (4 * j)) & ((1u << c) - 1u));
+      const uint32_t pos = base + before_j + ((excl >> (8 * j)) & 0xFFu) + in_lane;
+      const uint32_t off = j * 128 + lane * 4 + c;
+      const float v = value(off);
+      ws.cand_idx[pos] = tile_start + off;
+      ws.cand_val[pos] = v;
+      atomicAdd(sh.hist + (key_of(v) >> 20), 1u);
     }
   }
 }
 
 // A ragged tile (first or last of a layer, fewer than kWarpTile elements or not 16-byte
-// aligned): one element per lane and step, straight from global memory.  At most 16
-// steps; candidate flags are kept as one bit per step.
+// aligned): one element per lane and step, straight from global memory, at most 16 steps.
+// Returns the candidate flags (one bit per step); writes the new velocity (push).
 template <int MODE>
-__device__ __forceinline__ void ragged_tile(const Workspace& ws, const SelArgs& a, StreamShared& sh, const Tile tile,
-                                            uint32_t L, uint32_t slot0, int lane, uint32_t lt,
-                                            const float* __restrict__ in, float* __restrict__ out) {
+__device__ __forceinline__ uint32_t ragged_mask(const SelArgs& a, const Tile tile, uint32_t L, int lane,
+                                                const float* __restrict__ in, float* __restrict__ out) {
   uint32_t flags = 0;
   for (int st = 0; st * 32 < (int)tile.len; ++st) {
     const uint32_t off = st * 32 + lane;
@@ -255,32 +290,34 @@ __device__ __forceinline__ void ragged_tile(const Workspace& ws, const SelArgs& 
       if (cand) flags |= 1u << st;
     }
   }
-  const uint32_t total = __reduce_add_sync(kFull, (uint32_t)__popc(flags));
-  if (total) {
-    uint32_t base = 0;
-    if (lane == 0) base = slot0 + atomicAdd(&sh.cursor, total);
-    base = __shfl_sync(kFull, base, 0);
-    for (int st = 0; st * 32 < (int)tile.len; ++st) {
-      const bool cand = (flags >> st) & 1u;
-      const uint32_t b = __ballot_sync(kFull, cand);
-      if (cand) {
-        // a candidate's value is what this thread just stored (push) or the input itself (pull)
-        const uint32_t i = tile.start + st * 32 + lane;
-        const float x = MODE == kPull ? in[i] : out[i];
-        const uint32_t pos = base + __popc(b & lt);
-        ws.cand_idx[pos] = i;
-        ws.cand_val[pos] = x;
-        atomicAdd(sh.hist + (key_of(x) >> 20), 1u);
-      }
-      base += __popc(b);
+  return flags;
+}
+// Writes its candidates from slot `base` on, in index order.
+template <int MODE>
+__device__ __forceinline__ void ragged_emit(const Workspace& ws, StreamShared& sh, const Tile tile, uint32_t flags,
+                                            uint32_t base, int lane, uint32_t lt, const float* __restrict__ in,
+                                            const float* __restrict__ out) {
+  if (!__any_sync(kFull, flags != 0)) return;
+  for (int st = 0; st * 32 < (int)tile.len; ++st) {
+    const bool cand = (flags >> st) & 1u;
+    const uint32_t b = __ballot_sync(kFull, cand);
+    if (cand) {
+      // a candidate's value is what this thread just stored (push) or the input itself (pull)
+      const uint32_t i = tile.start + st * 32 + lane;
+      const float x = MODE == kPull ? in[i] : out[i];
+      const uint32_t pos = base + __popc(b & lt);
+      ws.cand_idx[pos] = i;
+      ws.cand_val[pos] = x;
+      atomicAdd(sh.hist + (key_of(x) >> 20), 1u);
     }
+    base += __popc(b);
   }
 }
 
-// CTA `cta` of `G` handles a contiguous range of tiles, one tile per warp at a time,
-// layer by layer, so that the CTA's shared histogram always belongs to one layer; it
-// is added to the global one when the CTA leaves the layer.  Loads go straight from
-// global memory to registers (used where only a few CTAs run the pass).
+// CTA `cta` of `G` handles a contiguous range of tiles, kWarps consecutive tiles per round,
+// layer by layer, so that the CTA's shared histogram always belongs to one layer; it is added
+// to the global one when the CTA leaves the layer.  Loads go straight from global memory to
+// registers (used where only a few CTAs run the pass).
 template <int MODE>
 __device__ void stream_tiles(const Workspace& ws, const SelArgs& a, const uint32_t* Larr,
                              const float* __restrict__ in, float* __restrict__ out, uint32_t cta, uint32_t G,
@@ -303,22 +340,46 @@ __device__ void stream_tiles(const Workspace& ws, const SelArgs& a, const uint32
   }
   const uint32_t slot0 = ws.tiles[t0].start;  // first slot of this CTA's region
   const uint32_t seg_first = ws.tiles[t0].seg, seg_last = ws.tiles[t1 - 1].seg;
+  uint32_t cur = 0;      // candidates appended so far (the same in every thread)
+  uint32_t round = 0;
   for (uint32_t s = seg_first; s <= seg_last; ++s) {
     const uint32_t a0 = max(t0, ws.segs[s].tile_begin), a1 = min(t1, ws.segs[s].tile_end);
     const uint32_t L = Larr[s];
-    uint32_t t = a0 + warp;
-    Tile next;
-    next.start = 0; next.len = 0; next.seg = 0;
-    if (t < a1) next = ws.tiles[t];
-    for (; t < a1; t += kWarps) {
-      const Tile tile = next;
-      if (t + kWarps < a1) next = ws.tiles[t + kWarps];
-      if (tile.len == kWarpTile) {
-        float x[4 * kVecIters];
-        load_tile_vec<MODE>(in, a.grad, tile.start, lane, a.m, a.lr, x);
-        finish_full_tile<MODE>(ws, a, sh, tile.start, x, L, slot0, lane, lt, out);
-      } else {
-        ragged_tile<MODE>(ws, a, sh, tile, L, slot0, lane, lt, in, out);
+    for (uint32_t tb = a0; tb < a1; tb += kWarps, ++round) {
+      const uint32_t t = tb + warp;
+      Tile tile;
+      tile.start = 0; tile.len = 0; tile.seg = 0;
+      float x[4 * kVecIters];
+      uint32_t mask = 0;
+      if (t < a1) {
+        tile = ws.tiles[t];
+        if (tile.len == kWarpTile) {
+          load_tile_vec<MODE>(in, a.grad, tile.start, lane, a.m, a.lr, x);
+          mask = tile_mask_regs<MODE>(a, tile.start, x, L, lane, out);
+        } else {
+          mask = ragged_mask<MODE>(a, tile, L, lane, in, out);
+        }
+      }
+      const uint32_t count = __reduce_add_sync(kFull, (uint32_t)__popc(mask));
+      if (lane == 0) sh.wcnt[round & 1][warp] = count;
+      __syncthreads();
+      uint32_t total;
+      const uint32_t base = slot0 + cur + round_offset(sh.wcnt[round & 1], warp, total);
+      cur += total;
+      if (t < a1) {
+        if (tile.len == kWarpTile) {
+          tile_emit(ws, sh, tile.start, mask, base, lane, [&](uint32_t off) {
+            // element off = j*128 + lane*4 + c is register 4*j + c of this lane
+            const int e = (int)(((off >> 7) << 2) | (off & 3u));
+            float v = x[0];
+#pragma unroll
+            for (int q = 1; q < 4 * kVecIters; ++q)
+              if (q == e) v = x[q];
+            return v;
+          });
+        } else {
+          ragged_emit<MODE>(ws, sh, tile, mask, base, lane, lt, in, out);
+        }
       }
     }
     __syncthreads();
@@ -326,22 +387,16 @@ __device__ void stream_tiles(const Workspace& ws, const SelArgs& a, const uint32
     __syncthreads();
   }
   if (threadIdx.x == 0) {
-    ws.part_cands[cta] = sh.cursor;
+    ws.part_cands[cta] = cur;
     ws.part_slot0[cta] = slot0;
   }
 }
 
-// The same for a tile staged in shared memory (su: the tile of the state vector, sg: the
-// tile of the gradient, push only).  The cost beyond the streaming part is kept
-// proportional to the number of candidates: one packed warp scan gives every lane the
-// rank of its candidates (lane l holds elements j*128 + l*4 + c, order is j-major, so the
-// four per-j counts travel as four bytes of one word), and a lane that has candidates
-// walks its set bits and recomputes their values from shared memory.
+// Step one for a tile staged in shared memory (su: the tile of the state vector, sg: the tile
+// of the gradient, push only): candidate mask, new velocity (push), block bound (pull).
 template <int MODE>
-__device__ __forceinline__ void finish_full_tile_smem(const Workspace& ws, const SelArgs& a, StreamShared& sh,
-                                                      uint32_t tile_start, const float* su, const float* sg,
-                                                      uint32_t L, uint32_t slot0, int lane,
-                                                      float* __restrict__ out) {
+__device__ __forceinline__ uint32_t tile_mask_smem(const SelArgs& a, uint32_t tile_start, const float* su,
+                                                   const float* sg, uint32_t L, int lane, float* __restrict__ out) {
   const float Lf = __uint_as_float(L);   // |x| >= Lf  <=>  key(x) >= L for finite x (no flush-to-zero)
   const float4* pu = reinterpret_cast<const float4*>(su) + lane;
   const float4* pg = reinterpret_cast<const float4*>(sg) + lane;
@@ -374,53 +429,37 @@ __device__ __forceinline__ void finish_full_tile_smem(const Workspace& ws, const
     top = __reduce_max_sync(kFull, top);
     if (lane == 0) a.blk_max[tile_start / kWarpTile] = top;
   }
-  if (!__any_sync(kFull, mask != 0)) return;
-  // per-j candidate counts of this lane, one per byte
-  uint32_t t = mask - ((mask >> 1) & 0x5555u);
-  t = (t & 0x3333u) + ((t >> 2) & 0x3333u);                       // nibble j = count of nibble j of mask
-  const uint32_t packed = (t & 0xFu) | ((t & 0xF0u) << 4) | ((t & 0xF00u) << 8) | ((t & 0xF000u) << 12);
-  uint32_t incl = packed;                                          // byte j: inclusive prefix over lanes (<= 128)
-#pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    const uint32_t o = __shfl_up_sync(kFull, incl, d);
-    if (lane >= d) incl += o;
-  }
-  const uint32_t tot = __shfl_sync(kFull, incl, 31);
-  const uint32_t t0 = tot & 0xFFu, t1 = (tot >> 8) & 0xFFu, t2 = (tot >> 16) & 0xFFu, t3 = tot >> 24;
-  uint32_t base = 0;
-  if (lane == 0) base = slot0 + atomicAdd(&sh.cursor, t0 + t1 + t2 + t3);
-  base = __shfl_sync(kFull, base, 0);
-  if (mask) {
-    const uint32_t excl = incl - packed;                           // byte j: candidates of lower lanes at step j
-    uint32_t m = mask;
-    while (m) {
-      const int e = __ffs(m) - 1;
-      m &= m - 1;
-      const int j = e >> 2, c = e & 3;
-      const uint32_t before_j = j == 0 ? 0u : (j == 1 ? t0 : (j == 2 ? t0 + t1 : t0 + t1 + t2));
-      const uint32_t in_lane = __popc((mask >> (4 * j)) & ((1u << c) - 1u));
-      const uint32_t pos = base + before_j + ((excl >> (8 * j)) & 0xFFu) + in_lane;
-      const uint32_t off = j * 128 + lane * 4 + c;
-      const float v = combine<MODE>(su[off], MODE != kPull ? sg[off] : 0.f, a.m, a.lr);
-      ws.cand_idx[pos] = tile_start + off;
-      ws.cand_val[pos] = v;
-      atomicAdd(sh.hist + (key_of(v) >> 20), 1u);
-    }
-  }
+  return mask;
 }
 
 // ---- the same pass with TMA-staged tiles --------------------------------------------
 // Full tiles are brought into a ring of shared-memory stages by bulk asynchronous copies
 // (cp.async.bulk, completion counted on an mbarrier per stage), kStageTiles tiles of each
 // input per stage, so that several stages are in flight while the warps work on one: the
-// bytes in flight no longer depend on how many warps are waiting at a load.
+// bytes in flight no longer depend on how many warps are waiting at a load.  One round of the
+// ordered append = one stage; the barrier between counting and writing is also the one after
+// which the stage of the round before is free, so a ring of kStages stages keeps kStages - 1
+// of them in flight.
 constexpr int kStageTiles = kWarps;                        // one tile per warp and stage
 constexpr int kStageFloats = kStageTiles * kWarpTile;      // per input array
+// Tunables of the ring (compile-time): stages per CTA, and the least dynamic shared memory a push
+// CTA asks for.  Asking for more than the ring needs caps the CTAs of the push pass per SM, which
+// leaves room on every SM for the short kernels of other streams (finalize, catch-up, pull).
+#ifndef DGS_PUSH_STAGES
+#define DGS_PUSH_STAGES 3
+#endif
+#ifndef DGS_PULL_STAGES
+#define DGS_PULL_STAGES 4
+#endif
+#ifndef DGS_PUSH_MIN_SMEM
+#define DGS_PUSH_MIN_SMEM 0
+#endif
 template <int MODE> struct StreamRing {
   static constexpr int kInputs = MODE == kPull ? 1 : 2;
-  static constexpr int kStages = MODE == kPull ? 3 : 2;
-  static constexpr int kStageBytes = kInputs * kStageFloats * 4;
-  static constexpr int kBytes = kStages * kStageBytes;     // 80 KB (pull) / 96 KB (push)
+  static constexpr int kStages = MODE == kPull ? DGS_PULL_STAGES : DGS_PUSH_STAGES;
+  static constexpr int kStageBytes = kInputs * kStageFloats * 4;          // 16 KB per input
+  static constexpr int kRingBytes = kStages * kStageBytes;
+  static constexpr int kBytes = MODE != kPull && kRingBytes < DGS_PUSH_MIN_SMEM ? DGS_PUSH_MIN_SMEM : kRingBytes;
 };
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -456,6 +495,7 @@ __device__ void stream_tiles_tma(const Workspace& ws, const SelArgs& a, const ui
                                  const float* __restrict__ in, float* __restrict__ out, uint32_t cta, uint32_t G,
                                  StreamShared& sh, float* ring, uint64_t* full, int* s_dead) {
   using R = StreamRing<MODE>;
+  static_assert(R::kStages >= 2, "the ring needs a stage in flight besides the one being read");
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t t0 = part_first_tile(cta, G, ws.num_tiles), t1 = part_first_tile(cta + 1, G, ws.num_tiles);
   const uint32_t lt = lanemask_lt();
@@ -478,6 +518,7 @@ __device__ void stream_tiles_tma(const Workspace& ws, const SelArgs& a, const ui
   const uint32_t slot0 = ws.tiles[t0].start;
   const uint32_t seg_first = ws.tiles[t0].seg, seg_last = ws.tiles[t1 - 1].seg;
   uint32_t uses = 0;  // stage uses so far (same in every thread): stage = use % kStages, parity = (use / kStages) & 1
+  uint32_t cur = 0;   // candidates appended so far (same in every thread)
   for (uint32_t s = seg_first; s <= seg_last; ++s) {
     const uint32_t a0 = max(t0, ws.segs[s].tile_begin), a1 = min(t1, ws.segs[s].tile_end);
     const uint32_t L = Larr[s];
@@ -485,8 +526,20 @@ __device__ void stream_tiles_tma(const Workspace& ws, const SelArgs& a, const ui
     const bool head = ws.tiles[a0].len != kWarpTile;
     const bool tail = (a1 - 1 > a0 || !head) && ws.tiles[a1 - 1].len != kWarpTile;
     const uint32_t f0 = a0 + (head ? 1u : 0u), f1 = a1 - (tail ? 1u : 0u);   // full tiles [f0, f1)
-    if (head && warp == 0) ragged_tile<MODE>(ws, a, sh, ws.tiles[a0], L, slot0, lane, lt, in, out);
-    if (tail && warp == 1) ragged_tile<MODE>(ws, a, sh, ws.tiles[a1 - 1], L, slot0, lane, lt, in, out);
+    // a ragged tile is one warp's work; the warp tells the others how many candidates it appended
+    auto ragged = [&](uint32_t t) {
+      if (warp == 0) {
+        const Tile tile = ws.tiles[t];
+        const uint32_t flags = ragged_mask<MODE>(a, tile, L, lane, in, out);
+        const uint32_t count = __reduce_add_sync(kFull, (uint32_t)__popc(flags));
+        ragged_emit<MODE>(ws, sh, tile, flags, slot0 + cur, lane, lt, in, out);
+        if (lane == 0) sh.cursor = count;
+      }
+      __syncthreads();
+      cur += sh.cursor;
+      __syncthreads();
+    };
+    if (head) ragged(a0);
     const uint32_t nfull = f1 > f0 ? f1 - f0 : 0;
     const uint32_t nchunks = (nfull + kStageTiles - 1) / kStageTiles;
     const uint32_t e0 = nfull ? ws.tiles[f0].start : 0;   // first element of the full tiles (multiple of kWarpTile)
@@ -540,28 +593,38 @@ __device__ void stream_tiles_tma(const Workspace& ws, const SelArgs& a, const ui
     uint32_t pc = 0, issued = 0;                          // thread 0: next chunk to ask for, chunks asked for
     if (threadIdx.x == 0) {
       pc = next_live(0);
-      for (; issued < (uint32_t)R::kStages && pc < nchunks; ++issued, pc = next_live(pc + 1)) issue(pc, uses + issued);
+      for (; issued < (uint32_t)R::kStages - 1 && pc < nchunks; ++issued, pc = next_live(pc + 1))
+        issue(pc, uses + issued);
     }
     uint32_t done = 0;
     for (uint32_t c = next_live(0); c < nchunks; c = next_live(c + 1), ++done) {
       const uint32_t use = uses + done, st = use % R::kStages;
-      if (!mbar_wait(full + st, (use / R::kStages) & 1u)) *s_dead = 1;
+      const bool landed = mbar_wait(full + st, (use / R::kStages) & 1u);
+      if (!landed) *s_dead = 1;
       const uint32_t tl = c * kStageTiles + warp;          // this warp's tile among the full ones
-      if (tl < nfull && !*s_dead) {
-        const float* su = ring + (size_t)st * (R::kStageBytes / 4) + warp * kWarpTile;
-        finish_full_tile_smem<MODE>(ws, a, sh, e0 + tl * kWarpTile, su, su + kStageFloats, L, slot0, lane, out);
-      }
-      __syncthreads();                                     // every warp is done reading this stage
+      const float* su = ring + (size_t)st * (R::kStageBytes / 4) + warp * kWarpTile;
+      uint32_t mask = 0;
+      if (tl < nfull && landed) mask = tile_mask_smem<MODE>(a, e0 + tl * kWarpTile, su, su + kStageFloats, L, lane, out);
+      const uint32_t count = __reduce_add_sync(kFull, (uint32_t)__popc(mask));
+      if (lane == 0) sh.wcnt[use & 1][warp] = count;
+      __syncthreads();   // the counts of this round are known, and every warp has left the stage of the round before
       if (*s_dead) break;
-      if (threadIdx.x == 0 && pc < nchunks) {
+      if (threadIdx.x == 0 && pc < nchunks) {              // into the stage of the round before
         issue(pc, uses + issued);
         ++issued;
         pc = next_live(pc + 1);
       }
+      uint32_t total;
+      const uint32_t base = slot0 + cur + round_offset(sh.wcnt[use & 1], warp, total);
+      cur += total;
+      tile_emit(ws, sh, e0 + tl * kWarpTile, mask, base, lane, [&](uint32_t off) {
+        return combine<MODE>(su[off], MODE != kPull ? su[kStageFloats + off] : 0.f, a.m, a.lr);
+      });
     }
     if (*s_dead) break;
     uses += done;
-    __syncthreads();
+    __syncthreads();   // every warp has left the last stage (the next layer's first copies go anywhere in the ring)
+    if (tail) ragged(a1 - 1);
     flush_hist(sh.hist, ws.hist1 + (size_t)s * kBins1);
     __syncthreads();
   }
@@ -577,7 +640,7 @@ __device__ void stream_tiles_tma(const Workspace& ws, const SelArgs& a, const ui
     __syncthreads();
   }
   if (threadIdx.x == 0) {
-    ws.part_cands[cta] = sh.cursor;
+    ws.part_cands[cta] = cur;
     ws.part_slot0[cta] = slot0;
   }
 }
@@ -720,46 +783,47 @@ __device__ bool worker_barrier(uint32_t* sync, uint32_t W, int* status, int* s_o
 
 // ---- finalize -------------------------------------------------------------------
 // The candidates are numbered flat over the parts: part p holds part_cands[p] of them in
-// consecutive slots from part_slot0[p] on, tile after tile (the tiles of a part in the
-// order its warps happened to finish them, each tile's candidates in index order).
-// Every phase below is one flat loop over that numbering; the layer and the tile of a
-// candidate follow from its index.
+// consecutive slots from part_slot0[p] on.  Parts follow one another in index order and every
+// part lists its candidates in index order, so the flat numbering is the index order of all
+// candidates.  Every thread owns a run of consecutive flat candidates (kept in registers when
+// they are few) for all phases:
+//   levels 2 and 3   histograms of the next 10 + 10 key bits among the candidates that share the
+//                    bits fixed so far  ->  exact k-th largest key T and tie quota r per layer
+//   count            (key > T, key == T) per thread, prefix sums inside the CTA, totals per CTA
+//   emit             a candidate's rank among the selected ones of its layer follows from the
+//                    prefix sums (layers are consecutive in the flat order and layer s selects
+//                    exactly k_s entries)  ->  packet in index order, state updates
+// With one layer every CTA works out the picks itself from the shared histograms, which leaves
+// three grid-wide barriers; with several layers the picks are spread over the CTAs.
 constexpr int kSegCap = 1024;  // layers whose tables fit in shared memory; more fall back to global reads
 constexpr int kBatch = 8;       // independent loads a thread issues before using any (latency-bound loops)
 
 struct FinalizeShared {
-  StreamShared stream;                 // only used when the guess failed and the passes are redone here
+  StreamShared stream;                 // redo of the passes (guess failed); its histogram also serves levels 2 and 3
   unsigned long long warp_scan[kWarps];
   uint32_t res[2];
   int ok;
   uint32_t pre_cands[kMaxGrid + 1];    // exclusive prefix of part_cands
   uint32_t slot0[kMaxGrid];            // first slot of each part
-  uint2 base[kMaxWorkers];             // exclusive prefix of the scanning CTAs' (gt, eq) totals
-  uint32_t seg_off[kSegCap + 1];       // first element of each layer, and n
-  uint32_t seg_tile0[kSegCap];         // first tile of each layer
-  uint32_t seg_a[kSegCap];             // per-layer parameter of the current phase (prefix, or T)
-  uint32_t seg_b[kSegCap];             // second one (r)
-  uint2 seg_start[kSegCap];            // (gt, eq) counted before the layer's first tile
 };
-
-struct SegView {  // per-layer tables, in shared memory when they fit
-  const uint32_t* off;
-  const uint32_t* tile0;
-  uint32_t S;
-};
+// Per-layer tables of finalize live in dynamic shared memory, sized by the number of layers S (up
+// to kSegCap layers; with more, the kernel reads the tables from global memory and needs none):
+//   uint2 seg_start[S]   (key > T, key == T) candidates of all earlier layers
+//   u32 seg_off[S + 1]   first element of each layer, and n
+//   u32 seg_a[S]         per-layer parameter of the current phase (prefix, or T)
+//   u32 seg_b[S]         second one (r)
+__host__ __device__ inline uint32_t finalize_dyn_bytes(uint32_t S) {
+  return S <= (uint32_t)kSegCap ? 20u * S + 8u : 0u;
+}
 
 // layer that holds element i: last s with off[s] <= i
-__device__ __forceinline__ uint32_t seg_of(const SegView& v, uint32_t i) {
-  uint32_t lo = 0, hi = v.S - 1;
+__device__ __forceinline__ uint32_t seg_of(const uint32_t* off, uint32_t S, uint32_t i) {
+  uint32_t lo = 0, hi = S - 1;
   while (lo < hi) {
     const uint32_t mid = (lo + hi + 1) >> 1;
-    if (v.off[mid] <= i) lo = mid; else hi = mid - 1;
+    if (off[mid] <= i) lo = mid; else hi = mid - 1;
   }
   return lo;
-}
-// tiles of a layer are cut at the multiples of kWarpTile of the global index
-__device__ __forceinline__ uint32_t tile_of(const SegView& v, uint32_t seg, uint32_t i) {
-  return v.tile0[seg] + (i / kWarpTile - v.off[seg] / kWarpTile);
 }
 // slot of flat candidate p: last part with pre[part] <= p
 __device__ __forceinline__ uint32_t slot_of(const FinalizeShared& sh, uint32_t parts, uint32_t p, uint32_t* part_out) {
@@ -772,8 +836,8 @@ __device__ __forceinline__ uint32_t slot_of(const FinalizeShared& sh, uint32_t p
   return sh.slot0[lo] + (p - sh.pre_cands[lo]);
 }
 
-// Walks the flat numbering: a thread (or a lane) owns consecutive flat candidates, finds
-// the first one by binary search and then only steps.
+// Walks the flat numbering: a thread owns consecutive flat candidates, finds the first one by
+// binary search and then only steps.
 struct Cursor {
   uint32_t part, slot, left;   // part of the current candidate, its slot, candidates left in that part (>= 1 if valid)
 };
@@ -783,12 +847,12 @@ __device__ __forceinline__ Cursor cursor_at(const FinalizeShared& sh, uint32_t p
   c.left = sh.pre_cands[c.part + 1] - p;
   return c;
 }
-// advance by n candidates; the caller never advances past the last candidate + 1
+// advance by n candidates; the caller never dereferences a cursor that ran past the last candidate
 __device__ __forceinline__ void cursor_advance(const FinalizeShared& sh, uint32_t parts, Cursor& c, uint32_t n) {
   while (n >= c.left) {
     n -= c.left;
     do { ++c.part; } while (c.part < parts && sh.pre_cands[c.part + 1] == sh.pre_cands[c.part]);
-    if (c.part >= parts) { c.left = 0xFFFFFFFFu; c.slot = 0; return; }   // ran off the end: never dereferenced
+    if (c.part >= parts) { c.left = 0xFFFFFFFFu; c.slot = 0; return; }   // ran off the end
     c.slot = sh.slot0[c.part];
     c.left = sh.pre_cands[c.part + 1] - sh.pre_cands[c.part];
   }
@@ -796,14 +860,16 @@ __device__ __forceinline__ void cursor_advance(const FinalizeShared& sh, uint32_
   c.left -= n;
 }
 
+#ifndef DGS_FINALIZE_REGS
+#define DGS_FINALIZE_REGS 96
+#endif
 template <int MODE>
-__global__ void __maxnreg__(96) k_finalize(Workspace ws, SelArgs a) {
+__global__ void __maxnreg__(DGS_FINALIZE_REGS) k_finalize(Workspace ws, SelArgs a) {
   __shared__ FinalizeShared sh;
+  extern __shared__ __align__(16) unsigned char fin_dyn[];   // finalize_dyn_bytes(S) bytes
 
   constexpr int PM = MODE == kPull ? 1 : 0;
   const uint32_t cta = blockIdx.x, W = gridDim.x, S = ws.num_segs;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t lt = lanemask_lt();
   const uint32_t gthread = cta * kThreads + threadIdx.x, nthreads = W * kThreads;
 
   // pointers are read once, before anything may exchange them
@@ -818,21 +884,22 @@ __global__ void __maxnreg__(96) k_finalize(Workspace ws, SelArgs a) {
 
   // layer tables
   const bool seg_smem = S <= (uint32_t)kSegCap;
-  if (seg_smem) {
-    for (uint32_t s = threadIdx.x; s <= S; s += kThreads) sh.seg_off[s] = ws.seg_off[s];
-    for (uint32_t s = threadIdx.x; s < S; s += kThreads) sh.seg_tile0[s] = ws.segs[s].tile_begin;
-  }
-  SegView sv;
-  sv.off = seg_smem ? sh.seg_off : ws.seg_off;
-  sv.tile0 = seg_smem ? sh.seg_tile0 : ws.seg_tile0;
-  sv.S = S;
+  uint2* const sm_seg_start = reinterpret_cast<uint2*>(fin_dyn);
+  uint32_t* const sm_seg_off = reinterpret_cast<uint32_t*>(fin_dyn + 8u * S);
+  uint32_t* const sm_seg_a = sm_seg_off + S + 1;
+  uint32_t* const sm_seg_b = sm_seg_a + S;
+  if (seg_smem)
+    for (uint32_t s = threadIdx.x; s <= S; s += kThreads) sm_seg_off[s] = ws.seg_off[s];
+  const uint32_t* const seg_off = seg_smem ? sm_seg_off : ws.seg_off;
   __syncthreads();
 
   // flat numbering of the candidates, and this thread's own candidates
   uint32_t parts = 0, C = 0, per_thread = 0, my_lo = 0, my_hi = 0;
   constexpr int kKeep = 8;            // candidates a thread keeps in registers between the phases
-  uint32_t rkey[kKeep], ridx[kKeep];  // valid when per_thread <= kKeep
+  float rraw[kKeep];
+  uint32_t ridx[kKeep];               // valid when per_thread <= kKeep
   uint32_t bar_target = 0;
+  uint32_t one_prefix = 0, one_krem = 0;   // S == 1: the layer's selection state, the same in every thread of the grid
   bool redo = false;
   for (int attempt = 0; attempt < 2; ++attempt) {
     if (redo) {
@@ -892,35 +959,38 @@ __global__ void __maxnreg__(96) k_finalize(Workspace ws, SelArgs a) {
     my_hi = min(C, my_lo + per_thread);
     if (per_thread <= (uint32_t)kKeep && my_lo < my_hi) {
       Cursor cur = cursor_at(sh, parts, my_lo);
-      float raw[kKeep];
 #pragma unroll
       for (int u = 0; u < kKeep; ++u) {
-        raw[u] = 0.f;
+        rraw[u] = 0.f;
         ridx[u] = 0;
         if (my_lo + u < my_hi) {
-          raw[u] = __ldcg(ws.cand_val + cur.slot);
+          rraw[u] = __ldcg(ws.cand_val + cur.slot);
           ridx[u] = __ldcg(ws.cand_idx + cur.slot);
           cursor_advance(sh, parts, cur, 1);
         }
       }
-#pragma unroll
-      for (int u = 0; u < kKeep; ++u) rkey[u] = key_of(raw[u]);
     }
-    // level 1: pick the bin of the k-th largest among the candidates; check the guess
-    for (uint32_t s = cta; s < S; s += W) {
+    // level 1: the bin of the k-th largest among the candidates; checks the guess, suggests the next one
+    bool failed = false;
+    const bool everyone_picks = S == 1;   // one layer: every CTA reads the histogram itself, no barrier needed
+    for (uint32_t s = everyone_picks ? 0 : cta; s < S; s += everyone_picks ? 1 : W) {
       uint32_t bin, krem;
       uint32_t* h = ws.hist1 + (size_t)s * kBins1;
       const uint32_t k = ws.segs[s].k[PM];
       const uint32_t total = block_pick<kBins1>(h, k, bin, krem, sh.warp_scan, sh.res);
+      const bool owner = !everyone_picks || cta == 0;
       if (total < k) {
-        if (threadIdx.x == 0) atomicOr(ws.sync + kFail, 1u);
+        failed = true;
+        if (owner && threadIdx.x == 0) atomicOr(ws.sync + kFail, 1u);
       } else {
-        if (threadIdx.x == 0) {
+        one_prefix = bin;
+        one_krem = krem;
+        if (owner && threadIdx.x == 0) {
           ws.sel[s].prefix = bin;
           ws.sel[s].krem = krem;
           atomicAdd(ws.stats + 2, (unsigned long long)total);
         }
-        if (a.speculate) {
+        if (owner && a.speculate) {
           // bound suggested for a later selection on this layer
           const uint32_t want = max(k * kSpecFactor, k + kSpecSlack);
           uint32_t lbin, lrem;
@@ -942,114 +1012,37 @@ __global__ void __maxnreg__(96) k_finalize(Workspace ws, SelArgs a) {
           if (threadIdx.x == 0) a.L_next[s] = flood ? 0xFFFFFFFFu : lbin << 20;
         }
       }
-      __syncthreads();
-      for (int b = threadIdx.x; b < kBins1; b += kThreads) h[b] = 0;
+      if (!everyone_picks) {   // the histogram has served; with one layer the others may still be reading it
+        __syncthreads();
+        for (int b = threadIdx.x; b < kBins1; b += kThreads) h[b] = 0;
+      }
     }
-    if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
-    if (redo || ld_volatile(ws.sync + kFail) == 0) break;
-    redo = true;
+    if (everyone_picks) {
+      if (!failed || redo) break;
+      // every CTA has seen the same histogram and comes here: clear it once all have read it, then redo
+      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+      if (cta == 0)
+        for (int b = threadIdx.x; b < kBins1; b += kThreads) ws.hist1[b] = 0;
+      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+      redo = true;
+    } else {
+      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+      if (redo || ld_volatile(ws.sync + kFail) == 0) break;
+      redo = true;
+    }
   }
 
-  // ---- levels 2 and 3 ----------------------------------------------------------------
-#pragma unroll 1
-  for (int level = 2; level <= 3; ++level) {
-    uint32_t* hist = level == 2 ? ws.hist2 : ws.hist3;
-    const int B = level == 2 ? kBins2 : kBins3;   // both 1024
-    const int SH = level == 2 ? 20 : 10;
-    if (seg_smem) {
-      for (uint32_t s = threadIdx.x; s < S; s += kThreads) sh.seg_a[s] = __ldcg(&ws.sel[s].prefix);
-      __syncthreads();
-    }
-    if (S == 1) {
-      for (int b = threadIdx.x; b < B; b += kThreads) sh.stream.hist[b] = 0;
-      __syncthreads();
-    }
-    auto add_level = [&](uint32_t key, uint32_t idx) {
-      const uint32_t seg = S > 1 ? seg_of(sv, idx) : 0;
-      const uint32_t prefix = seg_smem ? sh.seg_a[seg] : __ldcg(&ws.sel[seg].prefix);
-      if ((key >> SH) == prefix) {
-        const uint32_t digit = (key >> (SH - 10)) & 1023u;
-        if (S == 1) atomicAdd(sh.stream.hist + digit, 1u);       // one layer: CTA-private histogram first
-        else atomicAdd(hist + (size_t)seg * B + digit, 1u);
-      }
-    };
+  // visits this thread's candidates in flat order: fn(value, index)
+  auto each_own = [&](auto fn) {
     if (per_thread <= (uint32_t)kKeep) {
 #pragma unroll
       for (int u = 0; u < kKeep; ++u)
-        if (my_lo + u < my_hi) add_level(rkey[u], ridx[u]);
+        if (my_lo + u < my_hi) fn(rraw[u], ridx[u]);
     } else if (my_lo < my_hi) {
       Cursor cur = cursor_at(sh, parts, my_lo);
       for (uint32_t p = my_lo; p < my_hi; p += kBatch) {
         // all loads of the batch are issued before any loaded value is touched (a use right
         // after its load would make the loads wait for one another)
-        float raw[kBatch];
-        uint32_t idx[kBatch];
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-          raw[u] = 0.f;
-          idx[u] = 0;
-          if (p + u < my_hi) {
-            raw[u] = __ldcg(ws.cand_val + cur.slot);
-            if (S > 1) idx[u] = __ldcg(ws.cand_idx + cur.slot);
-            cursor_advance(sh, parts, cur, 1);
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u)
-          if (p + u < my_hi) add_level(key_of(raw[u]), idx[u]);
-      }
-    }
-    if (S == 1) {
-      __syncthreads();
-      for (int b = threadIdx.x; b < B; b += kThreads) {
-        const uint32_t v = sh.stream.hist[b];
-        if (v) atomicAdd(hist + b, v);
-      }
-    }
-    if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
-    for (uint32_t s = cta; s < S; s += W) {
-      uint32_t bin, krem;
-      uint32_t* h = hist + (size_t)s * B;
-      block_pick<kBins2>(h, __ldcg(&ws.sel[s].krem), bin, krem, sh.warp_scan, sh.res);
-      if (threadIdx.x == 0) {
-        const uint32_t pre = (__ldcg(&ws.sel[s].prefix) << 10) | bin;
-        ws.sel[s].prefix = pre;
-        ws.sel[s].krem = krem;
-        if (level == 3) {
-          ws.sel[s].T = pre;   // all 31 key bits are fixed now
-          ws.sel[s].r = krem;
-        }
-      }
-      for (int b = threadIdx.x; b < B; b += kThreads) h[b] = 0;
-    }
-    if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
-  }
-
-  // ---- count: per tile, how many candidates have key > T and key == T ----------------
-  // (tile_sel is all zero on entry: the scan below clears what it reads)
-  if (seg_smem) {
-    for (uint32_t s = threadIdx.x; s < S; s += kThreads) {
-      sh.seg_a[s] = __ldcg(&ws.sel[s].T);
-      sh.seg_b[s] = __ldcg(&ws.sel[s].r);
-    }
-    __syncthreads();
-  }
-  {
-    auto add_count = [&](uint32_t key, uint32_t idx) {
-      const uint32_t seg = S > 1 ? seg_of(sv, idx) : 0;
-      const uint32_t T = seg_smem ? sh.seg_a[seg] : __ldcg(&ws.sel[seg].T);
-      if (key >= T) {
-        uint2* c = ws.tile_sel + tile_of(sv, seg, idx);
-        atomicAdd(key > T ? &c->x : &c->y, 1u);
-      }
-    };
-    if (per_thread <= (uint32_t)kKeep) {
-#pragma unroll
-      for (int u = 0; u < kKeep; ++u)
-        if (my_lo + u < my_hi) add_count(rkey[u], ridx[u]);
-    } else if (my_lo < my_hi) {
-      Cursor cur = cursor_at(sh, parts, my_lo);
-      for (uint32_t p = my_lo; p < my_hi; p += kBatch) {
         float raw[kBatch];
         uint32_t idx[kBatch];
 #pragma unroll
@@ -1064,170 +1057,161 @@ __global__ void __maxnreg__(96) k_finalize(Workspace ws, SelArgs a) {
         }
 #pragma unroll
         for (int u = 0; u < kBatch; ++u)
-          if (p + u < my_hi) add_count(key_of(raw[u]), idx[u]);
+          if (p + u < my_hi) fn(raw[u], idx[u]);
       }
     }
-  }
-  if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+  };
 
-  // ---- scan over the tiles in index order: CTA c owns tiles [c*chunk, (c+1)*chunk) ----
-  const uint32_t chunk_tiles = (ws.num_tiles + W - 1) / W;
-  {
-    const uint32_t t0 = min(ws.num_tiles, cta * chunk_tiles), t1 = min(ws.num_tiles, t0 + chunk_tiles);
-    unsigned long long carry = 0;
-    for (uint32_t base0 = t0; base0 < t1; base0 += kThreads * kBatch) {
-      unsigned long long v[kBatch];
-#pragma unroll
-      for (int u = 0; u < kBatch; ++u) {
-        const uint32_t t = base0 + u * kThreads + threadIdx.x;
-        v[u] = 0;
-        if (t < t1) {
-          const uint2 c = __ldcg(ws.tile_sel + t);
-          v[u] = ((unsigned long long)c.x << 32) | c.y;
-        }
+  // ---- levels 2 and 3 ----------------------------------------------------------------
+#pragma unroll 1
+  for (int level = 2; level <= 3; ++level) {
+    uint32_t* hist = level == 2 ? ws.hist2 : ws.hist3;
+    constexpr int B = kBins2;   // both levels have 1024 bins
+    const int SH = level == 2 ? 20 : 10;
+    if (S == 1) {
+      for (int b = threadIdx.x; b < B; b += kThreads) sh.stream.hist[b] = 0;
+      __syncthreads();
+      each_own([&](float v, uint32_t) {
+        const uint32_t key = key_of(v);
+        if ((key >> SH) == one_prefix) atomicAdd(sh.stream.hist + ((key >> (SH - 10)) & 1023u), 1u);
+      });
+      __syncthreads();
+      for (int b = threadIdx.x; b < B; b += kThreads) {
+        const uint32_t v = sh.stream.hist[b];
+        if (v) atomicAdd(hist + b, v);
       }
-#pragma unroll
-      for (int u = 0; u < kBatch; ++u) {
-        if (base0 + u * kThreads < t1) {   // CTA-uniform
-          const uint32_t t = base0 + u * kThreads + threadIdx.x;
-          if (v[u]) ws.tile_sel[t] = make_uint2(0, 0);
-          unsigned long long total;
-          const unsigned long long ex = block_excl_scan(v[u], sh.warp_scan, total) + carry;
-          if (t < t1) ws.tile_pre[t] = make_uint2((uint32_t)(ex >> 32), (uint32_t)ex);
-          carry += total;
+      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+      // the histogram of the level before has been read by everyone
+      if (cta == 0) {
+        uint32_t* old = level == 2 ? ws.hist1 : ws.hist2;
+        for (int b = threadIdx.x; b < (level == 2 ? kBins1 : kBins2); b += kThreads) old[b] = 0;
+      }
+      uint32_t bin, krem;
+      block_pick<B>(hist, one_krem, bin, krem, sh.warp_scan, sh.res);
+      one_prefix = (one_prefix << 10) | bin;
+      one_krem = krem;
+    } else {
+      if (seg_smem) {
+        for (uint32_t s = threadIdx.x; s < S; s += kThreads) sm_seg_a[s] = __ldcg(&ws.sel[s].prefix);
+        __syncthreads();
+      }
+      each_own([&](float v, uint32_t idx) {
+        const uint32_t key = key_of(v);
+        const uint32_t seg = seg_of(seg_off, S, idx);
+        const uint32_t prefix = seg_smem ? sm_seg_a[seg] : __ldcg(&ws.sel[seg].prefix);
+        if ((key >> SH) == prefix) atomicAdd(hist + (size_t)seg * B + ((key >> (SH - 10)) & 1023u), 1u);
+      });
+      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+      for (uint32_t s = cta; s < S; s += W) {
+        uint32_t bin, krem;
+        uint32_t* h = hist + (size_t)s * B;
+        block_pick<B>(h, __ldcg(&ws.sel[s].krem), bin, krem, sh.warp_scan, sh.res);
+        if (threadIdx.x == 0) {
+          const uint32_t pre = (__ldcg(&ws.sel[s].prefix) << 10) | bin;
+          ws.sel[s].prefix = pre;
+          ws.sel[s].krem = krem;
+          if (level == 3) {
+            ws.sel[s].T = pre;   // all 31 key bits are fixed now
+            ws.sel[s].r = krem;
+            ws.sel[s].neq = __ldcg(h + bin);
+          }
         }
+        __syncthreads();
+        for (int b = threadIdx.x; b < B; b += kThreads) h[b] = 0;
+      }
+      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+    }
+  }
+
+  // ---- count: (key > T, key == T) among this thread's candidates, prefix inside the CTA -------
+  if (S > 1) {
+    if (seg_smem) {
+      for (uint32_t s = threadIdx.x; s < S; s += kThreads) {
+        sm_seg_a[s] = __ldcg(&ws.sel[s].T);
+        sm_seg_b[s] = __ldcg(&ws.sel[s].r);
       }
     }
-    if (threadIdx.x == 0) ws.cta_tot[cta] = make_uint2((uint32_t)(carry >> 32), (uint32_t)carry);
+    if (cta == 0) {
+      // (key > T, key == T) candidates of all earlier layers: layer s selects k_s - r_s of the first kind
+      unsigned long long carry = 0;
+      for (uint32_t base = 0; base < S; base += kThreads) {
+        const uint32_t s = base + threadIdx.x;
+        unsigned long long v = 0;
+        if (s < S) v = ((unsigned long long)(ws.segs[s].k[PM] - __ldcg(&ws.sel[s].r)) << 32) | __ldcg(&ws.sel[s].neq);
+        unsigned long long total;
+        const unsigned long long ex = block_excl_scan(v, sh.warp_scan, total) + carry;
+        if (s < S) ws.seg_start[s] = make_uint2((uint32_t)(ex >> 32), (uint32_t)ex);
+        carry += total;
+      }
+    }
+    __syncthreads();
   }
+  unsigned long long mine = 0;   // (gt << 32) | eq
+  each_own([&](float v, uint32_t idx) {
+    const uint32_t key = key_of(v);
+    uint32_t T = one_prefix;
+    if (S > 1) {
+      const uint32_t seg = seg_of(seg_off, S, idx);
+      T = seg_smem ? sm_seg_a[seg] : __ldcg(&ws.sel[seg].T);
+    }
+    if (key > T) mine += 1ull << 32;
+    else if (key == T) mine += 1ull;
+  });
+  unsigned long long cta_total;
+  unsigned long long before = block_excl_scan(mine, sh.warp_scan, cta_total);
+  if (threadIdx.x == 0) ws.cta_tot[cta] = make_uint2((uint32_t)(cta_total >> 32), (uint32_t)cta_total);
   if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+  if (S == 1 && cta == 0)
+    for (int b = threadIdx.x; b < kBins3; b += kThreads) ws.hist3[b] = 0;
 
   // ---- emit: packet in index order, and the state updates that depend on selection ----
   {
-    unsigned long long carry = 0;  // exclusive prefix of the CTAs' totals (W <= kMaxWorkers)
-    for (uint32_t base = 0; base < W; base += kThreads) {
-      const uint32_t c = base + threadIdx.x;
-      unsigned long long v = 0;
-      if (c < W) {
-        const uint2 q = __ldcg(ws.cta_tot + c);
-        v = ((unsigned long long)q.x << 32) | q.y;
-      }
-      unsigned long long total;
-      const unsigned long long ex = block_excl_scan(v, sh.warp_scan, total) + carry;
-      if (c < W) sh.base[c] = make_uint2((uint32_t)(ex >> 32), (uint32_t)ex);
-      carry += total;
+    unsigned long long lower = 0;   // totals of the CTAs before this one (W <= kMaxWorkers)
+    for (uint32_t c = threadIdx.x; c < cta; c += kThreads) {
+      const uint2 q = __ldcg(ws.cta_tot + c);
+      lower += ((unsigned long long)q.x << 32) | q.y;
     }
-    __syncthreads();
-    // (gt, eq) counted before tile t, over all layers
-    auto before_tile = [&](uint32_t t) {
-      const uint2 pre = __ldcg(ws.tile_pre + t), b = sh.base[t / chunk_tiles];
-      return make_uint2(b.x + pre.x, b.y + pre.y);
-    };
-    if (seg_smem) {
-      for (uint32_t s = threadIdx.x; s < S; s += kThreads) sh.seg_start[s] = before_tile(sh.seg_tile0[s]);
+    unsigned long long lower_total;
+    block_excl_scan(lower, sh.warp_scan, lower_total);
+    before += lower_total;
+    if (S > 1 && seg_smem) {
+      for (uint32_t s = threadIdx.x; s < S; s += kThreads) sm_seg_start[s] = __ldcg(ws.seg_start + s);
       __syncthreads();
     }
-    // every warp owns a run of consecutive flat candidates, 32 per step
-    const uint32_t gwarp = cta * kWarps + warp, nwarps = W * kWarps;
-    const uint32_t per_warp = ((C + nwarps - 1) / nwarps + 31) / 32 * 32;
-    const uint32_t w_lo = min(C, gwarp * per_warp), w_hi = min(C, w_lo + per_warp);
-    Cursor cur;
-    cur.part = 0; cur.slot = 0; cur.left = 0xFFFFFFFFu;
-    if (w_lo + lane < w_hi) cur = cursor_at(sh, parts, w_lo + lane);
-    // counts carried from the previous step for the tile its last lane was in
-    uint32_t carry_gt = 0, carry_eq = 0, carry_tile = 0xFFFFFFFFu, carry_part = 0xFFFFFFFFu;
-    for (uint32_t c0 = w_lo; c0 < w_hi; c0 += 32) {
-      const uint32_t p = c0 + lane;
-      const bool valid = p < w_hi;
-      uint32_t part = 0xFFFFFFFEu, idx = 0, key = 0, seg = 0, tile = 0xFFFFFFFFu, T = 0, r = 0;
-      float val = 0.f;
-      if (valid) {
-        part = cur.part;
-        idx = __ldcg(ws.cand_idx + cur.slot);
-        val = __ldcg(ws.cand_val + cur.slot);
-        key = key_of(val);
-        seg = S > 1 ? seg_of(sv, idx) : 0;
-        tile = tile_of(sv, seg, idx);
-        T = seg_smem ? sh.seg_a[seg] : __ldcg(&ws.sel[seg].T);
-        r = seg_smem ? sh.seg_b[seg] : __ldcg(&ws.sel[seg].r);
-        if (p + 32 < w_hi) cursor_advance(sh, parts, cur, 32);
+    uint32_t gt_before = (uint32_t)(before >> 32), eq_before = (uint32_t)before;   // over all layers
+    each_own([&](float val, uint32_t idx) {
+      const uint32_t key = key_of(val);
+      uint32_t T = one_prefix, r = one_krem, pkt_off = 0;
+      uint2 start = make_uint2(0, 0);
+      if (S > 1) {
+        const uint32_t seg = seg_of(seg_off, S, idx);
+        T = seg_smem ? sm_seg_a[seg] : __ldcg(&ws.sel[seg].T);
+        r = seg_smem ? sm_seg_b[seg] : __ldcg(&ws.sel[seg].r);
+        start = seg_smem ? sm_seg_start[seg] : __ldcg(ws.seg_start + seg);
+        pkt_off = ws.segs[seg].pkt_off[PM];
       }
-      const bool is_gt = valid && key > T, is_eq = valid && key == T;
-      const uint32_t bgt = __ballot_sync(kFull, is_gt), beq = __ballot_sync(kFull, is_eq);
-      // the candidates of one tile are consecutive: a lane starts a tile if its left neighbour is in another one
-      const uint32_t left = __shfl_up_sync(kFull, tile, 1);
-      const uint32_t heads = __ballot_sync(kFull, lane == 0 || left != tile);
-      const int head = 31 - __clz(heads & (lt | (1u << lane)));       // first lane of my tile in this step
-      const uint32_t mine = lt & ~((1u << head) - 1u);                  // lanes of my tile before me
-      // what the tile of lane 0 holds in earlier slots
-      const uint32_t tile0 = __shfl_sync(kFull, tile, 0), part0 = __shfl_sync(kFull, part, 0);
-      uint32_t pre_gt = 0, pre_eq = 0;
-      if (c0 != w_lo) {
-        if (carry_tile == tile0 && carry_part == part0) {
-          pre_gt = carry_gt;
-          pre_eq = carry_eq;
+      const bool is_gt = key > T, is_eq = key == T;
+      const uint32_t eq_in_layer = eq_before - start.y;
+      const bool sel = is_gt || (is_eq && eq_in_layer < r);
+      if (sel) {
+        const uint32_t pos = pkt_off + (gt_before - start.x) + min(eq_in_layer, r);
+        if (pos < a.pkt_count) {
+          a.pkt_idx[pos] = idx;
+          a.pkt_val[pos] = val;
+        } else {
+          atomicMin(ws.status, -1000 - MODE);
+        }
+        if (MODE == kPushResidual) out[idx] = 0.f;       // Algorithm 1: the sent part leaves v
+        if (MODE == kPull) {
+          a.D[idx] = 0.f;                                // Eq. 6b: v_k <- v_k + G
+          if (a.theta_local) a.theta_local[idx] = __fadd_rn(a.theta_local[idx], val);  // Eq. 5
         }
       } else {
-        // first step of this warp: the tile may have begun in slots that belong to the previous warp
-        const uint32_t T0 = __shfl_sync(kFull, T, 0), seg0 = __shfl_sync(kFull, seg, 0);
-        const uint32_t first = sh.pre_cands[part0];                     // flat number of the part's first candidate
-        uint32_t back = c0;
-        while (back > first) {                                          // warp-uniform
-          const uint32_t lo = back - min(back - first, 32u);
-          const uint32_t pp = lo + lane;
-          bool same = false;
-          uint32_t k2 = 0;
-          if (pp < back) {
-            const uint32_t slot = sh.slot0[part0] + (pp - first);
-            const uint32_t i2 = __ldcg(ws.cand_idx + slot);
-            const uint32_t s2 = S > 1 ? seg_of(sv, i2) : 0;
-            same = s2 == seg0 && tile_of(sv, s2, i2) == tile0;
-            k2 = key_of(__ldcg(ws.cand_val + slot));
-          }
-          const uint32_t bs = __ballot_sync(kFull, same);
-          pre_gt += __popc(__ballot_sync(kFull, same && k2 > T0));
-          pre_eq += __popc(__ballot_sync(kFull, same && k2 == T0));
-          if (bs != __ballot_sync(kFull, pp < back)) break;             // reached another tile
-          back = lo;
-        }
+        if (MODE == kPushSam) out[idx] = __fmul_rn(val, a.inv_m);  // Eq. 12, lower branch
       }
-      if (valid) {
-        const uint2 tb = before_tile(tile);
-        const uint2 s0 = seg_smem ? sh.seg_start[seg] : before_tile(sv.tile0[seg]);
-        uint32_t gt_before = (tb.x - s0.x) + __popc(bgt & mine);
-        uint32_t eq_before = (tb.y - s0.y) + __popc(beq & mine);
-        if (head == 0) {
-          gt_before += pre_gt;
-          eq_before += pre_eq;
-        }
-        const bool sel = is_gt || (is_eq && eq_before < r);
-        if (sel) {
-          const uint32_t pos = ws.segs[seg].pkt_off[PM] + gt_before + min(eq_before, r);
-          if (pos < a.pkt_count) {
-            a.pkt_idx[pos] = idx;
-            a.pkt_val[pos] = val;
-          } else {
-            atomicMin(ws.status, -1000 - MODE);
-          }
-          if (MODE == kPushResidual) out[idx] = 0.f;       // Algorithm 1: the sent part leaves v
-          if (MODE == kPull) {
-            a.D[idx] = 0.f;                                // Eq. 6b: v_k <- v_k + G
-            if (a.theta_local) a.theta_local[idx] = __fadd_rn(a.theta_local[idx], val);  // Eq. 5
-          }
-        } else {
-          if (MODE == kPushSam) out[idx] = __fmul_rn(val, a.inv_m);  // Eq. 12, lower branch
-        }
-      }
-      // carry for the next step: counts of the tile that lane 31 is in (all lanes of a full step are valid)
-      {
-        const int head31 = 31 - __clz(heads);
-        const uint32_t tail_lanes = ~((1u << head31) - 1u);
-        carry_gt = __popc(bgt & tail_lanes) + (head31 == 0 ? pre_gt : 0u);
-        carry_eq = __popc(beq & tail_lanes) + (head31 == 0 ? pre_eq : 0u);
-        carry_tile = __shfl_sync(kFull, tile, 31);
-        carry_part = __shfl_sync(kFull, part, 31);
-      }
-    }
+      gt_before += is_gt ? 1u : 0u;
+      eq_before += is_eq ? 1u : 0u;
+    });
   }
   if (cta == 0 && threadIdx.x == 0) {
     if (MODE != kPull) {  // the spare buffer now holds the worker's velocity
@@ -1300,9 +1284,15 @@ __global__ void __maxnreg__(64) k_stream(Workspace ws, SelArgs a) {
 // bit for bit, and each packet is folded into D_q while the entries it touches are hot
 // instead of being scattered into all N vectors at once.
 //
-constexpr int kCatchGrid = 128;                             // CTAs of k_catch_up
-constexpr uint32_t kCatchWarps = kCatchGrid * (kThreads / 32);
-constexpr int kCatchBatch = 2;                              // entries per lane in flight per packet
+constexpr int kCatchMaxPackets = 64;     // most packets one k_catch_up launch folds in
+constexpr int kCatchCap = 2048;          // entries a CTA of k_catch_up can hold in shared memory
+constexpr int kCatchSlots = 4096;        // slots of its table of distinct indices (power of two, >= 2 * kCatchCap)
+constexpr uint32_t kCatchTarget = 1024;  // entries per CTA the launch aims at
+constexpr int kCatchMaxGrid = 8192;
+#ifndef DGS_CATCH_THREADS
+#define DGS_CATCH_THREADS 256
+#endif
+constexpr int kCatchThreads = DGS_CATCH_THREADS;   // threads per CTA of k_catch_up (>= 2 * kCatchMaxPackets)
 
 struct PacketLog {
   uint32_t* idx;   // [ring][stride], each packet sorted by index
@@ -1310,13 +1300,44 @@ struct PacketLog {
   uint32_t stride; // entries between slots
   uint32_t cap;    // entries per packet
   uint32_t ring;   // slots
+  // The index space is cut once, at the first packet filed, into `ranges` ranges that hold equally
+  // many of that packet's entries (later packets are spread much alike): range g is
+  // [bnd[g], bnd[g+1]), bnd[0] = 0, the last range is open-ended.  pos[slot][g] is the position of
+  // the first entry of the packet in `slot` whose index is >= bnd[g]; pos[slot][ranges] = cap.
+  uint32_t* bnd;   // [ranges]
+  uint32_t* pos;   // [ring][ranges + 1]
+  uint32_t ranges;
 };
 
-// theta -= packet, and a copy of the packet into slot `slot` of the log.
+// The ranges of the log, from the quantiles of the first packet filed (sorted by index).
+__global__ void __launch_bounds__(kThreads) k_log_ranges(const uint32_t* __restrict__ idx, PacketLog lg) {
+  const uint32_t g = blockIdx.x * kThreads + threadIdx.x;
+  if (g < lg.ranges) lg.bnd[g] = g == 0 ? 0u : idx[(uint64_t)g * lg.cap / lg.ranges];
+}
+
+// theta -= packet, and a copy of the packet into slot `slot` of the log: CTAs [0, copy_ctas).
+// The remaining CTAs find where the ranges of the log begin in this packet.
 __global__ void __launch_bounds__(kThreads) k_apply_log(const uint32_t* __restrict__ idx,
                                                         const float* __restrict__ val, uint32_t count,
                                                         float* __restrict__ theta, uint64_t n, int* status,
-                                                        PacketLog lg, uint32_t slot) {
+                                                        PacketLog lg, uint32_t slot, uint32_t copy_ctas) {
+  if (blockIdx.x >= copy_ctas) {
+    const uint32_t g = (blockIdx.x - copy_ctas) * kThreads + threadIdx.x;
+    if (g > lg.ranges) return;
+    uint32_t l = 0;
+    if (g == lg.ranges) {
+      l = count;
+    } else if (g > 0) {
+      const uint32_t key = __ldcg(lg.bnd + g);
+      uint32_t r = count;
+      while (l < r) {
+        const uint32_t mid = (l + r) >> 1;
+        if (__ldg(idx + mid) < key) l = mid + 1; else r = mid;
+      }
+    }
+    lg.pos[(uint64_t)slot * (lg.ranges + 1) + g] = l;
+    return;
+  }
   const uint32_t j = blockIdx.x * kThreads + threadIdx.x;
   if (j >= count) return;
   const uint32_t i = idx[j];
@@ -1330,110 +1351,158 @@ __global__ void __launch_bounds__(kThreads) k_apply_log(const uint32_t* __restri
   theta[i] = __fsub_rn(theta[i], v);
 }
 
-// D -= packets first .. first + count - 1 of the log, in that order (count <= 64).  The index
-// space is cut into kCatchWarps ranges holding equally many entries of the newest packet (the
-// others are spread much alike); a warp owns one range, finds its part of every packet by
-// binary search (packets are sorted), and takes the packets one after the other.  No two
-// warps touch the same entry of D, so no atomics and no block-wide barriers are needed.
-__global__ void __launch_bounds__(kThreads) k_catch_up(PacketLog lg, uint64_t first, uint32_t count,
+// D -= packets first .. first + count - 1 of the log, in that order (count <= kCatchMaxPackets).
+// CTA c owns range c of the log (gridDim.x = ranges); its part of every packet is known from the
+// positions filed with the packet.  It gathers the distinct indices of all those parts in a
+// shared-memory table, loads each D[i] once, subtracts the packets' values from the table in
+// packet order (indices inside one packet are distinct, so a packet is one parallel step) and
+// stores each D[i] once: every D[i] sees the same subtractions in the same order as if the
+// packets had been applied one by one, with one trip to memory instead of one per packet.  No two
+// CTAs touch the same entry of D.  A range with more entries than the table holds (later packets
+// much denser there than the one the ranges were taken from) is taken in several rounds, each over
+// a piece of the range (halved until its entries fit).
+struct CatchShared {
+  uint32_t keys[kCatchSlots];            // index held by a slot, kFull = empty
+  float vals[kCatchSlots];               // running value of D at that index
+  uint16_t ent_slot[kCatchCap];          // slot of each entry (packet-major order), 0xFFFF = index out of range
+  float ent_val[kCatchCap];
+  uint32_t lo[kCatchMaxPackets], hi[kCatchMaxPackets], end[kCatchMaxPackets];   // per packet: piece, end of the range
+  uint32_t pre[kCatchMaxPackets + 1];    // exclusive prefix of hi - lo
+};
+
+__global__ void __launch_bounds__(kCatchThreads) k_catch_up(PacketLog lg, uint64_t first, uint32_t count,
                                                        float* __restrict__ D, uint32_t* __restrict__ blk_max,
                                                        uint64_t n) {
-  const uint32_t lane = threadIdx.x & 31;
-  const uint32_t w = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
-  if (w >= kCatchWarps || count == 0) return;
-  const uint32_t* ref = lg.idx + ((first + count - 1) % lg.ring) * (uint64_t)lg.stride;
-  const uint32_t key_lo = w == 0 ? 0u : __ldcg(ref + (uint64_t)w * lg.cap / kCatchWarps);
-  const uint32_t key_hi = w + 1 == kCatchWarps ? 0xFFFFFFFFu : __ldcg(ref + (uint64_t)(w + 1) * lg.cap / kCatchWarps);
-  // positions of [key_lo, key_hi) in packet `lane` and in packet `lane + 32`
-  uint32_t lo_r[2] = {0, 0}, hi_r[2] = {0, 0};
-  {
-    const uint32_t* a[2];
-    uint32_t l0[2], r0[2], l1[2], r1[2];
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const uint32_t p = lane + 32 * h;
-      a[h] = lg.idx + ((first + min(p, count - 1)) % lg.ring) * (uint64_t)lg.stride;
-      l0[h] = l1[h] = 0;
-      r0[h] = r1[h] = p < count ? lg.cap : 0;
-    }
-    for (uint32_t span = lg.cap; span > 0; span >>= 1) {  // enough halvings for a range of cap entries
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        if (l0[h] < r0[h]) {
-          const uint32_t mid = (l0[h] + r0[h]) >> 1;
-          if (__ldcg(a[h] + mid) < key_lo) l0[h] = mid + 1; else r0[h] = mid;
-        }
-        if (l1[h] < r1[h]) {
-          const uint32_t mid = (l1[h] + r1[h]) >> 1;
-          if (__ldcg(a[h] + mid) < key_hi) l1[h] = mid + 1; else r1[h] = mid;
-        }
-      }
-    }
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      lo_r[h] = l0[h];
-      hi_r[h] = l1[h];
-    }
+  __shared__ CatchShared sh;
+  const uint32_t tid = threadIdx.x, c = blockIdx.x;
+  if (count == 0 || count > (uint32_t)kCatchMaxPackets) return;
+  if (tid < 2 * count) {
+    // thread 2p reads where range c begins in packet p, thread 2p+1 where it ends
+    const uint32_t p = tid >> 1;
+    const uint32_t v = __ldcg(lg.pos + ((first + p) % lg.ring) * (uint64_t)(lg.ranges + 1) + c + (tid & 1u));
+    if (tid & 1u) sh.end[p] = v; else sh.lo[p] = v;
   }
-  uint32_t ci[kCatchBatch], ni[kCatchBatch];
-  float cv[kCatchBatch], nv[kCatchBatch];
-  uint32_t lo = 0, hi = 0, nlo = 0, nhi = 0;
-  const uint32_t* pi = nullptr;
-  const float* pv = nullptr;
-  const uint32_t* npi = nullptr;
-  const float* npv = nullptr;
-  auto fetch = [&](uint32_t p, uint32_t& flo, uint32_t& fhi, const uint32_t*& fpi, const float*& fpv,
-                   uint32_t (&fi)[kCatchBatch], float (&fv)[kCatchBatch]) {
-    const uint32_t a0 = __shfl_sync(0xFFFFFFFFu, lo_r[0], p & 31), a1 = __shfl_sync(0xFFFFFFFFu, lo_r[1], p & 31);
-    const uint32_t b0 = __shfl_sync(0xFFFFFFFFu, hi_r[0], p & 31), b1 = __shfl_sync(0xFFFFFFFFu, hi_r[1], p & 31);
-    flo = p < 32 ? a0 : a1;
-    fhi = p < 32 ? b0 : b1;
-    const uint64_t at = ((first + p) % lg.ring) * (uint64_t)lg.stride;
-    fpi = lg.idx + at;
-    fpv = lg.val + at;
+  const uint32_t range_b = c + 1 == lg.ranges ? (uint32_t)n : __ldcg(lg.bnd + c + 1);   // n < 2^32
+  uint32_t a = c == 0 ? 0u : __ldcg(lg.bnd + c);
+  for (;;) {   // one round per piece [a, b) of the range; everything here is uniform over the CTA
+    for (int s = tid; s < kCatchSlots; s += kCatchThreads) sh.keys[s] = kFull;
+    __syncthreads();
+    if (tid < count) sh.hi[tid] = sh.end[tid];
+    uint32_t b = range_b;
+    uint32_t E;
+    for (;;) {
+      __syncthreads();
+      if (tid < 32) {
+        // exclusive prefix of the pieces' lengths over the packets (two per lane)
+        const uint32_t p0 = tid, p1 = tid + 32;
+        const uint32_t x = p0 < count ? sh.hi[p0] - sh.lo[p0] : 0u, y = p1 < count ? sh.hi[p1] - sh.lo[p1] : 0u;
+        uint32_t ix = x, iy = y;
 #pragma unroll
-    for (int e = 0; e < kCatchBatch; ++e) {
-      const uint32_t j = flo + lane + 32 * e;
-      const bool in = j < fhi;
-      fi[e] = in ? __ldcg(fpi + j) : 0xFFFFFFFFu;
-      fv[e] = in ? __ldcg(fpv + j) : 0.0f;
-    }
-  };
-  fetch(0, lo, hi, pi, pv, ci, cv);
-  for (uint32_t p = 0; p < count; ++p) {
-    if (p + 1 < count) fetch(p + 1, nlo, nhi, npi, npv, ni, nv);
-    for (uint32_t base = lo;;) {
-      float d[kCatchBatch];
-#pragma unroll
-      for (int e = 0; e < kCatchBatch; ++e)
-        if (ci[e] < n) d[e] = __ldcg(D + ci[e]);
-#pragma unroll
-      for (int e = 0; e < kCatchBatch; ++e)
-        if (ci[e] < n) {
-          const float r = __fsub_rn(d[e], cv[e]);
-          __stcg(D + ci[e], r);
-          atomicMax(blk_max + ci[e] / kWarpTile, key_of(r));   // keeps the block's bound an upper bound
+        for (int d = 1; d < 32; d <<= 1) {
+          const uint32_t ox = __shfl_up_sync(kFull, ix, d), oy = __shfl_up_sync(kFull, iy, d);
+          if ((int)tid >= d) {
+            ix += ox;
+            iy += oy;
+          }
         }
-      base += 32 * kCatchBatch;
-      if (base >= hi) break;
-#pragma unroll
-      for (int e = 0; e < kCatchBatch; ++e) {  // a range with more entries than one batch
-        const uint32_t j = base + lane + 32 * e;
-        const bool in = j < hi;
-        ci[e] = in ? __ldcg(pi + j) : 0xFFFFFFFFu;
-        cv[e] = in ? __ldcg(pv + j) : 0.0f;
+        const uint32_t tx = __shfl_sync(kFull, ix, 31), ty = __shfl_sync(kFull, iy, 31);
+        if (p0 < count) sh.pre[p0] = ix - x;
+        if (p1 < count) sh.pre[p1] = tx + iy - y;
+        if (tid == 0) sh.pre[count] = tx + ty;
+      }
+      __syncthreads();
+      E = sh.pre[count];
+      if (E <= (uint32_t)kCatchCap || b - a <= 1) break;   // one index has at most `count` entries
+      b = a + (b - a) / 2;
+      if (tid < count) {
+        const uint32_t* pi = lg.idx + ((first + tid) % lg.ring) * (uint64_t)lg.stride;
+        uint32_t l = sh.lo[tid], r = sh.end[tid];
+        while (l < r) {
+          const uint32_t mid = (l + r) >> 1;
+          if (__ldcg(pi + mid) < b) l = mid + 1; else r = mid;
+        }
+        sh.hi[tid] = l;
       }
     }
-    __syncwarp();  // orders this packet's stores before the next packet's loads within the warp
-    lo = nlo;
-    hi = nhi;
-    pi = npi;
-    pv = npv;
+    if (E > 0 && E <= (uint32_t)kCatchCap) {
+      // gather: entry e (packet-major) -> its index and value; the index gets a slot of the table
+      constexpr int PER = kCatchCap / kCatchThreads;
+      uint32_t ei[PER];
+      float ev[PER];
 #pragma unroll
-    for (int e = 0; e < kCatchBatch; ++e) {
-      ci[e] = ni[e];
-      cv[e] = nv[e];
+      for (int u = 0; u < PER; ++u) {
+        const uint32_t e = tid + u * kCatchThreads;
+        ei[u] = kFull;
+        ev[u] = 0.f;
+        if (e < E) {
+          uint32_t l = 0, r = count - 1;        // last packet p with pre[p] <= e
+          while (l < r) {
+            const uint32_t mid = (l + r + 1) >> 1;
+            if (sh.pre[mid] <= e) l = mid; else r = mid - 1;
+          }
+          const uint64_t at = ((first + l) % lg.ring) * (uint64_t)lg.stride + sh.lo[l] + (e - sh.pre[l]);
+          ei[u] = __ldcg(lg.idx + at);
+          ev[u] = __ldcg(lg.val + at);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < PER; ++u) {
+        const uint32_t e = tid + u * kCatchThreads;
+        if (e < E) {
+          uint32_t slot = 0xFFFFu;
+          const uint32_t i = ei[u];
+          if (i < n) {
+            uint32_t h = (i * 2654435761u) >> 20;   // top 12 bits: kCatchSlots = 4096
+            for (;;) {
+              const uint32_t old = atomicCAS(sh.keys + h, kFull, i);
+              if (old == kFull || old == i) break;
+              h = (h + 1) & (kCatchSlots - 1);
+            }
+            slot = h;
+          }
+          sh.ent_slot[e] = (uint16_t)slot;
+          sh.ent_val[e] = ev[u];
+        }
+      }
+      __syncthreads();
+      // one load of D per distinct index, all in flight together
+      constexpr int SPT = kCatchSlots / kCatchThreads;
+      {
+        uint32_t k[SPT];
+        float d[SPT];
+#pragma unroll
+        for (int u = 0; u < SPT; ++u) {
+          k[u] = sh.keys[tid + u * kCatchThreads];
+          d[u] = 0.f;
+          if (k[u] != kFull) d[u] = __ldcg(D + k[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < SPT; ++u)
+          if (k[u] != kFull) sh.vals[tid + u * kCatchThreads] = d[u];
+      }
+      __syncthreads();
+      // the packets in arrival order; inside one packet every index, and so every slot, occurs once
+      for (uint32_t p = 0; p < count; ++p) {
+        for (uint32_t e = sh.pre[p] + tid; e < sh.pre[p + 1]; e += kCatchThreads) {
+          const uint32_t slot = sh.ent_slot[e];
+          if (slot != 0xFFFFu) sh.vals[slot] = __fsub_rn(sh.vals[slot], sh.ent_val[e]);
+        }
+        __syncthreads();
+      }
+#pragma unroll
+      for (int u = 0; u < SPT; ++u) {
+        const uint32_t i = sh.keys[tid + u * kCatchThreads];
+        if (i != kFull) {
+          const float r = sh.vals[tid + u * kCatchThreads];
+          __stcg(D + i, r);
+          atomicMax(blk_max + i / kWarpTile, key_of(r));   // keeps the block's bound an upper bound
+        }
+      }
     }
+    if (b == range_b) break;
+    __syncthreads();   // the table and the pieces are read until here
+    if (tid < count) sh.lo[tid] = sh.hi[tid];
+    a = b;
   }
 }
 

@@ -66,6 +66,7 @@ def test_selection_adversarial(name, x, segs, ks):
 
 
 @pytest.mark.parametrize("flags", [0, dgs.DGS_NO_SPECULATION, dgs.DGS_KEEP_LOCAL_MODEL, dgs.DGS_RESIDUAL_MODE,
+                                   dgs.DGS_SINGLE_STREAM,
                                    dgs.DGS_RESIDUAL_MODE | dgs.DGS_KEEP_LOCAL_MODEL | dgs.DGS_NO_SPECULATION])
 def test_trajectory_small_ragged(flags):
     # several tiles, ragged heads and tails, tiny layers, repeated arrivals of the same worker
