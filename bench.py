@@ -43,8 +43,7 @@ UNIT = "events/s"
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (same n, so the same bytes per launch); None for kernels or workloads not captured
-NCU_TRAFFIC = {("resnet50-global", "stream_push"): 204538368 + 58706432,
-               ("resnet50-global", "stream_pull"): 102305280 + 3409408}
+NCU_TRAFFIC = {("resnet50-global", "stream_push"): 204536832 + 58724352}
 FALLBACK_HBM_GBS = 6650.0
 
 

@@ -26,9 +26,10 @@
  *     index wins.  Packets list (index, value) pairs in ascending index order.
  *   - DEVICE pointers are marked DEVICE, everything else is host memory.
  *   - The caller owns all device memory (the arena); the library allocates no device
- *     memory.  Calls only enqueue work and return.  The work runs on two streams of the
- *     library's own (one for the pushes, one for apply and pull, so that the push of the
- *     next event overlaps the server side of the current one); it is ordered after
+ *     memory.  Calls only enqueue work and return.  The work runs on streams of the
+ *     library's own (several for the pushes, one for the apply, several for the pulls, so
+ *     that the push of the next events overlaps the server side of the current one; a
+ *     dependency tracker keeps, per buffer, the order of the calls); it is ordered after
  *     everything the caller had enqueued on the stream given at dgs_init when the call
  *     was made.  Results (packets, state) are complete for that stream after dgs_flush,
  *     and for the host after any call that is documented to wait.  One host thread per
@@ -105,8 +106,8 @@ typedef struct {
 enum { DGS_THETA = 0, DGS_U = 1, DGS_D = 2, DGS_THETA_LOCAL = 3 };
 
 /* Bytes of device memory a context for this configuration carves from the arena
- * (model, N velocities + one spare, N differences, packet slots, selection
- * scratch).  No GPU work.  arena/arena_bytes/theta0/stream are ignored. */
+ * (model, N velocities + spares, N differences, packet slots, the log of applied
+ * packets, selection scratch).  No GPU work.  arena/arena_bytes/theta0/stream are ignored. */
 int dgs_arena_bytes(const dgs_config* cfg, uint64_t* out_bytes);
 
 /* Creates the context: u_k = 0 and D_k = 0 for every worker (Algorithm 3 and
@@ -118,13 +119,17 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out);
 /* Worker push (Algorithm 3, velocity update through encode(); Eq. 11a, Eq. 12).
  * grad: DEVICE f32[n], 16-byte aligned, read only, must stay valid until the work of
  * this call has run (dgs_flush, then the stream reaching that point).  On return *out
- * describes the push packet slot (two slots are used alternately). */
+ * describes the push packet slot (a few slots are used in turn). */
 int dgs_worker_push(dgs_ctx* ctx, uint32_t worker, const float* grad, dgs_packet* out);
 
 /* Server apply (Algorithm 2, "M <- M - decode(g)"; Eq. 1-3): theta[i] -= val and
  * D_q[i] -= val for every worker q, the sender included, for each (i, val) of the
  * packet.  pkt may be the library's own push packet or any DEVICE packet with
- * strictly ascending indices < n.  Also advances the server timestamp t. */
+ * strictly ascending indices < n.  Also advances the server timestamp t.
+ * For the library's own packets the subtraction from D_q is deferred: the packet is
+ * filed in a log and folded into D_q, in arrival order, before anything reads D_q
+ * (that worker's next pull, dgs_state_ptr); every D_q[i] sees the same subtractions
+ * in the same order, so the values are the same bit for bit. */
 int dgs_server_apply(dgs_ctx* ctx, uint32_t worker, const dgs_packet* pkt);
 
 /* Worker pull with secondary compression (Algorithm 2, per-layer top-k of
@@ -189,16 +194,16 @@ enum {
   DGS_KERNEL_STREAM_PUSH = 0,   /* push, single-pass route: velocity update + candidate collection      */
   DGS_KERNEL_FINALIZE_PUSH = 1, /* push, single-pass route: exact k-th key, ordered packet, fix-ups      */
   DGS_KERNEL_TWO_PASS_PUSH = 2, /* push, two-pass route only: histogram of the whole input + bound pick  */
-  DGS_KERNEL_SCATTER = 3,       /* apply                                                                 */
+  DGS_KERNEL_SCATTER = 3,       /* apply: theta -= packet, packet filed in the log (or the eager scatter) */
   DGS_KERNEL_STREAM_PULL = 4,
   DGS_KERNEL_FINALIZE_PULL = 5,
   DGS_KERNEL_TWO_PASS_PULL = 6,
-  DGS_KERNEL_CATCH_UP = 7,      /* pull: applied packets folded into the worker's difference vector   */
+  DGS_KERNEL_CATCH_UP = 7,      /* pull: filed packets folded into the worker's difference vector        */
   DGS_NUM_KERNELS = 8
 };
 
 /* Measurement aid (no counterpart in the paper).  While on, every kernel launch of
- * this context is bracketed by two CUDA events on the context's stream (at most
+ * this context is bracketed by two CUDA events on the stream it runs on (at most
  * 65536 launches between two reads are recorded). */
 int dgs_timing_enable(dgs_ctx* ctx, int on);
 

@@ -179,6 +179,12 @@ def test_trajectory_gpt2_small_few_workers():
     replay_and_compare(wl)
 
 
+def test_trajectory_gpt2_small_per_layer_few_workers():
+    # 148 layers from 768 to 38.6 M elements, each selected on its own
+    wl = W.gpt2_small(num_workers=2, num_events=4, per_layer=True)
+    replay_and_compare(wl)
+
+
 @pytest.mark.parametrize("log2n", [16, 18, 20, 22, 24])
 @pytest.mark.parametrize("ppm", W.SWEEP_PPM)
 def test_sweep_selection(log2n, ppm):

@@ -242,6 +242,7 @@ BY_NAME = {
     "resnet18": resnet18,
     "resnet50": resnet50,
     "gpt2": gpt2_small,
+    "gpt2-layerwise": lambda **kw: gpt2_small(per_layer=True, **kw),   # one selection per tensor (148 layers)
 }
 
 
