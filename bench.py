@@ -449,6 +449,7 @@ def run_sweep(args) -> dict:
                 c2.state_load(dgs.DGS_D, 0, x)
                 two_pass.append(timed(lambda: c2.worker_pull(0), c2, reps=1))
                 c2.close()
+                del c2
             t_two = statistics.median(two_pass)
             pull_fresh()                                   # leaves a carried bound behind
             single = []
@@ -460,17 +461,22 @@ def run_sweep(args) -> dict:
             idx, val = sel.packet(p)
             idx, val = idx.clone(), val.clone()
             sel.close()
+            del sel
             row = {"log2n": log2n, "density_ppm": ppm, "k": k,
                    "select_two_pass_us": t_two, "select_single_pass_us": t_single,
                    "select_two_pass_GBs": 4 * n / t_two / 1e3, "select_single_pass_GBs": 4 * n / t_single / 1e3,
                    "select_single_pass_frac_of_peak": 4 * n / t_single / 1e3 / peak}
             for nb_workers in (1, 32):
-                if (2 * nb_workers + 8) * 4 * n > 150e9:
+                torch.cuda.empty_cache()        # the arenas of closed contexts go back to the device
+                need = dgs.dgs_arena_bytes(dgs.make_config(n, nb_workers, 0.1, 0.9, [0], [n], [k], [k]))
+                free, _ = torch.cuda.mem_get_info(dev)
+                if need + (8 << 30) > free:
                     continue
                 ap = dgs.Context(n, nb_workers, 0.1, 0.9, [0], [n], [k], [k], torch.zeros(n, device=dev))
                 fp = dgs.dgs_packet(idx.data_ptr(), val.data_ptr(), k)
                 t_ap = timed(lambda: ap.server_apply(0, fp), ap)
                 ap.close()
+                del ap
                 bytes_alg = 8 * k * (nb_workers + 1) + 8 * k
                 row[f"scatter_{nb_workers + 1}buf_us"] = t_ap
                 row[f"scatter_{nb_workers + 1}buf_GBs"] = bytes_alg / t_ap / 1e3
