@@ -274,43 +274,62 @@ __device__ __forceinline__ void tile_emit(const Workspace& ws, StreamShared& sh,
 }
 
 // A ragged tile (first or last of a layer, fewer than kWarpTile elements or not 16-byte
-// aligned): one element per lane and step, straight from global memory, at most 16 steps.
-// Returns the candidate flags (one bit per step); writes the new velocity (push).
+// aligned): one element per lane and step, straight from global memory, at most 16 steps, the
+// loads of eight steps in flight together.  Returns the candidate flags (one bit per step) and
+// leaves the values of this lane's elements in x[step]; writes the new velocity (push).
+constexpr int kRaggedSteps = kWarpTile / 32;
 template <int MODE>
 __device__ __forceinline__ uint32_t ragged_mask(const SelArgs& a, const Tile tile, uint32_t L, int lane,
-                                                const float* __restrict__ in, float* __restrict__ out) {
+                                                const float* __restrict__ in, float* __restrict__ out,
+                                                float (&x)[kRaggedSteps]) {
   uint32_t flags = 0;
-  for (int st = 0; st * 32 < (int)tile.len; ++st) {
-    const uint32_t off = st * 32 + lane;
-    if (off < tile.len) {
-      const uint32_t i = tile.start + off;
-      const float x = combine<MODE>(in[i], MODE != kPull ? a.grad[i] : 0.f, a.m, a.lr);
-      const bool cand = key_of(x) >= L;
-      if (MODE != kPull) out[i] = cand ? x : unsent<MODE>(x, a.inv_m);
-      if (cand) flags |= 1u << st;
+#pragma unroll
+  for (int s0 = 0; s0 < kRaggedSteps; s0 += 8) {
+    if (s0 * 32 < (int)tile.len) {   // warp-uniform
+      float vu[8], vg[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const uint32_t off = (s0 + j) * 32 + lane;
+        vu[j] = 0.f;
+        vg[j] = 0.f;
+        if (off < tile.len) {
+          vu[j] = in[tile.start + off];
+          if (MODE != kPull) vg[j] = a.grad[tile.start + off];
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const uint32_t off = (s0 + j) * 32 + lane;
+        x[s0 + j] = 0.f;
+        if (off < tile.len) {
+          const float v = combine<MODE>(vu[j], vg[j], a.m, a.lr);
+          const bool cand = key_of(v) >= L;
+          if (MODE != kPull) out[tile.start + off] = cand ? v : unsent<MODE>(v, a.inv_m);
+          if (cand) flags |= 1u << (s0 + j);
+          x[s0 + j] = v;
+        }
+      }
     }
   }
   return flags;
 }
 // Writes its candidates from slot `base` on, in index order.
-template <int MODE>
 __device__ __forceinline__ void ragged_emit(const Workspace& ws, StreamShared& sh, const Tile tile, uint32_t flags,
-                                            uint32_t base, int lane, uint32_t lt, const float* __restrict__ in,
-                                            const float* __restrict__ out) {
+                                            uint32_t base, int lane, uint32_t lt, const float (&x)[kRaggedSteps]) {
   if (!__any_sync(kFull, flags != 0)) return;
-  for (int st = 0; st * 32 < (int)tile.len; ++st) {
-    const bool cand = (flags >> st) & 1u;
-    const uint32_t b = __ballot_sync(kFull, cand);
-    if (cand) {
-      // a candidate's value is what this thread just stored (push) or the input itself (pull)
-      const uint32_t i = tile.start + st * 32 + lane;
-      const float x = MODE == kPull ? in[i] : out[i];
-      const uint32_t pos = base + __popc(b & lt);
-      ws.cand_idx[pos] = i;
-      ws.cand_val[pos] = x;
-      atomicAdd(sh.hist + (key_of(x) >> 20), 1u);
+#pragma unroll
+  for (int st = 0; st < kRaggedSteps; ++st) {
+    if (st * 32 < (int)tile.len) {   // warp-uniform
+      const bool cand = (flags >> st) & 1u;
+      const uint32_t b = __ballot_sync(kFull, cand);
+      if (cand) {
+        const uint32_t pos = base + __popc(b & lt);
+        ws.cand_idx[pos] = tile.start + st * 32 + lane;
+        ws.cand_val[pos] = x[st];
+        atomicAdd(sh.hist + (key_of(x[st]) >> 20), 1u);
+      }
+      base += __popc(b);
     }
-    base += __popc(b);
   }
 }
 
@@ -357,7 +376,7 @@ __device__ void stream_tiles(const Workspace& ws, const SelArgs& a, const uint32
           load_tile_vec<MODE>(in, a.grad, tile.start, lane, a.m, a.lr, x);
           mask = tile_mask_regs<MODE>(a, tile.start, x, L, lane, out);
         } else {
-          mask = ragged_mask<MODE>(a, tile, L, lane, in, out);
+          mask = ragged_mask<MODE>(a, tile, L, lane, in, out, x);
         }
       }
       const uint32_t count = __reduce_add_sync(kFull, (uint32_t)__popc(mask));
@@ -378,7 +397,7 @@ __device__ void stream_tiles(const Workspace& ws, const SelArgs& a, const uint32
             return v;
           });
         } else {
-          ragged_emit<MODE>(ws, sh, tile, mask, base, lane, lt, in, out);
+          ragged_emit(ws, sh, tile, mask, base, lane, lt, x);
         }
       }
     }
@@ -530,9 +549,10 @@ __device__ void stream_tiles_tma(const Workspace& ws, const SelArgs& a, const ui
     auto ragged = [&](uint32_t t) {
       if (warp == 0) {
         const Tile tile = ws.tiles[t];
-        const uint32_t flags = ragged_mask<MODE>(a, tile, L, lane, in, out);
+        float x[kRaggedSteps];
+        const uint32_t flags = ragged_mask<MODE>(a, tile, L, lane, in, out, x);
         const uint32_t count = __reduce_add_sync(kFull, (uint32_t)__popc(flags));
-        ragged_emit<MODE>(ws, sh, tile, flags, slot0 + cur, lane, lt, in, out);
+        ragged_emit(ws, sh, tile, flags, slot0 + cur, lane, lt, x);
         if (lane == 0) sh.cursor = count;
       }
       __syncthreads();
@@ -1294,6 +1314,12 @@ constexpr int kCatchMaxGrid = 8192;
 #endif
 constexpr int kCatchThreads = DGS_CATCH_THREADS;   // threads per CTA of k_catch_up (>= 2 * kCatchMaxPackets)
 
+// Keeps a block's bound an upper bound on the magnitudes in the block.  Bounds only rise while
+// packets are being subtracted, so a bound already read as high enough needs no atomic.
+__device__ __forceinline__ void raise_bound(uint32_t* bound, uint32_t key) {
+  if (key > __ldcg(bound)) atomicMax(bound, key);
+}
+
 struct PacketLog {
   uint32_t* idx;   // [ring][stride], each packet sorted by index
   float* val;      // [ring][stride]
@@ -1527,7 +1553,7 @@ __global__ void __launch_bounds__(kThreads) k_scatter_sub(const uint32_t* __rest
   float* p = (q == num_workers ? theta : D + (uint64_t)q * d_stride) + i;
   const float r = __fsub_rn(*p, v);
   *p = r;
-  if (q < num_workers) atomicMax(blk_max + (uint64_t)q * blk_stride + i / kWarpTile, key_of(r));
+  if (q < num_workers) raise_bound(blk_max + (uint64_t)q * blk_stride + i / kWarpTile, key_of(r));
 }
 
 }  // namespace dgs
