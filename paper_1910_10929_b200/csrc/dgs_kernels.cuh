@@ -1309,6 +1309,7 @@ constexpr int kCatchCap = 2048;          // entries a CTA of k_catch_up can hold
 constexpr int kCatchSlots = 4096;        // slots of its table of distinct indices (power of two, >= 2 * kCatchCap)
 constexpr uint32_t kCatchTarget = 1024;  // entries per CTA the launch aims at
 constexpr int kCatchMaxGrid = 8192;
+constexpr int kCatchBlocks = 256;        // blocks of D whose bounds a CTA of k_catch_up collects in shared memory first
 #ifndef DGS_CATCH_THREADS
 #define DGS_CATCH_THREADS 256
 #endif
@@ -1394,6 +1395,7 @@ struct CatchShared {
   float ent_val[kCatchCap];
   uint32_t lo[kCatchMaxPackets], hi[kCatchMaxPackets], end[kCatchMaxPackets];   // per packet: piece, end of the range
   uint32_t pre[kCatchMaxPackets + 1];    // exclusive prefix of hi - lo
+  uint32_t bmax[kCatchBlocks];           // largest new magnitude per block of kWarpTile elements, from the piece's first block on
 };
 
 __global__ void __launch_bounds__(kCatchThreads) k_catch_up(PacketLog lg, uint64_t first, uint32_t count,
@@ -1412,6 +1414,7 @@ __global__ void __launch_bounds__(kCatchThreads) k_catch_up(PacketLog lg, uint64
   uint32_t a = c == 0 ? 0u : __ldcg(lg.bnd + c);
   for (;;) {   // one round per piece [a, b) of the range; everything here is uniform over the CTA
     for (int s = tid; s < kCatchSlots; s += kCatchThreads) sh.keys[s] = kFull;
+    for (int s = tid; s < kCatchBlocks; s += kCatchThreads) sh.bmax[s] = 0;
     __syncthreads();
     if (tid < count) sh.hi[tid] = sh.end[tid];
     uint32_t b = range_b;
@@ -1521,8 +1524,17 @@ __global__ void __launch_bounds__(kCatchThreads) k_catch_up(PacketLog lg, uint64
         if (i != kFull) {
           const float r = sh.vals[tid + u * kCatchThreads];
           __stcg(D + i, r);
-          atomicMax(blk_max + i / kWarpTile, key_of(r));   // keeps the block's bound an upper bound
+          // keeps the block's bound an upper bound: collected per block in shared memory, one global
+          // atomic per block afterwards (a piece spanning more blocks than fit sends the rest directly)
+          const uint32_t blk = i / kWarpTile - a / kWarpTile;
+          if (blk < (uint32_t)kCatchBlocks) atomicMax(sh.bmax + blk, key_of(r));
+          else atomicMax(blk_max + i / kWarpTile, key_of(r));
         }
+      }
+      __syncthreads();
+      for (int s = tid; s < kCatchBlocks; s += kCatchThreads) {
+        const uint32_t v = sh.bmax[s];
+        if (v) atomicMax(blk_max + a / kWarpTile + s, v);
       }
     }
     if (b == range_b) break;
