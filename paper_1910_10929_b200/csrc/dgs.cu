@@ -50,7 +50,7 @@ inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
 // Scratch of one selection pipeline ([0] push, on the worker stream; [1] pull, on the server stream)
 struct ScratchLayout {
-  uint64_t cand_idx, cand_val, part_cands, part_slot0, cta_tot, seg_start;
+  uint64_t cand_idx, cand_val, part_cands, part_slot0, plan, part_live, cta_tot, seg_start;
   uint64_t hist1, hist2, hist3, sel, L_safe, L_wide, sync;
   uint64_t zero_begin, zero_end;  // [hist1, end of sync): cleared at init
 };
@@ -168,6 +168,8 @@ void make_layout(const dgs_config* c, Layout* L) {
     sc.cand_val = take(vec);
     sc.part_cands = take((uint64_t)kMaxGrid * 4);
     sc.part_slot0 = take((uint64_t)kMaxGrid * 4);
+    sc.plan = take((uint64_t)(kMaxGrid + 1) * 4);
+    sc.part_live = take((uint64_t)kMaxGrid * 4);
     sc.cta_tot = take((uint64_t)kMaxWorkers * sizeof(uint2));
     sc.seg_start = take(S * sizeof(uint2));
     sc.hist1 = take(S * kBins1 * 4);
@@ -533,9 +535,10 @@ int occupancy_grids(dgs_ctx* c, int sms) {
                                                             StreamRing<MODE>::kBytes));
   if (occ < 1) occ = 1;
   c->stream_grid[MODE] = std::min(sms * occ, kMaxGrid);
-#ifdef DGS_PULL_GRID
-  if (MODE == kPull) c->stream_grid[MODE] = std::min(c->stream_grid[MODE], DGS_PULL_GRID);
-#endif
+  // With several workers a pull's stream pass shares the GPU with the push passes of later events, and
+  // what counts is how few SM resources it holds, not how fast it is alone: one CTA per SM (its ranges
+  // are balanced by the plan that finalize leaves behind).  A context with one worker selects alone.
+  if (MODE == kPull && c->cfg.num_workers > 1) c->stream_grid[MODE] = std::min(c->stream_grid[MODE], sms);
   DGS_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_hist_all<MODE>, kThreads, 0));
   if (occ < 1) occ = 1;
   c->hist_grid[MODE] = std::min(sms * occ, kMaxGrid);
@@ -709,6 +712,8 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
     INIT_CUDA(cudaMemsetAsync(c->at<char>(sc.zero_begin), 0, sc.zero_end - sc.zero_begin, st));
     INIT_CUDA(cudaMemsetAsync(c->at<char>(sc.part_cands), 0, (uint64_t)kMaxGrid * 4, st));
     INIT_CUDA(cudaMemsetAsync(c->at<char>(sc.part_slot0), 0, (uint64_t)kMaxGrid * 4, st));
+    INIT_CUDA(cudaMemsetAsync(c->at<char>(sc.plan), 0, (uint64_t)(kMaxGrid + 1) * 4, st));   // no plan yet
+    INIT_CUDA(cudaMemsetAsync(c->at<char>(sc.part_live), 0, (uint64_t)kMaxGrid * 4, st));
   }
   INIT_CUDA(cudaMemsetAsync(c->at<char>(L.blk_max), 0, N * L.blk_stride * 4, st));   // D = 0
   INIT_CUDA(cudaMemsetAsync(c->at<char>(L.L_next), 0xFF, 2 * N * cfg->num_segments * 4, st));
@@ -743,6 +748,8 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
     w.cand_val = c->at<float>(sc.cand_val);
     w.part_cands = c->at<uint32_t>(sc.part_cands);
     w.part_slot0 = c->at<uint32_t>(sc.part_slot0);
+    w.plan = c->at<uint32_t>(sc.plan);
+    w.part_live = c->at<uint32_t>(sc.part_live);
     w.cta_tot = c->at<uint2>(sc.cta_tot);
     w.seg_start = c->at<uint2>(sc.seg_start);
     w.hist1 = c->at<uint32_t>(sc.hist1);
@@ -1332,6 +1339,8 @@ extern "C" int dgs_topk_encode_static(const float* x, uint32_t n, uint32_t k, ui
   ws.cand_val = sc->cand_val;
   ws.part_cands = sc->part_cands;
   ws.part_slot0 = sc->part_slot0;
+  ws.plan = nullptr;
+  ws.part_live = nullptr;
   ws.seg_off = sc->seg_off;
   ws.seg_tile0 = sc->seg_tile0;
   ws.cta_tot = sc->cta_tot;

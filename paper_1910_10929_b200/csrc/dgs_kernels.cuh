@@ -65,7 +65,7 @@ struct SegSel {        // per-layer selection state of the selection in flight
 };
 
 // word indices in Workspace::sync
-enum SyncWord : int { kBarCount = 0, kBarGen = 1, kDecision = 2, kFail = 3, kParts = 4, kNumSyncWords = 8 };
+enum SyncWord : int { kBarCount = 0, kBarGen = 1, kDecision = 2, kFail = 3, kParts = 4, kPlanParts = 5, kNumSyncWords = 8 };
 
 struct Workspace {
   const Tile* tiles;
@@ -77,6 +77,10 @@ struct Workspace {
   float* cand_val;        // [n]
   uint32_t* part_cands;   // [kMaxGrid] candidates written by each part
   uint32_t* part_slot0;   // [kMaxGrid] first slot of each part
+  // Pull, one layer: where the parts of the NEXT stream pass on this scratch set begin (tiles), planned by
+  // finalize from what this pass cost each part; plan[parts] == num_tiles and plan_parts == parts mark it valid.
+  uint32_t* plan;         // [kMaxGrid + 1], or null
+  uint32_t* part_live;    // [kMaxGrid] chunks each part read in the last stream pass, or null
   const uint32_t* seg_off;   // [S+1] first element of each layer, and n
   const uint32_t* seg_tile0; // [S]   first tile of each layer
   uint2* cta_tot;         // [kMaxWorkers] (#key > T, #key == T) among the candidates of each CTA of finalize
@@ -516,7 +520,14 @@ __device__ void stream_tiles_tma(const Workspace& ws, const SelArgs& a, const ui
   using R = StreamRing<MODE>;
   static_assert(R::kStages >= 2, "the ring needs a stage in flight besides the one being read");
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t t0 = part_first_tile(cta, G, ws.num_tiles), t1 = part_first_tile(cta + 1, G, ws.num_tiles);
+  uint32_t t0 = part_first_tile(cta, G, ws.num_tiles), t1 = part_first_tile(cta + 1, G, ws.num_tiles);
+  if (MODE == kPull && ws.plan != nullptr && ld_volatile(ws.sync + kPlanParts) == G &&
+      __ldcg(ws.plan + G) == ws.num_tiles) {
+    // boundaries planned by the finalize of the previous selection on this scratch set
+    t0 = __ldcg(ws.plan + cta);
+    t1 = __ldcg(ws.plan + cta + 1);
+  }
+  uint32_t live_read = 0;   // thread 0: chunks this part reads
   const uint32_t lt = lanemask_lt();
   for (int b = threadIdx.x; b < kBins1; b += kThreads) sh.hist[b] = 0;
   if (threadIdx.x == 0) {
@@ -531,6 +542,7 @@ __device__ void stream_tiles_tma(const Workspace& ws, const SelArgs& a, const ui
     if (threadIdx.x == 0) {
       ws.part_cands[cta] = 0;
       ws.part_slot0[cta] = 0;
+      if (MODE == kPull && ws.part_live != nullptr) ws.part_live[cta] = 0;
     }
     return;
   }
@@ -609,6 +621,7 @@ __device__ void stream_tiles_tma(const Workspace& ws, const SelArgs& a, const ui
       }
       atomicAdd(ws.stats + 3, (unsigned long long)nchunks);
       atomicAdd(ws.stats + 4, (unsigned long long)read);
+      live_read += read;
     }
     uint32_t pc = 0, issued = 0;                          // thread 0: next chunk to ask for, chunks asked for
     if (threadIdx.x == 0) {
@@ -662,6 +675,7 @@ __device__ void stream_tiles_tma(const Workspace& ws, const SelArgs& a, const ui
   if (threadIdx.x == 0) {
     ws.part_cands[cta] = cur;
     ws.part_slot0[cta] = slot0;
+    if (MODE == kPull && ws.part_live != nullptr) ws.part_live[cta] = live_read;
   }
 }
 
@@ -1232,6 +1246,69 @@ __global__ void __maxnreg__(DGS_FINALIZE_REGS) k_finalize(Workspace ws, SelArgs 
       gt_before += is_gt ? 1u : 0u;
       eq_before += is_eq ? 1u : 0u;
     });
+  }
+  if (MODE == kPull && S == 1 && !redo && ws.plan != nullptr && ws.part_live != nullptr && cta == 0) {
+    // Plan for the next pull's stream pass on this scratch set: its CTAs get ranges of tiles that cost
+    // about the same, judged by what this pass cost each part (chunks read, candidates appended).  The
+    // chunks that have to be read cluster in the tensors with the largest updates, and those tensors are
+    // the same for every worker; with equal ranges a few CTAs do most of the reading.
+    constexpr int PER = kMaxGrid / kThreads;
+    const bool had = ld_volatile(ws.sync + kPlanParts) == parts && __ldcg(ws.plan + parts) == ws.num_tiles;
+    uint32_t cost[PER], old_t0[PER];
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      const uint32_t p = j * kThreads + threadIdx.x;
+      cost[j] = 0;
+      old_t0[j] = 0;
+      if (p < parts) {
+        cost[j] = 4u + 8u * __ldcg(ws.part_live + p) + (sh.pre_cands[p + 1] - sh.pre_cands[p]) / 16u;
+        old_t0[j] = had ? __ldcg(ws.plan + p) : part_first_tile(p, parts, ws.num_tiles);
+      }
+    }
+    __syncthreads();   // pre_cands and slot0 have been read for the last time
+    unsigned long long carry = 0;
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      if ((uint32_t)(j * kThreads) < parts) {   // CTA-uniform
+        const uint32_t p = j * kThreads + threadIdx.x;
+        unsigned long long total;
+        const unsigned long long ex = block_excl_scan(cost[j], sh.warp_scan, total) + carry;
+        if (p < parts) {
+          sh.pre_cands[p] = (uint32_t)ex;    // cost of the parts before p
+          sh.slot0[p] = old_t0[j];
+          sh.stream.hist[kMaxGrid + 1 + p] = cost[j];
+        }
+        carry += total;
+      }
+    }
+    __syncthreads();
+    const unsigned long long total_cost = carry;
+    for (uint32_t j = threadIdx.x; j <= parts; j += kThreads) {
+      uint32_t tile = j == 0 ? 0u : ws.num_tiles;
+      if (j > 0 && j < parts) {
+        const unsigned long long target = total_cost * j / parts;
+        uint32_t lo = 0, hi = parts - 1;       // last part whose earlier parts cost no more than the target
+        while (lo < hi) {
+          const uint32_t mid = (lo + hi + 1) >> 1;
+          if (sh.pre_cands[mid] <= target) lo = mid; else hi = mid - 1;
+        }
+        const uint32_t a0 = sh.slot0[lo], a1 = lo + 1 < parts ? sh.slot0[lo + 1] : ws.num_tiles;
+        const unsigned long long into = target - sh.pre_cands[lo], c = sh.stream.hist[kMaxGrid + 1 + lo];
+        tile = a0 + (uint32_t)((unsigned long long)(a1 - a0) * min(into, c) / c);
+      }
+      sh.stream.hist[j] = tile;
+    }
+    __syncthreads();
+    // a part must not be longer than the pass can keep skip flags for; otherwise no plan
+    int ok = 1;
+    for (uint32_t j = threadIdx.x; j < parts; j += kThreads)
+      if (sh.stream.hist[j + 1] < sh.stream.hist[j] || sh.stream.hist[j + 1] - sh.stream.hist[j] > 16384u) ok = 0;
+    ok = __syncthreads_and(ok);
+    for (uint32_t j = threadIdx.x; j < parts; j += kThreads) ws.plan[j] = sh.stream.hist[j];
+    if (threadIdx.x == 0) {
+      ws.plan[parts] = ok ? ws.num_tiles : 0u;
+      ws.sync[kPlanParts] = parts;
+    }
   }
   if (cta == 0 && threadIdx.x == 0) {
     if (MODE != kPull) {  // the spare buffer now holds the worker's velocity
