@@ -43,7 +43,7 @@ UNIT = "events/s"
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (same n, so the same bytes per launch); None for kernels or workloads not captured
-NCU_TRAFFIC = {("resnet50-global", "stream_push"): 204555776 + 59887360}
+NCU_TRAFFIC = {("resnet50-global", "stream_push"): 204552960 + 58023168}
 FALLBACK_HBM_GBS = 6650.0
 
 
