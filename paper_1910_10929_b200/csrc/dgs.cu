@@ -242,6 +242,7 @@ struct dgs_ctx {
   std::vector<uint64_t> applied;  // per worker
   Workspace ws[kAllSets];  // push sets, then pull sets
   float inv_m;
+  int sms;               // SMs of the device
   int stream_grid[3];    // CTAs of the stand-alone stream pass, per mode
   int hist_grid[3];      // CTAs of the whole-input histogram pass, per mode
   int finalize_grid[3];  // CTAs of the cooperative finalize kernel, per mode
@@ -426,7 +427,10 @@ int catch_up_launch(dgs_ctx* c, uint32_t q, cudaStream_t st) {
   const uint32_t count = (uint32_t)(c->log_head - first);
   if (count > 0) {
     TimedLaunch tl(c, st, DGS_KERNEL_CATCH_UP);
-    k_catch_up<<<c->log.ranges, kCatchThreads, 0, st>>>(c->log, first, count, c->D_buf(q), c->blk_max(q), c->cfg.n);
+    // One CTA per SM at most, each taking several ranges in turn: the kernel runs beside the push passes of
+    // later events, and the loop is faster when it holds few SM resources than when it finishes early.
+    const unsigned catch_grid = std::min<unsigned>(c->log.ranges, (unsigned)c->sms);
+    k_catch_up<<<catch_grid, kCatchThreads, 0, st>>>(c->log, first, count, c->D_buf(q), c->blk_max(q), c->cfg.n);
     DGS_CUDA(c, cudaGetLastError());
     c->launches += 1;
   }
@@ -665,6 +669,7 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   INIT_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   INIT_CUDA(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
   if (!coop) return fail(DGS_ECUDA);
+  c->sms = sms;
   if (occupancy_grids<kPushSam>(c, sms) != DGS_OK || occupancy_grids<kPushResidual>(c, sms) != DGS_OK ||
       occupancy_grids<kPull>(c, sms) != DGS_OK)
     return fail(DGS_ECUDA);

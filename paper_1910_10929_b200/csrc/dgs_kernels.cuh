@@ -1456,7 +1456,7 @@ __global__ void __launch_bounds__(kThreads) k_apply_log(const uint32_t* __restri
 }
 
 // D -= packets first .. first + count - 1 of the log, in that order (count <= kCatchMaxPackets).
-// CTA c owns range c of the log (gridDim.x = ranges); its part of every packet is known from the
+// A CTA owns a range c of the log at a time; its part of every packet is known from the
 // positions filed with the packet.  It gathers the distinct indices of all those parts in a
 // shared-memory table, loads each D[i] once, subtracts the packets' values from the table in
 // packet order (indices inside one packet are distinct, so a packet is one parallel step) and
@@ -1479,8 +1479,10 @@ __global__ void __launch_bounds__(kCatchThreads) k_catch_up(PacketLog lg, uint64
                                                        float* __restrict__ D, uint32_t* __restrict__ blk_max,
                                                        uint64_t n) {
   __shared__ CatchShared sh;
-  const uint32_t tid = threadIdx.x, c = blockIdx.x;
+  const uint32_t tid = threadIdx.x;
   if (count == 0 || count > (uint32_t)kCatchMaxPackets) return;
+  // a CTA takes the ranges blockIdx.x, blockIdx.x + gridDim.x, ... one after the other
+  for (uint32_t c = blockIdx.x; c < lg.ranges; c += gridDim.x) {
   if (tid < 2 * count) {
     // thread 2p reads where range c begins in packet p, thread 2p+1 where it ends
     const uint32_t p = tid >> 1;
@@ -1618,6 +1620,8 @@ __global__ void __launch_bounds__(kCatchThreads) k_catch_up(PacketLog lg, uint64
     __syncthreads();   // the table and the pieces are read until here
     if (tid < count) sh.lo[tid] = sh.hi[tid];
     a = b;
+  }
+  __syncthreads();   // the tables are free for the next range
   }
 }
 
