@@ -543,6 +543,9 @@ int occupancy_grids(dgs_ctx* c, int sms) {
   // what counts is how few SM resources it holds, not how fast it is alone: one CTA per SM (its ranges
   // are balanced by the plan that finalize leaves behind).  A context with one worker selects alone.
   if (MODE == kPull && c->cfg.num_workers > 1) c->stream_grid[MODE] = std::min(c->stream_grid[MODE], sms);
+#ifdef DGS_PULL_GRID   // tunable for experiments
+  if (MODE == kPull && c->cfg.num_workers > 1) c->stream_grid[MODE] = std::min(c->stream_grid[MODE], DGS_PULL_GRID);
+#endif
   DGS_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_hist_all<MODE>, kThreads, 0));
   if (occ < 1) occ = 1;
   c->hist_grid[MODE] = std::min(sms * occ, kMaxGrid);
