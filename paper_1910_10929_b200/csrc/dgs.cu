@@ -480,8 +480,12 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age
   const bool single_pass = row >= 0;
   a.L_next = c->L_next(KIND, worker);
   a.force_two_pass = single_pass ? 0 : 1;
-  // a selection of very many entries (dense packets) gets more CTAs: one more per 4096 entries
-  const int fin_grid = std::min(c->finalize_max[MODE], std::max(c->finalize_grid[MODE], (int)(a.pkt_count / 4096)));
+  // A selection of very many entries (dense packets) gets more CTAs: one more per 4096 entries.  One whose
+  // candidates (about three times the entries) fit the registers of 48 CTAs' threads, eight each, gets only
+  // those 48: finalize runs beside the push passes of later events and should hold few SMs.
+  int fin_base = c->finalize_grid[MODE];
+  if (3ull * a.pkt_count <= 48ull * kThreads * 8) fin_base = std::min(fin_base, 48);
+  const int fin_grid = std::min(c->finalize_max[MODE], std::max(fin_base, (int)(a.pkt_count / 4096)));
   a.workers = (uint32_t)fin_grid;
   a.seq = ++c->select_seq;
   a.L_in = single_pass ? c->L_next(KIND, (uint32_t)row) : ws.L_safe;
