@@ -144,7 +144,8 @@ int dgs_event(dgs_ctx* ctx, uint32_t worker, const float* grad, dgs_packet* push
 
 /* Makes the stream given at dgs_init wait (on the device, not the host) for all work
  * enqueued by earlier calls: what that stream runs afterwards sees their packets and
- * state.  (No counterpart in the paper: it joins the library's two streams.) */
+ * state.  (No counterpart in the paper: it joins the library's own streams -- four for the
+ * pushes, one for the apply, six for the pulls -- to the caller's.) */
 int dgs_flush(dgs_ctx* ctx);
 
 /* The same event with HOST buffers (needs DGS_HOST_IO): copies grad (HOST f32[n],
@@ -258,6 +259,15 @@ int dgs_free(dgs_ctx* ctx);
  * two calls whose work overlaps on the GPU (different streams, no ordering) race on it --
  * order them. */
 int dgs_topk_encode_static(const float* x, uint32_t n, uint32_t k, uint32_t* out_idx, float* out_val, void* stream);
+
+/* Device-side outcome of the dgs_topk_encode_static calls enqueued on `stream` so far.  (No
+ * counterpart in the paper.)  dgs_topk_encode_static only enqueues work, so it cannot report a
+ * failure that happens on the device: a bounded wait that gave up (DGS_ETIMEOUT) or an
+ * internal rank check that failed leave out_idx / out_val partly unwritten.  This call waits
+ * for `stream` (host-side wait), then stores in *device_status the status word of the last
+ * call's kernels: 0 = the packet is complete, negative = it is not.  Like the selection itself
+ * it allocates nothing (one 4-byte copy from the fixed array). */
+int dgs_topk_encode_static_status(void* stream, int* device_status);
 
 /* Static text for a dgs_error value. */
 const char* dgs_error_string(int err);

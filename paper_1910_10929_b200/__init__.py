@@ -30,6 +30,7 @@ EXPORTS = (
     "dgs_event", "dgs_flush", "dgs_event_host", "dgs_state_ptr", "dgs_state_load", "dgs_status", "dgs_stats", "dgs_pull_read_stats",
     "dgs_prev", "dgs_launch_count", "dgs_last_cuda_error", "dgs_free", "dgs_error_string",
     "dgs_timing_enable", "dgs_timing_read", "dgs_timing_trace", "dgs_topk_encode_static",
+    "dgs_topk_encode_static_status",
 )
 DGS_ELIMIT = -6
 DGS_STATIC_MAX_N = 1 << 20
@@ -87,6 +88,7 @@ def lib() -> C.CDLL:
         L.dgs_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
         L.dgs_last_cuda_error.argtypes = [vp]
         L.dgs_topk_encode_static.argtypes = [vp, u32, u32, vp, vp, vp]
+        L.dgs_topk_encode_static_status.argtypes = [vp, C.POINTER(i32)]
         L.dgs_timing_enable.argtypes = [vp, i32]
         L.dgs_timing_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
         L.dgs_timing_trace.argtypes = [vp, u32, C.POINTER(C.c_float), C.POINTER(C.c_float), C.POINTER(C.c_int32),
@@ -230,6 +232,13 @@ def dgs_topk_encode_static(x_ptr: int, n: int, k: int, out_idx_ptr: int, out_val
     fixed array inside the library, n <= DGS_STATIC_MAX_N).  Enqueues on `stream`."""
     _check(lib().dgs_topk_encode_static(x_ptr, n, k, out_idx_ptr, out_val_ptr, stream or None),
            "dgs_topk_encode_static")
+
+
+def dgs_topk_encode_static_status(stream: int = 0) -> int:
+    """Waits for `stream`; 0 if the packets of the static selections enqueued so far are complete."""
+    out = C.c_int(0)
+    _check(lib().dgs_topk_encode_static_status(stream or None, C.byref(out)), "dgs_topk_encode_static_status")
+    return int(out.value)
 
 
 def dgs_free(ctx: int) -> None:

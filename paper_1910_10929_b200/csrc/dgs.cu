@@ -1,9 +1,9 @@
 // Host side of the C ABI declared in include/dgs.h: argument checks, the layout of
 // the caller's arena, and the kernel launches of one push / apply / pull event.
 //
-// Work runs on a few streams of the library's own so that independent steps of consecutive
-// events overlap: pushes alternate between two worker streams, the apply runs on a stream
-// of its own, pulls alternate between two server streams.  A push touches only the worker's
+// Work runs on streams of the library's own so that independent steps of consecutive
+// events overlap: pushes take kWorkerStreams worker streams in turn, the apply runs on a stream
+// of its own, pulls take kServerStreams server streams in turn.  A push touches only the worker's
 // velocity, the gradient and its own scratch; a pull touches one difference vector.  The
 // small, latency-bound finalize kernels thus share the GPU with the bandwidth-bound passes
 // of other events.  Order is kept by a small dependency tracker: every launch names the
@@ -200,7 +200,7 @@ void make_layout(const dgs_config* c, Layout* L) {
   L->L_next = take(2 * N * S * 4);
   L->u_slots = take((N + kPushSets) * sizeof(float*));
   L->status = take(4);
-  L->stats = take(32 * 8);
+  L->stats = take((uint64_t)kNumStats * 8);
   L->total = off;
 }
 
@@ -1249,8 +1249,10 @@ struct StaticScratch {
   uint32_t L_next[1];
   uint32_t sync[kNumSyncWords];
   int status;
-  unsigned long long stats[4];
+  unsigned long long stats[kNumStats];   // the kernels index words 0 .. 4
 };
+static_assert(sizeof(((StaticScratch*)nullptr)->stats) == kNumStats * sizeof(unsigned long long),
+              "the static scratch must hold every counter a Workspace has");
 
 // The scratch itself.  In host code this name is only a handle for cudaGetSymbolAddress,
 // never a device address.
@@ -1383,12 +1385,17 @@ extern "C" int dgs_topk_encode_static(const float* x, uint32_t n, uint32_t k, ui
   a.seq = 0;
 
   if (cudaMemcpyAsync(sc->x, x, (size_t)n * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return DGS_ECUDA;
+  // every launch is checked before the next one is enqueued: a kernel that did not start must not be
+  // followed by kernels that count on what it clears (peek: an earlier error of the caller's stays the caller's)
   const uint32_t prep_items = std::max<uint32_t>(num_tiles, kBins1);
   k_static_prepare<<<(prep_items + kThreads - 1) / kThreads, kThreads, 0, st>>>(sc, n, k, num_tiles);
+  if (cudaPeekAtLastError() != cudaSuccess) return DGS_ECUDA;
   k_hist_all<kPull><<<d->hist_grid, kThreads, 0, st>>>(ws, a);
+  if (cudaPeekAtLastError() != cudaSuccess) return DGS_ECUDA;
   k_pick_lower<kPull><<<1, kThreads, 0, st>>>(ws);
+  if (cudaPeekAtLastError() != cudaSuccess) return DGS_ECUDA;
   k_stream<kPull><<<d->stream_grid, kThreads, StreamRing<kPull>::kBytes, st>>>(ws, a);
-  if (cudaGetLastError() != cudaSuccess) return DGS_ECUDA;
+  if (cudaPeekAtLastError() != cudaSuccess) return DGS_ECUDA;
   void* args[] = {(void*)&ws, (void*)&a};
   if (cudaLaunchCooperativeKernel((const void*)k_finalize<kPull>, dim3(d->finalize_grid), dim3(kThreads), args,
                                   finalize_dyn_bytes(1), st) != cudaSuccess)
@@ -1396,3 +1403,18 @@ extern "C" int dgs_topk_encode_static(const float* x, uint32_t n, uint32_t k, ui
   return DGS_OK;
 }
 
+extern "C" int dgs_topk_encode_static_status(void* stream, int* device_status) {
+  if (!device_status) return DGS_EINVAL;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return DGS_ECUDA;
+  StaticDevice* d = nullptr;
+  const int rc = static_setup(dev, &d);
+  if (rc != DGS_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int word = 0;
+  if (cudaMemcpyAsync(&word, &d->scratch->status, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return DGS_ECUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return DGS_ECUDA;
+  *device_status = word;
+  return DGS_OK;
+}

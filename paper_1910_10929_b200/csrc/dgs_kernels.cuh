@@ -41,6 +41,7 @@ constexpr int kMaxGrid = 512;       // upper bound on the grid of a stream pass 
 constexpr int kMaxWorkers = 320;    // upper bound on the grid of finalize
 constexpr uint32_t kSpinLimit = 1u << 22;  // bounded waits: give up and report after this many polls
 constexpr int kStatusTimeout = -4;  // = DGS_ETIMEOUT
+constexpr int kNumStats = 8;        // words of Workspace::stats (every owner of a Workspace provides that many)
 
 enum Mode : int { kPushSam = 0, kPushResidual = 1, kPull = 2 };
 
@@ -93,7 +94,9 @@ struct Workspace {
   uint32_t* L_wide;       // [S] from the same histogram: the bound that admits max(3k, k+64) entries
   uint32_t* sync;         // [kNumSyncWords]
   int* status;            // sticky device status word
-  unsigned long long* stats;  // [0] single-pass selections, [1] two-pass selections, [2] candidates seen
+  // [kNumStats] counters: [0] single-pass selections, [1] two-pass selections, [2] candidates seen,
+  // [3] chunks of difference vectors covered by the pulls' stream passes, [4] those of them read
+  unsigned long long* stats;
 };
 
 struct SelArgs {

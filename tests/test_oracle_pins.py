@@ -72,12 +72,15 @@ def _read_golden(path):
     return head, events
 
 
-def test_hand_example():
-    head, events = _read_golden(os.path.join(GOLDEN, "hand_example.txt"))
+@pytest.mark.parametrize("name", ["hand_example.txt", "hand_example_algorithm1.txt"])
+def test_hand_example(name):
+    head, events = _read_golden(os.path.join(GOLDEN, name))
     n, N, k = int(head["n"][0]), int(head["workers"][0]), int(head["k"][0])
     theta0 = np.array([float(v) for v in head["theta0"]], np.float32)
+    residual = head.get("mode", ["momentum"])[0] == "residual"       # worker rule of Algorithm 1
     o = oracle.Oracle(n, N, float(head["lr"][0]), float(head["momentum"][0]),
-                      [0], [n], [k], [k], theta0, keep_local=True)
+                      [0], [n], [k], [k], theta0, keep_local=True, residual_mode=residual)
+    assert o.timestamp == 0 and [o.prev(q) for q in range(N)] == [-1] * N
     for ev in events:
         w = ev["worker"]
         pi, pv = o.push(w, ev["grad"].astype(np.float32))
@@ -92,6 +95,9 @@ def test_hand_example():
         assert list(o.state(oracle.D, 0)) == list(ev["D0"])
         assert list(o.state(oracle.D, 1)) == list(ev["D1"])
         assert list(o.state(oracle.THETA_LOCAL, w)) == list(ev["theta_local"])
+        # Algorithm 2, last lines: t counts the applied packets, prev(k) = t when k has been served
+        assert o.timestamp == int(ev["timestamp"][0])
+        assert [o.prev(q) for q in range(N)] == [int(v) for v in ev["prev"]]
         # Eq. 3-5: every worker's copy plus what the server still owes it is the global model
         for q in range(N):
             assert np.array_equal(o.state(oracle.THETA_LOCAL, q) + o.state(oracle.D, q),

@@ -8,8 +8,9 @@ one entry point whose scratch is a fixed array inside the library's device image
 
 The test calls it through the C ABI twice in a row (the second call sees whatever the
 first one left in the shared scratch) and requires the packets to be bit-identical to
-those of the ordinary route, dgs_worker_pull on a one-worker context: same indices,
-same value bits -- the bar every selection test here uses.  It sits in a file that is
+those of the ordinary route, dgs_worker_pull on a one-worker context, and to the CPU
+checker's selection of the same vector: same indices, same value bits -- the bar every
+selection test here uses.  It sits in a file that is
 collected last so that a failure here cannot hide any other test, and it must pass both
 alone in a fresh process and after the rest of the suite."""
 import ctypes as C
@@ -18,6 +19,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_1910_10929_b200 as dgs
 import workloads as W
 
@@ -42,6 +44,8 @@ def static_packet(x_dev: torch.Tensor, k: int):
     before = torch.cuda.memory_allocated(DEV)
     dgs.dgs_topk_encode_static(x_dev.data_ptr(), x_dev.numel(), k, idx.data_ptr(), val.data_ptr(),
                                torch.cuda.current_stream().cuda_stream)
+    # the call only enqueues: the device-side outcome is read back separately (and waits for the stream)
+    assert dgs.dgs_topk_encode_static_status(torch.cuda.current_stream().cuda_stream) == 0
     torch.cuda.synchronize()
     assert torch.cuda.memory_allocated(DEV) == before
     return idx, val
@@ -60,6 +64,9 @@ def test_static_selection_matches_pull_twice_in_a_row():
         got_idx, got_val = static_packet(x_dev, k)
         assert torch.equal(got_idx, want_idx)
         assert torch.equal(got_val.view(torch.int32), want_val.view(torch.int32))
+        chosen = oracle.topk(x, k)                                 # the CPU checker's selection of the same vector
+        assert np.array_equal(got_idx.cpu().numpy().view(np.uint32), chosen.astype(np.uint32))
+        assert np.array_equal(got_val.cpu().numpy().view(np.uint32), x[chosen].view(np.uint32))
         assert torch.equal(x_dev.view(torch.int32), keep.view(torch.int32))   # the input is left alone
 
 
