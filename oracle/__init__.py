@@ -46,6 +46,8 @@ def _load():
         L.dgs_oracle_apply.restype = None
         L.dgs_oracle_pull.argtypes = [vp, u32, vp, vp]
         L.dgs_oracle_pull.restype = u64
+        L.dgs_oracle_pull_all.argtypes = [vp, u32, vp, vp, u64]
+        L.dgs_oracle_pull_all.restype = u64
         L.dgs_oracle_state.argtypes = [vp, C.c_int, u32]
         L.dgs_oracle_state.restype = vp
         L.dgs_oracle_timestamp.argtypes = [vp]
@@ -118,6 +120,16 @@ class Oracle:
         c = self._L.dgs_oracle_pull(self._h, w, _p(idx), _p(val))
         assert c == self.K_pull
         return idx, val
+
+    def pull_all(self, w: int, cap: Optional[int] = None) -> Tuple[np.ndarray, np.ndarray, int]:
+        """Pull without secondary compression: every nonzero entry of D_w, ascending, then cleared.
+        Returns (idx, val, held) where held is how many nonzeros D_w had (> cap means overflow)."""
+        cap = self.n if cap is None else int(cap)
+        idx = np.empty(cap, dtype=np.uint32)
+        val = np.empty(cap, dtype=np.float32)
+        held = int(self._L.dgs_oracle_pull_all(self._h, w, _p(idx), _p(val), cap))
+        m = min(held, cap)
+        return idx[:m].copy(), val[:m].copy(), held
 
     def event(self, w: int, grad: np.ndarray):
         """push -> apply -> pull for worker w; returns both packets."""

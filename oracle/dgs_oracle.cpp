@@ -24,6 +24,8 @@
 //   * D_k is stored instead of (M, v_k): M - decode(g) lowers every D_k by the
 //     packet, and v_k <- v_k + G lowers D_k by G, i.e. clears the sent entries.
 //   * unsent velocity entries are multiplied once by fl(1/m)  (Eq. 12 form).
+//   * a pull without secondary compression sends every entry of D_k that is not zero
+//     (+0 and -0 both count as zero) and clears it.
 //
 // parity pins: see tests/test_oracle_*.py (brute-force sort, hand-worked example,
 // dense limit = serial momentum ASGD, Eq. 13 telescoping, Eq. 12, exact split).
@@ -183,6 +185,31 @@ uint64_t dgs_oracle_pull(void* h, uint32_t w, uint32_t* out_idx, float* out_val)
       ++cnt;
       if (o.keep_local) o.theta_local[w][i] = o.theta_local[w][i] + D[i];   // Eq. 5
       D[i] = 0.0f;                                                          // v_k <- v_k + G
+    }
+  }
+  o.prev[w] = static_cast<int64_t>(o.stamp);
+  return cnt;
+}
+
+// Worker pull WITHOUT secondary compression (Algorithm 2 with the switch off; the paper's normal
+// case: "there is no secondary compression for G"): the server sends all of G_k = M - v_k, which is
+// sparse, and v_k becomes M (Eq. 3, Eq. 4).  In accumulator form: every nonzero entry of D_k is
+// sent, in ascending index order, and cleared, so that D_k is zero afterwards; the worker adds G
+// to its model (Eq. 5).  At most `cap` entries are written; returns how many D_k held (the caller
+// sees an overflow as a return value above cap; entries beyond cap are neither sent nor cleared).
+uint64_t dgs_oracle_pull_all(void* h, uint32_t w, uint32_t* out_idx, float* out_val, uint64_t cap) {
+  Oracle& o = *static_cast<Oracle*>(h);
+  std::vector<float>& D = o.D[w];
+  uint64_t cnt = 0;
+  for (uint64_t i = 0; i < o.n; ++i) {
+    if (D[i] != 0.0f) {
+      if (cnt < cap) {
+        out_idx[cnt] = static_cast<uint32_t>(i);
+        out_val[cnt] = D[i];
+        if (o.keep_local) o.theta_local[w][i] = o.theta_local[w][i] + D[i];   // Eq. 5
+        D[i] = 0.0f;                                                          // v_k <- v_k + G = M (Eq. 4)
+      }
+      ++cnt;
     }
   }
   o.prev[w] = static_cast<int64_t>(o.stamp);

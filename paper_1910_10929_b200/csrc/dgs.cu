@@ -30,7 +30,10 @@ namespace {
 
 constexpr uint64_t kAlign = 256;
 constexpr uint32_t kMagic = 0x44475331u;  // "DGS1"
-constexpr int kPushSlots = 5;             // push packet slots, used in turn
+#ifndef DGS_PUSH_SLOTS
+#define DGS_PUSH_SLOTS 8
+#endif
+constexpr int kPushSlots = DGS_PUSH_SLOTS;  // push packet slots, used in turn (a slot is refilled once its apply has read it)
 constexpr int kPullSlots = 6;             // pull packet slots
 #ifndef DGS_WORKER_STREAMS
 #define DGS_WORKER_STREAMS 4
@@ -42,7 +45,7 @@ constexpr int kWorkerStreams = DGS_WORKER_STREAMS, kServerStreams = DGS_SERVER_S
 constexpr int kPushSets = kWorkerStreams;  // scratch sets and spare velocity buffers of the pushes
 constexpr int kPullSets = kServerStreams;  // scratch sets of the pulls
 constexpr int kAllSets = kPushSets + kPullSets;
-constexpr int kLogRingMax = kCatchMaxPackets;  // most packets the apply log keeps (one k_catch_up launch folds them all)
+constexpr int kLogRingMax = 64;             // most packets the apply log keeps
 enum StreamId : int { kStW0 = 0, kStApply = kWorkerStreams, kStS0 = kWorkerStreams + 1,
                       kNumStreams = kWorkerStreams + 1 + kServerStreams };
 
@@ -182,7 +185,13 @@ void make_layout(const dgs_config* c, Layout* L) {
     sc.sync = take(kNumSyncWords * 4);
     sc.zero_end = off;
   }
-  L->log_ring = (uint32_t)std::min<uint64_t>(kLogRingMax, std::max<uint64_t>(N + 8, 16));
+#ifndef DGS_LOG_SLACK
+#define DGS_LOG_SLACK 32
+#endif
+  // A slot of the log is reused `ring` packets later, and the apply that refills it waits for every catch-up that
+  // still reads the old packet.  A worker that comes back after N events reads the N newest packets, so ring - N
+  // is how many events the server side of an event may lag behind the pushes before the pushes stall.
+  L->log_ring = (uint32_t)std::min<uint64_t>(kLogRingMax, std::max<uint64_t>(N + DGS_LOG_SLACK, 16));
   L->log_stride = (uint32_t)align_up(L->K[0], 64);
   L->log_idx = take((uint64_t)L->log_ring * L->log_stride * 4);
   L->log_val = take((uint64_t)L->log_ring * L->log_stride * 4);
@@ -193,7 +202,7 @@ void make_layout(const dgs_config* c, Layout* L) {
     L->log_ranges = (uint32_t)std::min<uint64_t>(std::min<uint64_t>(kCatchMaxGrid, L->K[0]),
                                                  std::max<uint64_t>(1, (entries + kCatchTarget - 1) / kCatchTarget));
   }
-  L->log_bnd = take((uint64_t)L->log_ranges * 4);
+  L->log_bnd = take((uint64_t)L->log_ranges * 4 * 2);   // two generations of ranges, see apply_impl
   L->log_pos = take((uint64_t)L->log_ring * (L->log_ranges + 1) * 4);
   L->blk_stride = align_up((c->n + kWarpTile - 1) / kWarpTile, 64);
   L->blk_max = take(N * L->blk_stride * 4);
@@ -239,10 +248,15 @@ struct dgs_ctx {
   // p % ring of the log from its apply on; applied[q] packets have been folded into D_q so far.
   PacketLog log;
   uint64_t log_head;              // packets filed so far
+  uint64_t last_ranges;           // packet number at which the current generation of ranges was taken
+  int cur_gen;                    // generation of ranges that new packets are filed under
+  int64_t gen_last[2];            // newest packet filed under each generation, -1 if none
+  std::vector<uint8_t> slot_gen;  // per slot of the ring: generation its packet was filed under
   std::vector<uint64_t> applied;  // per worker
   Workspace ws[kAllSets];  // push sets, then pull sets
   float inv_m;
   int sms;               // SMs of the device
+  bool light_pull;       // pulls run the ring-less form of their stream pass
   int stream_grid[3];    // CTAs of the stand-alone stream pass, per mode
   int hist_grid[3];      // CTAs of the whole-input histogram pass, per mode
   int finalize_grid[3];  // CTAs of the cooperative finalize kernel, per mode
@@ -297,8 +311,8 @@ struct ResIds {
   uint32_t PKT(int slot) const { return 5 * N + 1 + kPushSets + kAllSets + slot; }   // push slots, then pull slots
   uint32_t STAGE() const { return PKT(kPushSlots + kPullSlots); }
   uint32_t LOG(uint32_t slot) const { return STAGE() + 1 + slot; }
-  uint32_t RANGES() const { return LOG(kLogRingMax); }   // the ranges of the log
-  uint32_t count() const { return RANGES() + 1; }
+  uint32_t RANGES(int gen) const { return LOG(kLogRingMax) + (uint32_t)gen; }   // the two generations of ranges of the log
+  uint32_t count() const { return RANGES(1) + 1; }
 };
 
 #define DGS_CUDA(ctx, call)                 \
@@ -417,22 +431,36 @@ int task_end(dgs_ctx* c, const Task& t) {
 // Dependencies of folding the filed packets that D_q has not seen yet into it.
 void catch_up_deps(const dgs_ctx* c, uint32_t q, Task* t) {
   const ResIds R{c->cfg.num_workers};
-  for (uint64_t p = c->applied[q]; p < c->log_head; ++p) t->reads.push_back(R.LOG((uint32_t)(p % c->log.ring)));
-  if (c->applied[q] < c->log_head) t->reads.push_back(R.RANGES());
+  bool gen_used[2] = {false, false};
+  for (uint64_t p = c->applied[q]; p < c->log_head; ++p) {
+    t->reads.push_back(R.LOG((uint32_t)(p % c->log.ring)));
+    gen_used[c->slot_gen[p % c->log.ring]] = true;
+  }
+  for (int g = 0; g < 2; ++g)
+    if (gen_used[g]) t->reads.push_back(R.RANGES(g));
   t->writes.push_back(R.D(q));
 }
 // The launch itself, on a stream that task_begin has prepared with those dependencies.
 int catch_up_launch(dgs_ctx* c, uint32_t q, cudaStream_t st) {
-  const uint64_t first = c->applied[q];
-  const uint32_t count = (uint32_t)(c->log_head - first);
-  if (count > 0) {
+  uint64_t first = c->applied[q];
+  // The packets still to be folded in were filed under at most two generations of ranges, the older
+  // ones first: one launch per generation and per kCatchMaxPackets packets, in that order (the order of
+  // the subtractions is kept).
+  while (first < c->log_head) {
+    const int gen = c->slot_gen[first % c->log.ring];
+    uint64_t end = first + 1;
+    while (end < c->log_head && end - first < (uint64_t)kCatchMaxPackets && c->slot_gen[end % c->log.ring] == gen) ++end;
+    const uint32_t count = (uint32_t)(end - first);
     TimedLaunch tl(c, st, DGS_KERNEL_CATCH_UP);
     // One CTA per SM at most, each taking several ranges in turn: the kernel runs beside the push passes of
     // later events, and the loop is faster when it holds few SM resources than when it finishes early.
     const unsigned catch_grid = std::min<unsigned>(c->log.ranges, (unsigned)c->sms);
-    k_catch_up<<<catch_grid, kCatchThreads, 0, st>>>(c->log, first, count, c->D_buf(q), c->blk_max(q), c->cfg.n);
+    PacketLog lg = c->log;
+    lg.bnd = c->log.bnd + (size_t)gen * c->log.ranges;
+    k_catch_up<<<catch_grid, kCatchThreads, 0, st>>>(lg, first, count, c->D_buf(q), c->blk_max(q), c->cfg.n);
     DGS_CUDA(c, cudaGetLastError());
     c->launches += 1;
+    first = end;
   }
   c->applied[q] = c->log_head;
   return DGS_OK;
@@ -511,7 +539,12 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age
   }
   {
     TimedLaunch t(c, st, MODE == kPull ? DGS_KERNEL_STREAM_PULL : DGS_KERNEL_STREAM_PUSH);
-    k_stream<MODE><<<c->stream_grid[MODE], kThreads, StreamRing<MODE>::kBytes, st>>>(ws, a);
+    // A pull in a context with several workers shares the GPU with the push passes of later events and reads
+    // only a small part of D_w: it takes the form of the pass that holds no ring of stages.
+    if (MODE == kPull && c->light_pull)
+      k_pull_light<<<c->stream_grid[MODE], kThreads, 0, st>>>(ws, a);
+    else
+      k_stream<MODE><<<c->stream_grid[MODE], kThreads, StreamRing<MODE>::kBytes, st>>>(ws, a);
     DGS_CUDA(c, cudaGetLastError());
     c->launches += 1;
   }
@@ -632,6 +665,9 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   }
   c->pull_count = c->event_count = 0;
   c->log_head = 0;
+  c->last_ranges = 0;
+  c->cur_gen = 0;
+  c->gen_last[0] = c->gen_last[1] = -1;
   c->applied.assign(cfg->num_workers, 0);
   c->kind_seq[0] = c->kind_seq[1] = 0;
   c->res.assign(ResIds{cfg->num_workers}.count(), dgs_ctx::Res());
@@ -677,6 +713,11 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   INIT_CUDA(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
   if (!coop) return fail(DGS_ECUDA);
   c->sms = sms;
+#ifdef DGS_NO_LIGHT_PULL
+  c->light_pull = false;
+#else
+  c->light_pull = cfg->num_workers > 1;
+#endif
   if (occupancy_grids<kPushSam>(c, sms) != DGS_OK || occupancy_grids<kPushResidual>(c, sms) != DGS_OK ||
       occupancy_grids<kPull>(c, sms) != DGS_OK)
     return fail(DGS_ECUDA);
@@ -782,6 +823,7 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   c->log.bnd = c->at<uint32_t>(L.log_bnd);
   c->log.pos = c->at<uint32_t>(L.log_pos);
   c->log.ranges = L.log_ranges;
+  c->slot_gen.assign(L.log_ring, 0);
   *out = c;
   return DGS_OK;
 }
@@ -841,15 +883,6 @@ int apply_impl(dgs_ctx* c, uint32_t worker, const dgs_packet* pkt) {
     // Its slot of the log still holds the packet filed `ring` applies ago; whoever has not folded that
     // one in yet does so first.
     const uint32_t lslot = (uint32_t)(c->log_head % c->log.ring);
-    // The ranges of the log are taken from the first packet filed, again from packet N (velocities have
-    // built up by then) and then every 16 N packets, so that they follow a drifting distribution.  The
-    // positions filed with older packets refer to the old ranges: nobody may still need those packets.
-    const bool new_ranges = c->log_head == 0 || c->log_head == N || c->log_head % (16ull * N) == 0;
-    if (new_ranges)
-      for (uint32_t q = 0; q < N; ++q) {
-        const int rc = catch_up_now(c, q);
-        if (rc != DGS_OK) return rc;
-      }
     if (c->log_head >= c->log.ring) {
       const uint64_t oldest = c->log_head - c->log.ring;
       for (uint32_t q = 0; q < N; ++q)
@@ -858,24 +891,52 @@ int apply_impl(dgs_ctx* c, uint32_t worker, const dgs_packet* pkt) {
           if (rc != DGS_OK) return rc;
         }
     }
+    // The ranges of the log are taken from the first packet filed, again from packet N (velocities have
+    // built up by then) and then every few rounds of the workers, so that they follow a drifting
+    // distribution.  Packets keep the positions they were filed with: the ranges come in two generations,
+    // a packet's slot remembers which one its positions refer to, and a catch-up folds the packets of the
+    // older generation before those of the newer one.  A generation is overwritten only when every packet
+    // filed under it has left the ring, so nobody has to catch up for the ranges to change.
+    const uint64_t period = std::max<uint64_t>(16ull * N, 2ull * c->log.ring);
+    const bool new_ranges = c->log_head == 0 || (c->log_head == N && c->last_ranges == 0) ||
+                            c->log_head >= c->last_ranges + period;
+    if (new_ranges) {
+      if (c->log_head > 0) {
+        // the other generation is taken over: whoever still has to fold in one of its packets (a worker that
+        // stayed away for very long) does so first
+        const int other = c->cur_gen ^ 1;
+        for (uint32_t q = 0; q < N; ++q)
+          if ((int64_t)c->applied[q] <= c->gen_last[other]) {
+            const int rc = catch_up_now(c, q);
+            if (rc != DGS_OK) return rc;
+          }
+        c->cur_gen = other;
+      }
+      c->last_ranges = c->log_head;
+    }
+    c->gen_last[c->cur_gen] = (int64_t)c->log_head;
+    c->slot_gen[lslot] = (uint8_t)c->cur_gen;
+    PacketLog lg = c->log;
+    lg.bnd = c->log.bnd + (size_t)c->cur_gen * c->log.ranges;
     Task t;
     t.stream = kStApply;
     t.reads.push_back(R.PKT(slot));
     t.writes = {R.THETA(), R.LOG(lslot)};
-    if (new_ranges) t.writes.push_back(R.RANGES());
+    if (new_ranges) t.writes.push_back(R.RANGES(c->cur_gen));
+    else t.reads.push_back(R.RANGES(c->cur_gen));
     int rc = task_begin(c, t);
     if (rc != DGS_OK) return rc;
     {
       TimedLaunch tl(c, c->st[kStApply], DGS_KERNEL_SCATTER);
       if (new_ranges) {
-        k_log_ranges<<<(c->log.ranges + kThreads - 1) / kThreads, kThreads, 0, c->st[kStApply]>>>(pkt->idx, c->log);
+        k_log_ranges<<<(c->log.ranges + kThreads - 1) / kThreads, kThreads, 0, c->st[kStApply]>>>(pkt->idx, lg);
         DGS_CUDA(c, cudaGetLastError());
         c->launches += 1;
       }
       const uint32_t pos_ctas = (c->log.ranges + 1 + kThreads - 1) / kThreads;
       k_apply_log<<<gx + pos_ctas, kThreads, 0, c->st[kStApply]>>>(pkt->idx, pkt->val, pkt->count,
                                                                    c->at<float>(c->lay.theta), c->cfg.n,
-                                                                   c->ws[0].status, c->log, lslot, gx);
+                                                                   c->ws[0].status, lg, lslot, gx);
       DGS_CUDA(c, cudaGetLastError());
       c->launches += 1;
     }

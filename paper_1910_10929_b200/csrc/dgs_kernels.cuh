@@ -682,6 +682,178 @@ __device__ void stream_tiles_tma(const Workspace& ws, const SelArgs& a, const ui
   }
 }
 
+// ---- the pull's pass without a staging ring ------------------------------------------
+// A pull of one worker among many reads only the chunks of D_w whose block bounds admit a
+// candidate -- a small part of the vector, a few chunks per CTA -- while the push passes of
+// later events stream beside it and need the SMs' shared memory for their own rings.  This
+// form of the pass therefore holds no ring: a warp loads its tile of the next chunk to be read
+// straight into registers while the CTA finishes the chunk before, so one chunk is in flight
+// per CTA, and the CTA keeps only its histogram in shared memory.  Candidates, bounds, plan and
+// counters are exactly those of the staged form.
+__device__ __forceinline__ void load_tile_raw(const float* __restrict__ in, uint32_t start, int lane,
+                                              float (&x)[4 * kVecIters]) {
+  const float4* pa = reinterpret_cast<const float4*>(in + start) + lane;
+#pragma unroll
+  for (int j = 0; j < kVecIters; ++j) {
+    const float4 v = __ldcs(pa + j * 32);
+    x[4 * j + 0] = v.x;
+    x[4 * j + 1] = v.y;
+    x[4 * j + 2] = v.z;
+    x[4 * j + 3] = v.w;
+  }
+}
+
+__device__ void pull_tiles_light(const Workspace& ws, const SelArgs& a, const uint32_t* Larr,
+                                 const float* __restrict__ in, uint32_t cta, uint32_t G, StreamShared& sh) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t t0 = part_first_tile(cta, G, ws.num_tiles), t1 = part_first_tile(cta + 1, G, ws.num_tiles);
+  if (ws.plan != nullptr && ld_volatile(ws.sync + kPlanParts) == G && __ldcg(ws.plan + G) == ws.num_tiles) {
+    // boundaries planned by the finalize of the previous selection on this scratch set
+    t0 = __ldcg(ws.plan + cta);
+    t1 = __ldcg(ws.plan + cta + 1);
+  }
+  uint32_t live_read = 0;   // thread 0: chunks this part reads
+  const uint32_t lt = lanemask_lt();
+  for (int b = threadIdx.x; b < kBins1; b += kThreads) sh.hist[b] = 0;
+  if (threadIdx.x == 0) {
+    sh.cursor = 0;
+    if (cta == 0) ws.sync[kParts] = G;
+  }
+  __syncthreads();
+  if (t0 >= t1) {
+    if (threadIdx.x == 0) {
+      ws.part_cands[cta] = 0;
+      ws.part_slot0[cta] = 0;
+      if (ws.part_live != nullptr) ws.part_live[cta] = 0;
+    }
+    return;
+  }
+  const uint32_t slot0 = ws.tiles[t0].start;
+  const uint32_t seg_first = ws.tiles[t0].seg, seg_last = ws.tiles[t1 - 1].seg;
+  uint32_t cur = 0;     // candidates appended so far (same in every thread)
+  uint32_t round = 0;
+  for (uint32_t s = seg_first; s <= seg_last; ++s) {
+    const uint32_t a0 = max(t0, ws.segs[s].tile_begin), a1 = min(t1, ws.segs[s].tile_end);
+    const uint32_t L = Larr[s];
+    const bool head = ws.tiles[a0].len != kWarpTile;
+    const bool tail = (a1 - 1 > a0 || !head) && ws.tiles[a1 - 1].len != kWarpTile;
+    const uint32_t f0 = a0 + (head ? 1u : 0u), f1 = a1 - (tail ? 1u : 0u);   // full tiles [f0, f1)
+    auto ragged = [&](uint32_t t) {
+      if (warp == 0) {
+        const Tile tile = ws.tiles[t];
+        float x[kRaggedSteps];
+        const uint32_t flags = ragged_mask<kPull>(a, tile, L, lane, in, nullptr, x);
+        const uint32_t count = __reduce_add_sync(kFull, (uint32_t)__popc(flags));
+        ragged_emit(ws, sh, tile, flags, slot0 + cur, lane, lt, x);
+        if (lane == 0) sh.cursor = count;
+      }
+      __syncthreads();
+      cur += sh.cursor;
+      __syncthreads();
+    };
+    if (head) ragged(a0);
+    const uint32_t nfull = f1 > f0 ? f1 - f0 : 0;
+    const uint32_t nchunks = (nfull + kStageTiles - 1) / kStageTiles;
+    const uint32_t e0 = nfull ? ws.tiles[f0].start : 0;   // first element of the full tiles (multiple of kWarpTile)
+    // a chunk all of whose blocks have a bound below L holds no candidate and is not read
+    const bool can_skip = a.blk_max != nullptr && L > 0 && nchunks <= kLiveWords * 32;
+    if (can_skip) {
+      for (uint32_t base = warp * 32; base < nchunks; base += kWarps * 32) {
+        const uint32_t c = base + lane;
+        bool live = false;
+        if (c < nchunks) {
+          const uint32_t tiles_here = min((uint32_t)kStageTiles, nfull - c * kStageTiles);
+          const uint32_t* bm = a.blk_max + e0 / kWarpTile + c * kStageTiles;
+          uint32_t top = 0;
+          if (tiles_here == kStageTiles && (reinterpret_cast<uintptr_t>(bm) & 15u) == 0) {
+            const uint4 q0 = __ldcg(reinterpret_cast<const uint4*>(bm)), q1 = __ldcg(reinterpret_cast<const uint4*>(bm) + 1);
+            top = max(max(max(q0.x, q0.y), max(q0.z, q0.w)), max(max(q1.x, q1.y), max(q1.z, q1.w)));
+          } else {
+            for (uint32_t j = 0; j < tiles_here; ++j) top = max(top, __ldcg(bm + j));
+          }
+          live = top >= L;
+        }
+        const uint32_t word = __ballot_sync(kFull, live);
+        if (lane == 0) sh.live[base / 32] = word;
+      }
+      __syncthreads();
+    }
+    auto next_live = [&](uint32_t c) -> uint32_t {       // first chunk >= c that is read, nchunks if none
+      while (can_skip && c < nchunks) {
+        const uint32_t w = sh.live[c >> 5] >> (c & 31);
+        if (w) return c + __ffs(w) - 1;
+        c = (c | 31u) + 1;
+      }
+      return min(c, nchunks);
+    };
+    if (threadIdx.x == 0 && nchunks) {     // bookkeeping: chunks of D_w that exist / that are read
+      uint32_t read = nchunks;
+      if (can_skip) {
+        read = 0;
+        for (uint32_t w = 0; w * 32 < nchunks; ++w) read += __popc(sh.live[w]);
+      }
+      atomicAdd(ws.stats + 3, (unsigned long long)nchunks);
+      atomicAdd(ws.stats + 4, (unsigned long long)read);
+      live_read += read;
+    }
+    float x[4 * kVecIters], xn[4 * kVecIters];
+    uint32_t c = next_live(0);
+    if (c < nchunks && c * kStageTiles + warp < nfull) load_tile_raw(in, e0 + (c * kStageTiles + warp) * kWarpTile, lane, x);
+    while (c < nchunks) {
+      const uint32_t cn = next_live(c + 1);
+      const uint32_t tl = c * kStageTiles + warp;          // this warp's tile among the full ones
+      const uint32_t tile_start = e0 + tl * kWarpTile;
+      uint32_t mask = 0;
+      if (tl < nfull) {
+        uint32_t top = 0;
+#pragma unroll
+        for (int e = 0; e < 4 * kVecIters; ++e) {
+          const uint32_t key = key_of(x[e]);
+          top = max(top, key);
+          if (key >= L) mask |= 1u << e;
+        }
+        if (a.blk_max != nullptr) {
+          // the tile is a whole block: its bound becomes exact again (entries sent later only lower it)
+          top = __reduce_max_sync(kFull, top);
+          if (lane == 0) a.blk_max[tile_start / kWarpTile] = top;
+        }
+      }
+      const uint32_t count = __reduce_add_sync(kFull, (uint32_t)__popc(mask));
+      if (lane == 0) sh.wcnt[round & 1][warp] = count;
+      // the next chunk is on its way while this one is written out
+      if (cn < nchunks && cn * kStageTiles + warp < nfull)
+        load_tile_raw(in, e0 + (cn * kStageTiles + warp) * kWarpTile, lane, xn);
+      __syncthreads();
+      uint32_t total;
+      const uint32_t base = slot0 + cur + round_offset(sh.wcnt[round & 1], warp, total);
+      cur += total;
+      if (tl < nfull)
+        tile_emit(ws, sh, tile_start, mask, base, lane, [&](uint32_t off) {
+          // element off = j*128 + lane*4 + c is register 4*j + c of this lane
+          const int e = (int)(((off >> 7) << 2) | (off & 3u));
+          float v = x[0];
+#pragma unroll
+          for (int q = 1; q < 4 * kVecIters; ++q)
+            if (q == e) v = x[q];
+          return v;
+        });
+#pragma unroll
+      for (int e = 0; e < 4 * kVecIters; ++e) x[e] = xn[e];
+      c = cn;
+      ++round;
+    }
+    __syncthreads();
+    if (tail) ragged(a1 - 1);
+    flush_hist(sh.hist, ws.hist1 + (size_t)s * kBins1);
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    ws.part_cands[cta] = cur;
+    ws.part_slot0[cta] = slot0;
+    if (ws.part_live != nullptr) ws.part_live[cta] = live_read;
+  }
+}
+
 // ---- histogram of ALL elements (top 11 key bits), for the bound that cannot fail ----
 // Adds one warp-wide batch of bins to the shared histogram.  Lanes holding the same
 // bin as lane 0's are counted with one ballot (values cluster in few bins: zeros in a
@@ -1375,6 +1547,16 @@ __global__ void __maxnreg__(64) k_stream(Workspace ws, SelArgs a) {
                          &s_dead);
 }
 
+// ---- the pull's stream pass in its ring-less form (contexts with several workers) -----
+#ifndef DGS_LIGHT_REGS
+#define DGS_LIGHT_REGS 64
+#endif
+__global__ void __maxnreg__(DGS_LIGHT_REGS) k_pull_light(Workspace ws, SelArgs a) {
+  __shared__ StreamShared sh;
+  if (blockIdx.x == 0 && threadIdx.x == 0) ws.sync[kBarCount] = 0;   // for the finalize launch that follows
+  pull_tiles_light(ws, a, a.L_in, a.D, blockIdx.x, gridDim.x, sh);
+}
+
 // ---- server apply ---------------------------------------------------------------
 // Algorithm 2 lowers theta and every D_q by the decoded packet.  D_q is read only by worker
 // q's pull, so the library keeps D_q lazily: an apply lowers theta at once and files the
@@ -1385,15 +1567,16 @@ __global__ void __maxnreg__(64) k_stream(Workspace ws, SelArgs a) {
 // instead of being scattered into all N vectors at once.
 //
 constexpr int kCatchMaxPackets = 64;     // most packets one k_catch_up launch folds in
-constexpr int kCatchCap = 2048;          // entries a CTA of k_catch_up can hold in shared memory
-constexpr int kCatchSlots = 4096;        // slots of its table of distinct indices (power of two, >= 2 * kCatchCap)
-constexpr uint32_t kCatchTarget = 1024;  // entries per CTA the launch aims at
-constexpr int kCatchMaxGrid = 8192;
-constexpr int kCatchBlocks = 256;        // blocks of D whose bounds a CTA of k_catch_up collects in shared memory first
-#ifndef DGS_CATCH_THREADS
-#define DGS_CATCH_THREADS 256
-#endif
-constexpr int kCatchThreads = DGS_CATCH_THREADS;   // threads per CTA of k_catch_up (>= 2 * kCatchMaxPackets)
+constexpr int kCatchCap = 1024;          // entries a CTA of k_catch_up can hold in shared memory (a power of two)
+constexpr int kCatchSlots = 2 * kCatchCap;        // sparse pieces: slots of the table of distinct indices (>= 2 * kCatchCap)
+constexpr int kCatchDense = 2 * kCatchSlots;      // dense pieces: elements of D a piece can mirror (= the bytes of the sparse table)
+constexpr int kCatchLines = kCatchDense / 32;
+constexpr uint32_t kCatchTarget = kCatchCap / 2;  // entries per range of the log the launch aims at
+constexpr int kCatchMaxGrid = 16384;
+constexpr int kCatchBlocks = kCatchCap / 8 < 16 ? 16 : kCatchCap / 8;   // blocks of D whose bounds a CTA of k_catch_up collects in shared memory first
+constexpr int catch_log2(int v) { return v <= 1 ? 0 : 1 + catch_log2(v / 2); }
+constexpr int kCatchSlotBits = catch_log2(kCatchSlots);
+constexpr int kCatchThreads = 256;       // threads per CTA of k_catch_up (>= 2 * kCatchMaxPackets)
 
 // Keeps a block's bound an upper bound on the magnitudes in the block.  Bounds only rise while
 // packets are being subtracted, so a bound already read as high enough needs no atomic.
@@ -1460,23 +1643,43 @@ __global__ void __launch_bounds__(kThreads) k_apply_log(const uint32_t* __restri
 
 // D -= packets first .. first + count - 1 of the log, in that order (count <= kCatchMaxPackets).
 // A CTA owns a range c of the log at a time; its part of every packet is known from the
-// positions filed with the packet.  It gathers the distinct indices of all those parts in a
-// shared-memory table, loads each D[i] once, subtracts the packets' values from the table in
-// packet order (indices inside one packet are distinct, so a packet is one parallel step) and
-// stores each D[i] once: every D[i] sees the same subtractions in the same order as if the
-// packets had been applied one by one, with one trip to memory instead of one per packet.  No two
-// CTAs touch the same entry of D.  A range with more entries than the table holds (later packets
-// much denser there than the one the ranges were taken from) is taken in several rounds, each over
-// a piece of the range (halved until its entries fit).
+// positions filed with the packet.  The values of D that the range's entries touch are brought
+// into shared memory once, the packets' values are subtracted there in packet order (indices
+// inside one packet are distinct, so a packet is one parallel step) and every value goes back
+// once: every D[i] sees the same subtractions in the same order as if the packets had been
+// applied one by one, with one trip to memory instead of one per packet.  No two CTAs touch the
+// same entry of D.  A range with more entries than the tables hold (later packets much denser
+// there than the one the ranges were taken from) is taken in several rounds, each over a piece
+// of the range (halved until its entries fit).
+//
+// Two ways to hold a piece's values of D:
+//   dense   the piece spans at most kCatchDense elements (counted from the 128-byte line its
+//           first element lies in): shared memory mirrors the piece, an entry's place is its
+//           offset.  Only the lines that hold an entry are read and written, each as one
+//           coalesced 128-byte access of a warp, so the number of memory requests is the number
+//           of lines touched, not the number of entries.  Where updates crowd -- the tensors
+//           with the largest gradients, which take most entries of every packet -- a line holds
+//           many entries.
+//   sparse  a wider piece: a table of the distinct indices, one load and one store per index.
 struct CatchShared {
-  uint32_t keys[kCatchSlots];            // index held by a slot, kFull = empty
-  float vals[kCatchSlots];               // running value of D at that index
-  uint16_t ent_slot[kCatchCap];          // slot of each entry (packet-major order), 0xFFFF = index out of range
+  union {
+    struct {
+      uint32_t keys[kCatchSlots];        // sparse: index held by a slot, kFull = empty
+      float vals[kCatchSlots];           //         running value of D at that index
+    } tab;
+    float dense[kCatchDense];            // dense: running values of D[a0 ..], a0 = first element of the piece's first line
+  };
+  uint16_t ent_slot[kCatchCap];          // place of each entry (packet-major order), 0xFFFF = index out of range
   float ent_val[kCatchCap];
   uint32_t lo[kCatchMaxPackets], hi[kCatchMaxPackets], end[kCatchMaxPackets];   // per packet: piece, end of the range
   uint32_t pre[kCatchMaxPackets + 1];    // exclusive prefix of hi - lo
   uint32_t bmax[kCatchBlocks];           // largest new magnitude per block of kWarpTile elements, from the piece's first block on
+  uint32_t dirty[kCatchLines / 4];       // dense: one byte per line, nonzero = the line holds an entry
 };
+static_assert(sizeof(float) * kCatchDense == (sizeof(uint32_t) + sizeof(float)) * kCatchSlots, "the two views share their bytes");
+static_assert(kCatchDense <= 0xFFFF && kCatchDense % kCatchThreads == 0 && kCatchThreads % 32 == 0 &&
+              kCatchThreads >= 2 * kCatchMaxPackets, "offsets fit the entry table");
+static_assert(kCatchDense / kWarpTile + 2 <= kCatchBlocks, "a dense piece's blocks fit the table of bounds");
 
 __global__ void __launch_bounds__(kCatchThreads) k_catch_up(PacketLog lg, uint64_t first, uint32_t count,
                                                        float* __restrict__ D, uint32_t* __restrict__ blk_max,
@@ -1484,6 +1687,7 @@ __global__ void __launch_bounds__(kCatchThreads) k_catch_up(PacketLog lg, uint64
   __shared__ CatchShared sh;
   const uint32_t tid = threadIdx.x;
   if (count == 0 || count > (uint32_t)kCatchMaxPackets) return;
+  uint8_t* const dirty = reinterpret_cast<uint8_t*>(sh.dirty);
   // a CTA takes the ranges blockIdx.x, blockIdx.x + gridDim.x, ... one after the other
   for (uint32_t c = blockIdx.x; c < lg.ranges; c += gridDim.x) {
   if (tid < 2 * count) {
@@ -1495,8 +1699,8 @@ __global__ void __launch_bounds__(kCatchThreads) k_catch_up(PacketLog lg, uint64
   const uint32_t range_b = c + 1 == lg.ranges ? (uint32_t)n : __ldcg(lg.bnd + c + 1);   // n < 2^32
   uint32_t a = c == 0 ? 0u : __ldcg(lg.bnd + c);
   for (;;) {   // one round per piece [a, b) of the range; everything here is uniform over the CTA
-    for (int s = tid; s < kCatchSlots; s += kCatchThreads) sh.keys[s] = kFull;
     for (int s = tid; s < kCatchBlocks; s += kCatchThreads) sh.bmax[s] = 0;
+    for (int s = tid; s < kCatchLines / 4; s += kCatchThreads) sh.dirty[s] = 0;
     __syncthreads();
     if (tid < count) sh.hi[tid] = sh.end[tid];
     uint32_t b = range_b;
@@ -1536,7 +1740,14 @@ __global__ void __launch_bounds__(kCatchThreads) k_catch_up(PacketLog lg, uint64
       }
     }
     if (E > 0 && E <= (uint32_t)kCatchCap) {
-      // gather: entry e (packet-major) -> its index and value; the index gets a slot of the table
+      const uint32_t a0 = a & ~31u;                         // first element of the line that holds a
+      const uint32_t span = b - a0;                         // b <= n
+      const bool dense = span <= (uint32_t)kCatchDense;
+      if (!dense) {
+        for (int s = tid; s < kCatchSlots; s += kCatchThreads) sh.tab.keys[s] = kFull;
+        __syncthreads();
+      }
+      // gather: entry e (packet-major) -> its index and value; the index gets a place in shared memory
       constexpr int PER = kCatchCap / kCatchThreads;
       uint32_t ei[PER];
       float ev[PER];
@@ -1562,55 +1773,100 @@ __global__ void __launch_bounds__(kCatchThreads) k_catch_up(PacketLog lg, uint64
         if (e < E) {
           uint32_t slot = 0xFFFFu;
           const uint32_t i = ei[u];
-          if (i < n) {
-            uint32_t h = (i * 2654435761u) >> 20;   // top 12 bits: kCatchSlots = 4096
-            for (;;) {
-              const uint32_t old = atomicCAS(sh.keys + h, kFull, i);
-              if (old == kFull || old == i) break;
-              h = (h + 1) & (kCatchSlots - 1);
+          if (i < n && i >= a && i < b) {       // entries of a piece lie inside it; anything else is left alone
+            if (dense) {
+              slot = i - a0;
+              dirty[slot >> 5] = 1;
+            } else {
+              uint32_t h = (i * 2654435761u) >> (32 - kCatchSlotBits);   // the top bits of the product
+              for (;;) {
+                const uint32_t old = atomicCAS(sh.tab.keys + h, kFull, i);
+                if (old == kFull || old == i) break;
+                h = (h + 1) & (kCatchSlots - 1);
+              }
+              slot = h;
             }
-            slot = h;
           }
           sh.ent_slot[e] = (uint16_t)slot;
           sh.ent_val[e] = ev[u];
         }
       }
       __syncthreads();
-      // one load of D per distinct index, all in flight together
-      constexpr int SPT = kCatchSlots / kCatchThreads;
-      {
+      float* const cur = dense ? sh.dense : sh.tab.vals;    // running values, by place
+      constexpr int SPT = kCatchSlots / kCatchThreads;      // sparse: table slots per thread
+      constexpr int EPT = kCatchDense / kCatchThreads;      // dense: elements per thread, element tid + j * kCatchThreads
+      constexpr int LB = EPT < 8 ? EPT : 8;                  // loads a thread has in flight together
+      if (dense) {
+        // a warp's 32 threads hold one line at every step j: one 128-byte request per line that holds an entry
+#pragma unroll 1
+        for (int j0 = 0; j0 < EPT; j0 += LB) {
+          if ((uint32_t)(j0 * kCatchThreads) >= span) break;
+          float d[LB];
+#pragma unroll
+          for (int j = 0; j < LB; ++j) {
+            const uint32_t off = tid + (j0 + j) * kCatchThreads;
+            d[j] = 0.f;
+            if (off < span && dirty[off >> 5]) d[j] = __ldcg(D + a0 + off);
+          }
+#pragma unroll
+          for (int j = 0; j < LB; ++j) sh.dense[tid + (j0 + j) * kCatchThreads] = d[j];
+        }
+      } else {
+        // one load of D per distinct index, all in flight together
         uint32_t k[SPT];
         float d[SPT];
 #pragma unroll
         for (int u = 0; u < SPT; ++u) {
-          k[u] = sh.keys[tid + u * kCatchThreads];
+          k[u] = sh.tab.keys[tid + u * kCatchThreads];
           d[u] = 0.f;
           if (k[u] != kFull) d[u] = __ldcg(D + k[u]);
         }
 #pragma unroll
         for (int u = 0; u < SPT; ++u)
-          if (k[u] != kFull) sh.vals[tid + u * kCatchThreads] = d[u];
+          if (k[u] != kFull) sh.tab.vals[tid + u * kCatchThreads] = d[u];
       }
       __syncthreads();
-      // the packets in arrival order; inside one packet every index, and so every slot, occurs once
+      // the packets in arrival order; inside one packet every index, and so every place, occurs once
       for (uint32_t p = 0; p < count; ++p) {
         for (uint32_t e = sh.pre[p] + tid; e < sh.pre[p + 1]; e += kCatchThreads) {
           const uint32_t slot = sh.ent_slot[e];
-          if (slot != 0xFFFFu) sh.vals[slot] = __fsub_rn(sh.vals[slot], sh.ent_val[e]);
+          if (slot != 0xFFFFu) cur[slot] = __fsub_rn(cur[slot], sh.ent_val[e]);
         }
         __syncthreads();
       }
+      // Back to memory.  The blocks' bounds must stay upper bounds: the largest new magnitude per block is
+      // collected in shared memory, one global atomic per block afterwards.
+      if (dense) {
+        const uint32_t lead = a - a0;            // elements of the first line that belong to the range before
+        const uint32_t blk0 = a / kWarpTile;
+#pragma unroll 1
+        for (int j = 0; j < EPT; ++j) {
+          const uint32_t off = tid + j * kCatchThreads;
+          if ((uint32_t)(j * kCatchThreads) >= span) break;
+          const bool live = off < span && dirty[off >> 5] != 0;    // the same for the whole warp but for off < span
+          uint32_t key = 0;
+          if (live && off >= lead) {
+            const float r = sh.dense[off];
+            __stcg(D + a0 + off, r);
+            key = key_of(r);
+          }
+          if (__any_sync(kFull, live)) {
+            key = __reduce_max_sync(kFull, key);
+            // a line lies inside one block (lines and blocks start at multiples of 32 and of kWarpTile)
+            if ((tid & 31u) == 0 && key) atomicMax(sh.bmax + ((a0 + off) / kWarpTile - blk0), key);
+          }
+        }
+      } else {
 #pragma unroll
-      for (int u = 0; u < SPT; ++u) {
-        const uint32_t i = sh.keys[tid + u * kCatchThreads];
-        if (i != kFull) {
-          const float r = sh.vals[tid + u * kCatchThreads];
-          __stcg(D + i, r);
-          // keeps the block's bound an upper bound: collected per block in shared memory, one global
-          // atomic per block afterwards (a piece spanning more blocks than fit sends the rest directly)
-          const uint32_t blk = i / kWarpTile - a / kWarpTile;
-          if (blk < (uint32_t)kCatchBlocks) atomicMax(sh.bmax + blk, key_of(r));
-          else atomicMax(blk_max + i / kWarpTile, key_of(r));
+        for (int u = 0; u < SPT; ++u) {
+          const uint32_t i = sh.tab.keys[tid + u * kCatchThreads];
+          if (i != kFull) {
+            const float r = sh.tab.vals[tid + u * kCatchThreads];
+            __stcg(D + i, r);
+            const uint32_t blk = i / kWarpTile - a / kWarpTile;
+            if (blk < (uint32_t)kCatchBlocks) atomicMax(sh.bmax + blk, key_of(r));
+            else atomicMax(blk_max + i / kWarpTile, key_of(r));   // a piece spanning more blocks than the table holds
+          }
         }
       }
       __syncthreads();
@@ -1620,7 +1876,7 @@ __global__ void __launch_bounds__(kCatchThreads) k_catch_up(PacketLog lg, uint64
       }
     }
     if (b == range_b) break;
-    __syncthreads();   // the table and the pieces are read until here
+    __syncthreads();   // the tables and the pieces are read until here
     if (tid < count) sh.lo[tid] = sh.hi[tid];
     a = b;
   }

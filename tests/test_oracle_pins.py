@@ -72,12 +72,13 @@ def _read_golden(path):
     return head, events
 
 
-@pytest.mark.parametrize("name", ["hand_example.txt", "hand_example_algorithm1.txt"])
+@pytest.mark.parametrize("name", ["hand_example.txt", "hand_example_algorithm1.txt", "hand_example_full_pull.txt"])
 def test_hand_example(name):
     head, events = _read_golden(os.path.join(GOLDEN, name))
     n, N, k = int(head["n"][0]), int(head["workers"][0]), int(head["k"][0])
     theta0 = np.array([float(v) for v in head["theta0"]], np.float32)
     residual = head.get("mode", ["momentum"])[0] == "residual"       # worker rule of Algorithm 1
+    full_pull = head.get("mode", ["momentum"])[0] == "full_pull"     # Algorithm 2 without secondary compression
     o = oracle.Oracle(n, N, float(head["lr"][0]), float(head["momentum"][0]),
                       [0], [n], [k], [k], theta0, keep_local=True, residual_mode=residual)
     assert o.timestamp == 0 and [o.prev(q) for q in range(N)] == [-1] * N
@@ -90,7 +91,11 @@ def test_hand_example(name):
         assert list(o.state(oracle.THETA)) == list(ev["theta"])
         assert list(o.state(oracle.D, 0)) == list(ev["D0_after_apply"])
         assert list(o.state(oracle.D, 1)) == list(ev["D1_after_apply"])
-        gi, gv = o.pull(w)
+        if full_pull:
+            gi, gv, held = o.pull_all(w)
+            assert held == len(gi)
+        else:
+            gi, gv = o.pull(w)
         assert list(gi) == list(ev["pull_idx"]) and list(gv) == list(ev["pull_val"])
         assert list(o.state(oracle.D, 0)) == list(ev["D0"])
         assert list(o.state(oracle.D, 1)) == list(ev["D1"])
@@ -218,6 +223,34 @@ def test_piecewise_state_and_exact_split(residual_mode):
             assert np.allclose(o.state(oracle.THETA_LOCAL, q) + o.state(oracle.D, q),
                                o.state(oracle.THETA), rtol=0, atol=1e-6)
     assert o.timestamp == wl.num_events
+
+
+# ---- pull without secondary compression: v_k = M afterwards (Eq. 4), theta_k = theta (Eq. 5) ----
+def test_full_pull_sends_every_nonzero_and_leaves_nothing():
+    wl = W.custom("mini", [300, 7, 1000, 64], 3, 12, 20_000, grad_kind="normal", grad_scale=1e-2)
+    o = oracle.Oracle.from_workload(wl, keep_local=True)
+    for e, w in enumerate(wl.schedule()):
+        w = int(w)
+        pi, pv = o.push(w, wl.gradient(e))
+        o.apply(w, pi, pv)
+        Dw = o.state(oracle.D, w).copy()
+        gi, gv, held = o.pull_all(w)
+        nz = np.nonzero(Dw)[0]
+        assert held == len(nz) and np.array_equal(gi, nz.astype(np.uint32)) and np.array_equal(gv, Dw[nz])
+        assert not o.state(oracle.D, w).any()                                   # Eq. 4: v_k = M
+        # Eq. 5: the worker's model is the global one, up to the rounding of summing differences
+        assert np.allclose(o.state(oracle.THETA_LOCAL, w), o.state(oracle.THETA), rtol=0, atol=1e-6)
+        assert o.prev(w) == o.timestamp
+    # overflow: a capacity below the number of nonzeros sends the first `cap` and keeps the rest
+    pi, pv = o.push(0, wl.gradient(99))
+    o.apply(0, pi, pv)
+    Dw = o.state(oracle.D, 1).copy()
+    nz = np.nonzero(Dw)[0]
+    assert len(nz) > 3
+    gi, gv, held = o.pull_all(1, cap=3)
+    assert held == len(nz) and list(gi) == list(nz[:3])
+    left = o.state(oracle.D, 1)
+    assert not left[nz[:3]].any() and np.array_equal(left[nz[3:]], Dw[nz[3:]])
 
 
 def test_fewer_nonzeros_than_k_fills_with_lowest_zero_indices():

@@ -217,54 +217,6 @@ def test_selection_with_many_candidates_per_thread():
     assert not left[want].any()
 
 
-def test_gpt2_small_32_workers_properties_at_full_size():
-    """Config 4 in the launch configuration the benchmark times (124.4 M parameters, 32 workers,
-    one global 0.1 % selection), too large for the CPU checker to follow within a test: what must
-    hold at any size is checked with plain tensor operations on the device instead.  Every
-    packet has exactly K strictly ascending indices; a pull sends the largest magnitudes of D_w
-    and clears them (Eq. 6a/6b), a push leaves u = t on the sent entries (Eq. 12); the model equals
-    theta_0 minus all applied packets (Eq. 2)."""
-    wl = W.gpt2_small(num_workers=32, num_events=40)
-    dev = torch.device(DEV)
-    theta0 = torch.from_numpy(wl.theta0()).to(dev)
-    ctx = dgs.Context.from_workload(wl, theta0=theta0)
-    sched = wl.schedule()
-    applied = torch.zeros(wl.n, dtype=torch.float64, device=dev)
-    K = wl.K_push
-    for e in range(wl.num_events):
-        w = int(sched[e])
-        g = torch.from_numpy(wl.gradient(e)).to(dev)
-        check = e % 8 == 7 or e < 2          # the full checks need the state on the host side of the stream
-        pkt = ctx.worker_push(w, g)
-        idx, val = (t.clone() for t in ctx.packet(pkt))
-        idx = idx.to(torch.int64) & 0xFFFFFFFF
-        assert idx.numel() == K and bool((idx[1:] > idx[:-1]).all()) and int(idx[-1]) < wl.n
-        applied.index_add_(0, idx, val.to(torch.float64))
-        if check:
-            u = ctx.state(dgs.DGS_U, w)
-            assert torch.equal(u[idx], val)                                  # sent entries keep t
-            rest = u.abs() * wl.momentum                                     # unsent entries hold t / m
-            rest[idx] = 0
-            assert float(rest.max()) <= float(val.abs().min()) * (1 + 1e-6)  # nothing larger was left behind
-        ctx.server_apply(w, pkt)
-        before = ctx.state(dgs.DGS_D, w).clone() if check else None
-        pull = ctx.worker_pull(w)
-        gi, gv = (t.clone() for t in ctx.packet(pull))
-        gi = gi.to(torch.int64) & 0xFFFFFFFF
-        assert gi.numel() == wl.K_pull and bool((gi[1:] > gi[:-1]).all()) and int(gi[-1]) < wl.n
-        if check:
-            after = ctx.state(dgs.DGS_D, w)
-            assert torch.equal(before[gi], gv)                               # sent values are D_w's own
-            assert not bool(after[gi].any())                                 # and are cleared
-            before[gi] = 0
-            assert torch.equal(before, after)                                # the rest is retained as it was
-            assert float(after.abs().max()) <= float(gv.abs().min())         # nothing larger was left behind
-    theta = ctx.state(dgs.DGS_THETA).to(torch.float64)
-    err = (theta - (theta0.to(torch.float64) - applied)).abs().max()
-    assert float(err) <= 1e-6 * float(theta0.abs().max())
-    assert ctx.status() == 0
-
-
 def test_trajectory_gpt2_small_few_workers():
     wl = W.gpt2_small(num_workers=3, num_events=7)
     replay_and_compare(wl)
