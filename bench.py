@@ -41,10 +41,40 @@ import workloads as W  # noqa: E402
 METRIC = "push+apply+pull events/sec"
 UNIT = "events/s"
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
-# profiles/ (same n, so the same bytes per launch); None for kernels or workloads not captured
-NCU_TRAFFIC = {("resnet50-global", "stream_push"): 204552960 + 58023168}
 FALLBACK_HBM_GBS = 6650.0
+# ncu DRAM traffic of the dominant kernel: read from the tracked summary of the capture, which names the
+# source state it was taken at; no number is reported once the kernel's source has changed since
+TRAFFIC_SUMMARY = os.path.join(ROOT, "profiles", "k_stream_push_resnet50_traffic.txt")
+KERNEL_SOURCE = os.path.join(ROOT, "paper_1910_10929_b200", "csrc", "dgs_kernels.cuh")
+
+
+def stream_pass_source_hash() -> str:
+    """Hash of the part of the kernel source that makes up the stream pass (everything up to the
+    histogram pass), so that edits to other kernels of the same file do not invalidate the capture."""
+    import hashlib
+    with open(KERNEL_SOURCE) as f:
+        text = f.read()
+    cut = text.find("// ---- histogram of ALL elements")
+    return hashlib.sha256(text[:cut if cut > 0 else len(text)].encode()).hexdigest()[:16]
+
+
+def ncu_traffic(workload: str, kernel: str):
+    """(bytes per launch, note) from the tracked summary if it covers this workload and kernel and was
+    captured from the present source of the stream pass; else (None, why)."""
+    try:
+        fields = {}
+        with open(TRAFFIC_SUMMARY) as f:
+            for line in f:
+                if ":" in line and not line.startswith("#"):
+                    k, v = line.split(":", 1)
+                    fields[k.strip()] = v.strip()
+        if fields.get("workload") != workload or fields.get("kernel") != kernel:
+            return None, "no capture for this workload and kernel"
+        if fields.get("stream_pass_source_hash") != stream_pass_source_hash():
+            return None, "the stream pass has changed since the capture"
+        return int(fields["dram_bytes_per_launch"]), f"ncu capture at commit {fields.get('commit', '?')}"
+    except Exception as e:           # no summary, or one that does not parse
+        return None, f"no usable capture summary ({type(e).__name__})"
 
 
 def make_workload(name: str, seed: int, workers: int = 0):
@@ -53,6 +83,22 @@ def make_workload(name: str, seed: int, workers: int = 0):
     if workers:
         return W.BY_NAME[name](seed=seed, num_workers=workers)
     return W.BY_NAME[name](seed=seed)
+
+
+def preroll_events(wl) -> int:
+    return wl.num_workers if wl.schedule_kind == "cyclic" else 2 * wl.num_workers
+
+
+def config_of(wl, args, world: int = 1) -> dict:
+    """The `config` object both arms print: the workload and the parameters of the run, the same keys
+    and values in both, so that the two lines can be matched."""
+    K, Wm, R = args.steps, args.warmup, max(1, args.windows)
+    return {"workload": wl.name, "n": wl.n, "workers": wl.num_workers, "K_push": wl.K_push, "K_pull": wl.K_pull,
+            "segments": wl.num_segments, "lr": wl.lr, "momentum": wl.momentum, "seed": wl.seed,
+            "schedule": wl.schedule_kind, "preroll_events": preroll_events(wl),
+            "distinct_gradients": min(preroll_events(wl) + Wm + (R + 1) * K, args.grad_pool),
+            "l2": "inputs larger than L2: every event reads a different gradient, velocity and difference vector",
+            "replicas": world, "windows": R}
 
 
 def algorithmic_bytes_per_event(n: int, K_push: int, K_pull: int, N: int) -> dict:
@@ -183,8 +229,7 @@ def run_reference(args, wl) -> dict:
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": done, "warmup": Wm_eff, "ms_per_step": 1e3 * elapsed / done, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": wl.name, "n": wl.n, "workers": wl.num_workers, "K_push": wl.K_push,
-                   "K_pull": wl.K_pull, "seed": wl.seed},
+        "config": config_of(wl, args, 1),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -230,9 +275,10 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
     dev = torch.device("cuda", local_rank)
     N = wl.num_workers
     sched_full = wl.schedule()
-    preroll = N if wl.schedule_kind == "cyclic" else 2 * N
+    preroll = preroll_events(wl)
     K, Wm = args.steps, args.warmup
-    total_events = preroll + Wm + 2 * K          # timed pass + per-kernel timing pass
+    R = max(1, args.windows)                     # timed windows of K events each, back to back
+    total_events = preroll + Wm + (R + 1) * K    # timed windows + per-kernel timing pass
     pool = min(total_events, args.grad_pool)
     sched = np.resize(sched_full, total_events)
 
@@ -258,6 +304,7 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
             dist.barrier()
         torch.cuda.synchronize(dev)
 
+    window_s = []
     with ClockSampler(local_rank) as clocks:
         run_events(0, preroll)
         run_events(preroll, Wm)
@@ -265,18 +312,20 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
         stats0 = ctx.stats()
         reads0 = ctx.pull_read_stats()
         launches0 = ctx.launch_count()
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
         t_begin = time.perf_counter()
-        ev0.record(stream)
-        run_events(preroll + Wm, K)
-        ctx.flush()
-        ev1.record(stream)
-        barrier()
+        for r in range(R):
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            barrier()
+            ev0.record(stream)
+            run_events(preroll + Wm + r * K, K)
+            ctx.flush()
+            ev1.record(stream)
+            barrier()
+            window_s.append(ev0.elapsed_time(ev1) * 1e-3)
         t_end = time.perf_counter()
     clocks.window(t_begin, t_end)
-    elapsed = ev0.elapsed_time(ev1) * 1e-3
-    launches = ctx.launch_count() - launches0
+    elapsed = statistics.median(window_s)         # of the R windows of exactly K events each
+    launches = (ctx.launch_count() - launches0) // R
     stats1 = ctx.stats()
     reads1 = ctx.pull_read_stats()
     assert ctx.status() == 0, "device status word is not clean"
@@ -284,7 +333,7 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
 
     # per-kernel device time, same loop continued, events around each launch
     dgs.dgs_timing_enable(ctx.handle, True)
-    run_events(preroll + Wm + K, K)
+    run_events(preroll + Wm + R * K, K)
     ktimes = dgs.dgs_timing_read(ctx.handle)
     dgs.dgs_timing_enable(ctx.handle, False)
 
@@ -292,7 +341,7 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
     Ke = min(K, len(host), 16)
     out_idx = torch.empty(wl.K_pull, dtype=torch.int32).pin_memory()
     out_val = torch.empty(wl.K_pull, dtype=torch.float32).pin_memory()
-    first = preroll + Wm + 2 * K
+    first = preroll + Wm + (R + 1) * K
     sched_e = np.resize(sched_full, first + Ke + 3)
     for j in range(3):
         ctx.event_host(int(sched_e[first + j]), host[j % len(host)], out_idx, out_val)
@@ -349,19 +398,16 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
             return ab["apply"] * K / ((ms + ktimes["scatter"][0]) * 1e-3) / 1e9
         return kernel_bytes[k] / (ms * 1e-3 / cnt) / 1e9 if kernel_bytes[k] else None
 
-    traffic = args.traffic_bytes
-    if traffic is None:
-        traffic = NCU_TRAFFIC.get((wl.name, dom))
+    traffic, traffic_note = ncu_traffic(wl.name, dom)
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": 1e3 * elapsed_max / K, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": wl.name, "n": wl.n, "workers": N, "K_push": wl.K_push, "K_pull": wl.K_pull,
-                   "segments": wl.num_segments, "lr": wl.lr, "momentum": wl.momentum, "seed": wl.seed,
-                   "preroll_events": preroll, "distinct_gradients": pool,
-                   "l2": "inputs larger than L2: every event reads a different gradient, velocity and "
-                         "difference vector", "replicas": world,
-                   "cuda_device_max_connections": os.environ.get("CUDA_DEVICE_MAX_CONNECTIONS")},
+        "config": config_of(wl, args, world),
+        "cuda_device_max_connections": os.environ.get("CUDA_DEVICE_MAX_CONNECTIONS"),
+        "windows": {"count": R, "events_each": K, "ms_per_step": [1e3 * t / K for t in window_s],
+                    "spread": (max(window_s) - min(window_s)) / elapsed if elapsed > 0 else None,
+                    "note": "value and ms_per_step are those of the median window"},
         "effective_hbm": {"algorithmic_bytes_per_event": ab, "GB/s": eff_gbs,
                           "frac_of_nominal_8TBs": eff_gbs / NOMINAL_HBM_GBS, "frac_of_peak": eff_gbs / peak,
                           "peak_GB/s": peak, "peak_kind": peak_kind},
@@ -379,6 +425,7 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
                                   for k, (ms, c) in stimes.items()},
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": peak_kind, "traffic": traffic,
+                     "traffic_note": traffic_note,
                      "algorithmic_bytes_per_launch": kernel_bytes[dom],
                      "achieved_overlapped": achieved_ovl, "frac_overlapped": achieved_ovl / peak,
                      "whole_event_frac": eff_gbs / peak,
@@ -392,9 +439,44 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
         "gpu_launches": launches,
         "clocks": clocks.summary(),
     }
+    if world == 1 and N > 1 and not args.no_jitter:
+        out["jittered_arrivals"] = run_jittered(wl, grads, pool, theta0, min(K, 512), dev)
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(wl, args.cpu_seconds)
     return out
+
+
+def run_jittered(wl, grads, pool, theta0, K, dev) -> dict:
+    """The same workload with an irregular arrival order: every event is served for a worker drawn
+    independently and uniformly (a worker may return at once or stay away for long), so the bounds
+    carried from earlier selections fit less often.  Reports the rate and which route the selections took."""
+    import torch
+
+    import paper_1910_10929_b200 as dgs
+    N = wl.num_workers
+    rng = np.random.Generator(np.random.Philox(key=wl.seed + 77))
+    sched = rng.integers(0, N, size=4 * N + K).astype(np.int32)
+    ctx = dgs.Context.from_workload(wl, theta0=theta0)
+    for e in range(4 * N):
+        ctx.event(int(sched[e]), grads[e % pool])
+    ctx.flush()
+    s0 = ctx.stats()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    ev0.record(ctx.stream)
+    for e in range(4 * N, 4 * N + K):
+        ctx.event(int(sched[e]), grads[e % pool])
+    ctx.flush()
+    ev1.record(ctx.stream)
+    torch.cuda.synchronize(dev)
+    s1 = ctx.stats()
+    assert ctx.status() == 0, "device status word is not clean"
+    ctx.close()
+    t = ev0.elapsed_time(ev1) * 1e-3
+    return {"schedule": "each event's worker drawn uniformly at random", "events": K, "value": K / t, "unit": UNIT,
+            "ms_per_step": 1e3 * t / K,
+            "selection_routes": {"single_pass": s1[0] - s0[0], "two_pass": s1[1] - s0[1],
+                                 "candidates_per_selection": (s1[3] - s0[3]) / max(1, 2 * K)}}
 
 
 
@@ -504,8 +586,8 @@ def main() -> None:
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="kernel sweep over vector sizes and densities")
     ap.add_argument("--sweep-max-log2n", type=int, default=28)
-    ap.add_argument("--traffic-bytes", type=float, default=None,
-                    help="ncu dram bytes per launch of the dominant kernel, copied from profiles/")
+    ap.add_argument("--windows", type=int, default=5, help="timed windows of --steps events each (the median is reported)")
+    ap.add_argument("--no-jitter", action="store_true", help="skip the extra pass with irregular arrivals")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

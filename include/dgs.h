@@ -53,7 +53,8 @@ typedef enum {
   DGS_ECUDA = -3,    /* a CUDA runtime call or launch failed; see dgs_last_cuda_error */
   DGS_ETIMEOUT = -4, /* a bounded device-side wait gave up (reported by dgs_status) */
   DGS_ESTATE = -5,   /* context already freed or unusable after an earlier error */
-  DGS_ELIMIT = -6    /* size beyond the fixed capacity of dgs_topk_encode_static */
+  DGS_ELIMIT = -6    /* size beyond a fixed capacity: dgs_topk_encode_static, or (as device status) more nonzero
+                        entries than a dgs_worker_pull_all packet can carry */
 } dgs_error;
 
 typedef struct dgs_ctx dgs_ctx; /* opaque, host side */
@@ -79,14 +80,28 @@ typedef struct {
   uint32_t count;      /* = sum of k_push (push) or k_pull (pull)  */
 } dgs_packet;
 
+/* A sparse update whose number of entries is only known on the device (the pull without
+ * secondary compression sends however many entries the difference vector holds). */
+typedef struct {
+  const uint32_t* idx;   /* DEVICE u32[capacity], ascending; the first *count entries are valid */
+  const float* val;      /* DEVICE f32[capacity]                                                */
+  const uint32_t* count; /* DEVICE u32: entries written, <= capacity                            */
+  uint32_t capacity;     /* = dgs_config.pull_all_capacity                                      */
+} dgs_var_packet;
+
 enum {
   DGS_KEEP_LOCAL_MODEL = 1u << 0, /* keep theta_k per worker and add every pulled G to it (Eq. 5) */
   DGS_RESIDUAL_MODE = 1u << 1,    /* worker rule of Algorithm 1 instead of Algorithm 3: v <- v + eta*grad,
                                      sent entries leave v, the rest stay (no momentum, no 1/m rescale) */
   DGS_HOST_IO = 1u << 2,          /* reserve staging buffers for dgs_event_host */
   DGS_NO_SPECULATION = 1u << 3,   /* always take the two-pass selection (histogram pass, then stream pass) */
-  DGS_SINGLE_STREAM = 1u << 4     /* enqueue every step on ONE internal stream: kernels run one after the other in
+  DGS_SINGLE_STREAM = 1u << 4,    /* enqueue every step on ONE internal stream: kernels run one after the other in
                                      call order (same results; for debugging and for timing a kernel on its own) */
+  DGS_TEST_STALLED_BARRIER = 1u << 5 /* testing only: the barrier among the CTAs of the finalize kernels waits for one
+                                     CTA that does not exist, with a limit of a few thousand polls.  Every wait then
+                                     runs out: the kernels return early, packets and state are NOT valid, and
+                                     dgs_status reports DGS_ETIMEOUT.  Shows that a wait that cannot end costs a
+                                     status word, not the GPU. */
 };
 
 typedef struct {
@@ -101,6 +116,8 @@ typedef struct {
   uint64_t arena_bytes;        /* >= what dgs_arena_bytes reports for this configuration               */
   void* stream;                /* cudaStream_t on which all work is enqueued (NULL = default stream)   */
   uint32_t flags;              /* DGS_* flags above                                                    */
+  uint32_t pull_all_capacity;  /* most entries a dgs_worker_pull_all packet can carry (0: that call is not
+                                  used and no packet slots are set aside for it); at most n              */
 } dgs_config;
 
 enum { DGS_THETA = 0, DGS_U = 1, DGS_D = 2, DGS_THETA_LOCAL = 3 };
@@ -137,6 +154,18 @@ int dgs_server_apply(dgs_ctx* ctx, uint32_t worker, const dgs_packet* pkt);
  * entries there, adds them to theta_worker when DGS_KEEP_LOCAL_MODEL is set
  * (Eq. 5), and records prev(worker) = t. */
 int dgs_worker_pull(dgs_ctx* ctx, uint32_t worker, dgs_packet* out);
+
+/* Worker pull WITHOUT secondary compression (Algorithm 2 with the switch off, the paper's
+ * normal case; Eq. 3, Eq. 4): the packet lists every entry of D_worker that is not zero (+0 and
+ * -0 both count as zero), in ascending index order, and those entries are cleared, so that
+ * v_worker = M afterwards; they are added to theta_worker when DGS_KEEP_LOCAL_MODEL is set
+ * (Eq. 5); prev(worker) = t.  The number of entries is written to a device word of the packet
+ * slot (no host synchronisation); *out is filled at once.  If D_worker holds more nonzero
+ * entries than cfg.pull_all_capacity, the first `capacity` of them (lowest indices) are sent
+ * and cleared, the others stay in D_worker for a later pull, and the device status word
+ * becomes DGS_ELIMIT (see dgs_status).  Needs pull_all_capacity > 0, else DGS_EINVAL.  A few
+ * packet slots are used in turn: a packet stays valid until the fourth later call. */
+int dgs_worker_pull_all(dgs_ctx* ctx, uint32_t worker, dgs_var_packet* out);
 
 /* One whole event for `worker`: push, apply of that packet, pull.  Either packet
  * pointer may be NULL. */

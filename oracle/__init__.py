@@ -7,6 +7,7 @@ lives in the C++ file; this wrapper only builds it and marshals numpy arrays.
 from __future__ import annotations
 
 import ctypes as C
+import hashlib
 import os
 import subprocess
 from typing import Optional, Tuple
@@ -19,13 +20,28 @@ _LIB = os.path.join(_HERE, "libdgs_oracle.so")
 _lib = None
 
 
+_FLAGS = ["-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math", "-shared", "-fPIC"]
+
+
+def _source_hash() -> str:
+    h = hashlib.sha256(" ".join(_FLAGS).encode())
+    with open(_SRC, "rb") as f:
+        h.update(f.read())
+    return h.hexdigest()
+
+
 def build(force: bool = False) -> str:
-    """Compile the checker (g++, no FMA contraction, no fast-math)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    """Compile the checker (g++, no FMA contraction, no fast-math).  Rebuilt whenever the source or the
+    flags differ from those the library beside it was built from (a hash is stored with it)."""
+    stamp = _LIB + ".hash"
+    digest = _source_hash()
+    fresh = os.path.exists(_LIB) and os.path.exists(stamp) and open(stamp).read().strip() == digest
+    if force or not fresh:
         tmp = _LIB + f".{os.getpid()}.tmp"
-        subprocess.check_call(["g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math",
-                               "-shared", "-fPIC", "-o", tmp, _SRC])
+        subprocess.check_call(["g++"] + _FLAGS + ["-o", tmp, _SRC])
         os.replace(tmp, _LIB)
+        with open(stamp, "w") as f:
+            f.write(digest + "\n")
     return _LIB
 
 

@@ -23,10 +23,11 @@ LIB_PATH = os.path.join(_HERE, "libdgs.so")
 
 DGS_OK, DGS_EINVAL, DGS_ENOMEM, DGS_ECUDA, DGS_ETIMEOUT, DGS_ESTATE = 0, -1, -2, -3, -4, -5
 DGS_KEEP_LOCAL_MODEL, DGS_RESIDUAL_MODE, DGS_HOST_IO, DGS_NO_SPECULATION, DGS_SINGLE_STREAM = 1, 2, 4, 8, 16
+DGS_TEST_STALLED_BARRIER = 32
 DGS_THETA, DGS_U, DGS_D, DGS_THETA_LOCAL = 0, 1, 2, 3
 
 EXPORTS = (
-    "dgs_arena_bytes", "dgs_init", "dgs_worker_push", "dgs_server_apply", "dgs_worker_pull",
+    "dgs_arena_bytes", "dgs_init", "dgs_worker_push", "dgs_server_apply", "dgs_worker_pull", "dgs_worker_pull_all",
     "dgs_event", "dgs_flush", "dgs_event_host", "dgs_state_ptr", "dgs_state_load", "dgs_status", "dgs_stats", "dgs_pull_read_stats",
     "dgs_prev", "dgs_launch_count", "dgs_last_cuda_error", "dgs_free", "dgs_error_string",
     "dgs_timing_enable", "dgs_timing_read", "dgs_timing_trace", "dgs_topk_encode_static",
@@ -47,10 +48,15 @@ class dgs_packet(C.Structure):
     _fields_ = [("idx", C.c_void_p), ("val", C.c_void_p), ("count", C.c_uint32)]
 
 
+class dgs_var_packet(C.Structure):
+    _fields_ = [("idx", C.c_void_p), ("val", C.c_void_p), ("count", C.c_void_p), ("capacity", C.c_uint32)]
+
+
 class dgs_config(C.Structure):
     _fields_ = [("n", C.c_uint64), ("num_workers", C.c_uint32), ("lr", C.c_float), ("momentum", C.c_float),
                 ("num_segments", C.c_uint32), ("segments", C.POINTER(dgs_segment)), ("theta0", C.c_void_p),
-                ("arena", C.c_void_p), ("arena_bytes", C.c_uint64), ("stream", C.c_void_p), ("flags", C.c_uint32)]
+                ("arena", C.c_void_p), ("arena_bytes", C.c_uint64), ("stream", C.c_void_p), ("flags", C.c_uint32),
+                ("pull_all_capacity", C.c_uint32)]
 
 
 class DgsError(RuntimeError):
@@ -76,6 +82,7 @@ def lib() -> C.CDLL:
         L.dgs_worker_push.argtypes = [vp, u32, vp, C.POINTER(dgs_packet)]
         L.dgs_server_apply.argtypes = [vp, u32, C.POINTER(dgs_packet)]
         L.dgs_worker_pull.argtypes = [vp, u32, C.POINTER(dgs_packet)]
+        L.dgs_worker_pull_all.argtypes = [vp, u32, C.POINTER(dgs_var_packet)]
         L.dgs_event.argtypes = [vp, u32, vp, C.POINTER(dgs_packet), C.POINTER(dgs_packet)]
         L.dgs_flush.argtypes = [vp]
         L.dgs_event_host.argtypes = [vp, u32, vp, vp, vp]
@@ -110,14 +117,15 @@ def _check(rc: int, where: str) -> None:
 
 def make_config(n: int, num_workers: int, lr: float, momentum: float, seg_offset: Sequence[int],
                 seg_len: Sequence[int], k_push: Sequence[int], k_pull: Sequence[int], *, theta0: int = 0,
-                arena: int = 0, arena_bytes: int = 0, stream: int = 0, flags: int = 0) -> dgs_config:
+                arena: int = 0, arena_bytes: int = 0, stream: int = 0, flags: int = 0,
+                pull_all_capacity: int = 0) -> dgs_config:
     """Fills a dgs_config; pointers are plain integers (device addresses)."""
     S = len(seg_len)
     segs = (dgs_segment * S)()
     for s in range(S):
         segs[s] = dgs_segment(int(seg_offset[s]), int(seg_len[s]), int(k_push[s]), int(k_pull[s]))
     cfg = dgs_config(int(n), int(num_workers), float(lr), float(momentum), S, segs, theta0 or None,
-                     arena or None, int(arena_bytes), stream or None, int(flags))
+                     arena or None, int(arena_bytes), stream or None, int(flags), int(pull_all_capacity))
     cfg._segs_keepalive = segs
     return cfg
 
@@ -147,6 +155,12 @@ def dgs_server_apply(ctx: int, worker: int, pkt: dgs_packet) -> None:
 def dgs_worker_pull(ctx: int, worker: int) -> dgs_packet:
     p = dgs_packet()
     _check(lib().dgs_worker_pull(ctx, worker, C.byref(p)), "dgs_worker_pull")
+    return p
+
+
+def dgs_worker_pull_all(ctx: int, worker: int) -> dgs_var_packet:
+    p = dgs_var_packet()
+    _check(lib().dgs_worker_pull_all(ctx, worker, C.byref(p)), "dgs_worker_pull_all")
     return p
 
 

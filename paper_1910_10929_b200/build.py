@@ -1,6 +1,7 @@
 """Builds libdgs.so (the C ABI of include/dgs.h) with nvcc for sm_100a, in-tree."""
 from __future__ import annotations
 
+import hashlib
 import os
 import subprocess
 
@@ -19,11 +20,27 @@ NVCC_FLAGS = [
 ]
 
 
+STAMP = LIB + ".hash"
+
+
+def source_hash() -> str:
+    """Hash of everything the library is made from: the sources, the header, the compiler flags."""
+    h = hashlib.sha256()
+    h.update("\0".join(NVCC_FLAGS).encode())
+    for p in DEPENDS:
+        h.update(b"\0" + os.path.basename(p).encode() + b"\0")
+        with open(p, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
 def stale() -> bool:
-    if not os.path.exists(LIB):
+    """True unless the library was built from exactly the sources that are here now (decided by content:
+    the hash stored beside the library at build time, not by file times)."""
+    if not os.path.exists(LIB) or not os.path.exists(STAMP):
         return True
-    t = os.path.getmtime(LIB)
-    return any(os.path.getmtime(p) > t for p in DEPENDS)
+    with open(STAMP) as f:
+        return f.read().strip() != source_hash()
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
@@ -33,8 +50,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
     tmp = LIB + f".{os.getpid()}.tmp"
     cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + [
         "-I", os.path.join(ROOT, "include"), "-o", tmp] + SOURCES
+    digest = source_hash()
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)
+    with open(STAMP, "w") as f:
+        f.write(digest + "\n")
     return LIB
 
 

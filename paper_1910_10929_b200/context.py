@@ -13,7 +13,7 @@ class Context:
 
     def __init__(self, n: int, num_workers: int, lr: float, momentum: float, seg_offset, seg_len, k_push, k_pull,
                  theta0: torch.Tensor, flags: int = 0, device: Optional[torch.device] = None,
-                 stream: Optional[torch.cuda.Stream] = None):
+                 stream: Optional[torch.cuda.Stream] = None, pull_all_capacity: int = 0):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required: this library has no CPU path")
         self.device = torch.device(device if device is not None else theta0.device)
@@ -23,7 +23,8 @@ class Context:
         self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
         theta0 = theta0.to(device=self.device, dtype=torch.float32).contiguous()
         assert theta0.numel() == self.n
-        cfg = dgs.make_config(n, num_workers, lr, momentum, seg_offset, seg_len, k_push, k_pull, flags=flags)
+        cfg = dgs.make_config(n, num_workers, lr, momentum, seg_offset, seg_len, k_push, k_pull, flags=flags,
+                              pull_all_capacity=pull_all_capacity)
         self.arena_bytes = dgs.dgs_arena_bytes(cfg)
         with torch.cuda.device(self.device):
             self.arena = torch.empty(self.arena_bytes, dtype=torch.uint8, device=self.device)
@@ -39,11 +40,11 @@ class Context:
 
     @classmethod
     def from_workload(cls, wl, theta0: Optional[torch.Tensor] = None, flags: int = 0,
-                      device: str = "cuda:0") -> "Context":
+                      device: str = "cuda:0", pull_all_capacity: int = 0) -> "Context":
         if theta0 is None:
             theta0 = torch.from_numpy(wl.theta0()).to(device)
         return cls(wl.n, wl.num_workers, wl.lr, wl.momentum, wl.seg_offset, wl.seg_len, wl.k_push, wl.k_pull,
-                   theta0, flags=flags, device=theta0.device)
+                   theta0, flags=flags, device=theta0.device, pull_all_capacity=pull_all_capacity)
 
     # ---- the three steps of an event ---------------------------------------------
     def worker_push(self, worker: int, grad: torch.Tensor) -> "dgs.dgs_packet":
@@ -55,6 +56,16 @@ class Context:
 
     def worker_pull(self, worker: int) -> "dgs.dgs_packet":
         return dgs.dgs_worker_pull(self.handle, worker)
+
+    def worker_pull_all(self, worker: int) -> "dgs.dgs_var_packet":
+        return dgs.dgs_worker_pull_all(self.handle, worker)
+
+    def var_packet(self, pkt: "dgs.dgs_var_packet") -> Tuple[torch.Tensor, torch.Tensor]:
+        """(idx, val) of a packet whose count lives on the device: flushes, reads the count (this waits
+        for the stream), returns views of the valid entries."""
+        self.flush()
+        count = int(self._view(pkt.count, 1, torch.int32).item())
+        return self._view(pkt.idx, count, torch.int32), self._view(pkt.val, count, torch.float32)
 
     def event(self, worker: int, grad: torch.Tensor) -> Tuple["dgs.dgs_packet", "dgs.dgs_packet"]:
         assert grad.is_cuda and grad.dtype == torch.float32 and grad.is_contiguous() and grad.numel() == self.n

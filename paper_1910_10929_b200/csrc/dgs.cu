@@ -30,22 +30,15 @@ namespace {
 
 constexpr uint64_t kAlign = 256;
 constexpr uint32_t kMagic = 0x44475331u;  // "DGS1"
-#ifndef DGS_PUSH_SLOTS
-#define DGS_PUSH_SLOTS 8
-#endif
-constexpr int kPushSlots = DGS_PUSH_SLOTS;  // push packet slots, used in turn (a slot is refilled once its apply has read it)
+constexpr int kPushSlots = 8;  // push packet slots, used in turn (a slot is refilled once its apply has read it)
 constexpr int kPullSlots = 6;             // pull packet slots
-#ifndef DGS_WORKER_STREAMS
-#define DGS_WORKER_STREAMS 4
-#endif
-#ifndef DGS_SERVER_STREAMS
-#define DGS_SERVER_STREAMS 6
-#endif
-constexpr int kWorkerStreams = DGS_WORKER_STREAMS, kServerStreams = DGS_SERVER_STREAMS;
+constexpr int kVarSlots = 4;              // packet slots of the pull without secondary compression
+constexpr int kWorkerStreams = 4, kServerStreams = 6;   // library streams for the pushes and for the pulls
 constexpr int kPushSets = kWorkerStreams;  // scratch sets and spare velocity buffers of the pushes
 constexpr int kPullSets = kServerStreams;  // scratch sets of the pulls
 constexpr int kAllSets = kPushSets + kPullSets;
 constexpr int kLogRingMax = 64;             // most packets the apply log keeps
+constexpr int kLogSlack = 32;               // slots of the log beyond one per worker
 enum StreamId : int { kStW0 = 0, kStApply = kWorkerStreams, kStS0 = kWorkerStreams + 1,
                       kNumStreams = kWorkerStreams + 1 + kServerStreams };
 
@@ -65,6 +58,7 @@ struct Layout {
   // byte offsets into the arena
   uint64_t theta, u, D, theta_local, grad_stage;
   uint64_t pkt_idx[kPushSlots + kPullSlots], pkt_val[kPushSlots + kPullSlots];  // push slots, then pull slots
+  uint64_t var_idx[kVarSlots], var_val[kVarSlots], var_count[kVarSlots], L_one;
   uint64_t tiles, segs, seg_off, seg_tile0;
   ScratchLayout sc[kAllSets];  // push sets, then pull sets
   uint64_t L_next, u_slots, status, stats;
@@ -81,6 +75,7 @@ int check_config(const dgs_config* c) {
   if (c->n == 0 || c->n >= (1ull << 32)) return DGS_EINVAL;
   if (c->num_workers == 0 || c->num_workers > 65535) return DGS_EINVAL;
   if (c->num_segments == 0 || c->num_segments >= 65536) return DGS_EINVAL;
+  if (c->pull_all_capacity > c->n) return DGS_EINVAL;
   if (!std::isfinite(c->lr)) return DGS_EINVAL;
   if (!(c->momentum > 0.0f) || !(c->momentum <= 1.0f)) return DGS_EINVAL;
   uint64_t pos = 0;
@@ -161,6 +156,12 @@ void make_layout(const dgs_config* c, Layout* L) {
     L->pkt_idx[p] = take(K * 4);
     L->pkt_val[p] = take(K * 4);
   }
+  for (int p = 0; p < kVarSlots; ++p) {
+    L->var_idx[p] = c->pull_all_capacity ? take((uint64_t)c->pull_all_capacity * 4) : 0;
+    L->var_val[p] = c->pull_all_capacity ? take((uint64_t)c->pull_all_capacity * 4) : 0;
+    L->var_count[p] = c->pull_all_capacity ? take(4) : 0;
+  }
+  L->L_one = take(S * 4);
   L->tiles = take((uint64_t)L->num_tiles * sizeof(Tile));
   L->segs = take(S * sizeof(SegDesc));
   L->seg_off = take((S + 1) * 4);
@@ -185,13 +186,10 @@ void make_layout(const dgs_config* c, Layout* L) {
     sc.sync = take(kNumSyncWords * 4);
     sc.zero_end = off;
   }
-#ifndef DGS_LOG_SLACK
-#define DGS_LOG_SLACK 32
-#endif
   // A slot of the log is reused `ring` packets later, and the apply that refills it waits for every catch-up that
   // still reads the old packet.  A worker that comes back after N events reads the N newest packets, so ring - N
   // is how many events the server side of an event may lag behind the pushes before the pushes stall.
-  L->log_ring = (uint32_t)std::min<uint64_t>(kLogRingMax, std::max<uint64_t>(N + DGS_LOG_SLACK, 16));
+  L->log_ring = (uint32_t)std::min<uint64_t>(kLogRingMax, std::max<uint64_t>(N + kLogSlack, 16));
   L->log_stride = (uint32_t)align_up(L->K[0], 64);
   L->log_idx = take((uint64_t)L->log_ring * L->log_stride * 4);
   L->log_val = take((uint64_t)L->log_ring * L->log_stride * 4);
@@ -243,7 +241,7 @@ struct dgs_ctx {
   size_t ev_next[kNumStreams];
   uint64_t task_seq;                               // tasks filed so far
   uint64_t waited_seq[kNumStreams][kNumStreams];   // [waiting stream][stream]: newest task already waited for
-  uint64_t push_count, pull_count, event_count;
+  uint64_t push_count, pull_count, event_count, var_count;
   // Lazy difference vectors: packet number p (counted from 0) of the library's own pushes sits in slot
   // p % ring of the log from its apply on; applied[q] packets have been folded into D_q so far.
   PacketLog log;
@@ -309,7 +307,8 @@ struct ResIds {
   uint32_t SPARE(int j) const { return 5 * N + 1 + j; }
   uint32_t SCR(int kind, int set) const { return 5 * N + 1 + kPushSets + (kind ? kPushSets : 0) + set; }
   uint32_t PKT(int slot) const { return 5 * N + 1 + kPushSets + kAllSets + slot; }   // push slots, then pull slots
-  uint32_t STAGE() const { return PKT(kPushSlots + kPullSlots); }
+  uint32_t VPKT(int slot) const { return PKT(kPushSlots + kPullSlots) + (uint32_t)slot; }
+  uint32_t STAGE() const { return VPKT(kVarSlots); }
   uint32_t LOG(uint32_t slot) const { return STAGE() + 1 + slot; }
   uint32_t RANGES(int gen) const { return LOG(kLogRingMax) + (uint32_t)gen; }   // the two generations of ranges of the log
   uint32_t count() const { return RANGES(1) + 1; }
@@ -332,10 +331,7 @@ inline int live(dgs_ctx* c) {
 }
 
 constexpr size_t kMaxTimedLaunches = 1 << 16;
-#ifndef DGS_FINALIZE_WORKERS
-#define DGS_FINALIZE_WORKERS 64
-#endif
-constexpr int kFinalizeWorkers = DGS_FINALIZE_WORKERS;  // CTAs of the finalize kernel (more of them take SM slots from the stream passes)
+constexpr int kFinalizeWorkers = 64;  // CTAs of the finalize kernel (more of them take SM slots from the stream passes)
 
 // Records an event before and after one launch when timing is on.
 struct TimedLaunch {
@@ -515,6 +511,10 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age
   if (3ull * a.pkt_count <= 48ull * kThreads * 8) fin_base = std::min(fin_base, 48);
   const int fin_grid = std::min(c->finalize_max[MODE], std::max(fin_base, (int)(a.pkt_count / 4096)));
   a.workers = (uint32_t)fin_grid;
+  if (c->cfg.flags & DGS_TEST_STALLED_BARRIER) {
+    a.phantom_workers = 1;
+    a.spin_limit = 4096;
+  }
   a.seq = ++c->select_seq;
   a.L_in = single_pass ? c->L_next(KIND, (uint32_t)row) : ws.L_safe;
   task.stream = stream_id;
@@ -580,9 +580,6 @@ int occupancy_grids(dgs_ctx* c, int sms) {
   // what counts is how few SM resources it holds, not how fast it is alone: one CTA per SM (its ranges
   // are balanced by the plan that finalize leaves behind).  A context with one worker selects alone.
   if (MODE == kPull && c->cfg.num_workers > 1) c->stream_grid[MODE] = std::min(c->stream_grid[MODE], sms);
-#ifdef DGS_PULL_GRID   // tunable for experiments
-  if (MODE == kPull && c->cfg.num_workers > 1) c->stream_grid[MODE] = std::min(c->stream_grid[MODE], DGS_PULL_GRID);
-#endif
   DGS_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_hist_all<MODE>, kThreads, 0));
   if (occ < 1) occ = 1;
   c->hist_grid[MODE] = std::min(sms * occ, kMaxGrid);
@@ -663,7 +660,7 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
     c->ev_next[i] = 0;
     for (int j = 0; j < kNumStreams; ++j) c->waited_seq[i][j] = 0;
   }
-  c->pull_count = c->event_count = 0;
+  c->pull_count = c->event_count = c->var_count = 0;
   c->log_head = 0;
   c->last_ranges = 0;
   c->cur_gen = 0;
@@ -713,11 +710,7 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   INIT_CUDA(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
   if (!coop) return fail(DGS_ECUDA);
   c->sms = sms;
-#ifdef DGS_NO_LIGHT_PULL
-  c->light_pull = false;
-#else
   c->light_pull = cfg->num_workers > 1;
-#endif
   if (occupancy_grids<kPushSam>(c, sms) != DGS_OK || occupancy_grids<kPushResidual>(c, sms) != DGS_OK ||
       occupancy_grids<kPull>(c, sms) != DGS_OK)
     return fail(DGS_ECUDA);
@@ -781,6 +774,8 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   seg_off[cfg->num_segments] = (uint32_t)cfg->n;  // n < 2^32
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.seg_off), seg_off.data(), seg_off.size() * 4, cudaMemcpyHostToDevice, st));
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.seg_tile0), seg_tile0.data(), seg_tile0.size() * 4, cudaMemcpyHostToDevice, st));
+  std::vector<uint32_t> ones(cfg->num_segments, 1u);   // the bound that admits every nonzero value
+  INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.L_one), ones.data(), ones.size() * 4, cudaMemcpyHostToDevice, st));
   std::vector<float*> slots(N + kPushSets);
   for (uint32_t q = 0; q < N + kPushSets; ++q) slots[q] = c->u_buf(q);
   INIT_CUDA(cudaMemcpyAsync(c->at<char>(L.u_slots), slots.data(), slots.size() * sizeof(float*), cudaMemcpyHostToDevice, st));
@@ -1010,7 +1005,78 @@ int pull_impl(dgs_ctx* c, uint32_t worker, dgs_packet* out) {
   return DGS_OK;
 }
 
+// Pull without secondary compression: catch-up, the pull's stream pass with the bound 1 (every nonzero entry
+// becomes a candidate, in index order), then the copy into the packet.  Shares the pulls' streams and scratch sets.
+int pull_all_impl(dgs_ctx* c, uint32_t worker, dgs_var_packet* out) {
+  const Layout& L = c->lay;
+  const ResIds R{c->cfg.num_workers};
+  const int vslot = (int)(c->var_count % kVarSlots);
+  const int set = (int)(c->pull_count % kPullSets);
+  const int stream_id = kStS0 + (int)(c->pull_count % kServerStreams);
+  cudaStream_t st = c->st[stream_id];
+  int rc = fork_from_user(c, stream_id);  // the caller may still be reading an older packet on its stream
+  if (rc != DGS_OK) return rc;
+  Workspace& ws = c->ws[kPushSets + set];
+  SelArgs a;
+  std::memset(&a, 0, sizeof(a));
+  a.D = c->D_buf(worker);
+  a.blk_max = c->blk_max(worker);
+  a.theta_local = (c->cfg.flags & DGS_KEEP_LOCAL_MODEL) ? c->theta_local_buf(worker) : nullptr;
+  a.L_in = c->at<uint32_t>(L.L_one);
+  a.m = c->cfg.momentum;
+  a.lr = c->cfg.lr;
+  a.inv_m = c->inv_m;
+  Task task;
+  task.stream = stream_id;
+  task.writes = {R.VPKT(vslot), R.SCR(1, set)};
+  catch_up_deps(c, worker, &task);  // D_worker is brought up to date first, on the same stream
+  if (a.theta_local) task.writes.push_back(R.TL(worker));
+  rc = task_begin(c, task);
+  if (rc != DGS_OK) return rc;
+  rc = catch_up_launch(c, worker, st);
+  if (rc != DGS_OK) return rc;
+  {
+    TimedLaunch t(c, st, DGS_KERNEL_STREAM_PULL);
+    if (c->light_pull)
+      k_pull_light<<<c->stream_grid[kPull], kThreads, 0, st>>>(ws, a);
+    else
+      k_stream<kPull><<<c->stream_grid[kPull], kThreads, StreamRing<kPull>::kBytes, st>>>(ws, a);
+    DGS_CUDA(c, cudaGetLastError());
+    c->launches += 1;
+  }
+  uint32_t* vi = c->at<uint32_t>(L.var_idx[vslot]);
+  float* vv = c->at<float>(L.var_val[vslot]);
+  uint32_t* vc = c->at<uint32_t>(L.var_count[vslot]);
+  {
+    TimedLaunch t(c, st, DGS_KERNEL_FINALIZE_PULL);
+    k_emit_all<<<2 * c->sms, kThreads, 0, st>>>(ws, a.D, a.theta_local, a.blk_max, vi, vv, vc, c->cfg.pull_all_capacity);
+    DGS_CUDA(c, cudaGetLastError());
+    c->launches += 1;
+  }
+  rc = task_end(c, task);
+  if (rc != DGS_OK) return rc;
+  c->prev[worker] = (int64_t)c->timestamp;
+  c->pull_count += 1;
+  c->var_count += 1;
+  if (out) {
+    out->idx = vi;
+    out->val = vv;
+    out->count = vc;
+    out->capacity = c->cfg.pull_all_capacity;
+  }
+  return DGS_OK;
+}
+
 }  // namespace
+
+int dgs_worker_pull_all(dgs_ctx* c, uint32_t worker, dgs_var_packet* out) {
+  int rc = live(c);
+  if (rc != DGS_OK) return rc;
+  if (worker >= c->cfg.num_workers || c->cfg.pull_all_capacity == 0) return DGS_EINVAL;
+  rc = begin_call(c);
+  if (rc != DGS_OK) return rc;
+  return pull_all_impl(c, worker, out);
+}
 
 int dgs_worker_push(dgs_ctx* c, uint32_t worker, const float* grad, dgs_packet* out) {
   int rc = live(c);

@@ -116,6 +116,8 @@ struct SelArgs {
   int speculate;          // 0: never carry a bound (L_next is left alone)
   uint32_t workers;       // CTAs of finalize that process the candidates
   uint32_t seq;           // launch sequence number (tags the decision word)
+  uint32_t phantom_workers;  // testing only: CTAs the finalize barrier waits for beyond those launched (0 in normal use)
+  uint32_t spin_limit;    // polls after which a bounded wait gives up (0: kSpinLimit)
 };
 
 __device__ __forceinline__ uint32_t key_of(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
@@ -468,24 +470,14 @@ __device__ __forceinline__ uint32_t tile_mask_smem(const SelArgs& a, uint32_t ti
 // of them in flight.
 constexpr int kStageTiles = kWarps;                        // one tile per warp and stage
 constexpr int kStageFloats = kStageTiles * kWarpTile;      // per input array
-// Tunables of the ring (compile-time): stages per CTA, and the least dynamic shared memory a push
-// CTA asks for.  Asking for more than the ring needs caps the CTAs of the push pass per SM, which
-// leaves room on every SM for the short kernels of other streams (finalize, catch-up, pull).
-#ifndef DGS_PUSH_STAGES
-#define DGS_PUSH_STAGES 3
-#endif
-#ifndef DGS_PULL_STAGES
-#define DGS_PULL_STAGES 4
-#endif
-#ifndef DGS_PUSH_MIN_SMEM
-#define DGS_PUSH_MIN_SMEM 0
-#endif
+// The ring: three stages for a push (96 KB, two CTAs per SM, 128 KB of the SM's shared memory in flight),
+// four for the staged form of a pull.
 template <int MODE> struct StreamRing {
   static constexpr int kInputs = MODE == kPull ? 1 : 2;
-  static constexpr int kStages = MODE == kPull ? DGS_PULL_STAGES : DGS_PUSH_STAGES;
+  static constexpr int kStages = MODE == kPull ? 4 : 3;
   static constexpr int kStageBytes = kInputs * kStageFloats * 4;          // 16 KB per input
   static constexpr int kRingBytes = kStages * kStageBytes;
-  static constexpr int kBytes = MODE != kPull && kRingBytes < DGS_PUSH_MIN_SMEM ? DGS_PUSH_MIN_SMEM : kRingBytes;
+  static constexpr int kBytes = kRingBytes;
 };
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -968,7 +960,8 @@ __device__ uint32_t block_pick(const uint32_t* hist, uint32_t k, uint32_t& bin, 
 // counter that only grows: the i-th barrier of a launch is passed when the counter has
 // reached i*W (the stream pass that precedes every finalize launch clears the counter).
 // Bounded: returns false, with the status word set, if the others do not arrive.
-__device__ bool worker_barrier(uint32_t* sync, uint32_t W, int* status, int* s_ok, uint32_t& target) {
+__device__ bool worker_barrier(uint32_t* sync, uint32_t W, int* status, int* s_ok, uint32_t& target,
+                               uint32_t limit = kSpinLimit) {
   target += W;
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -977,7 +970,7 @@ __device__ bool worker_barrier(uint32_t* sync, uint32_t W, int* status, int* s_o
     atomicAdd(sync + kBarCount, 1u);
     uint32_t spins = 0;
     while ((int32_t)(ld_volatile(sync + kBarCount) - target) < 0) {
-      if (++spins > kSpinLimit) {
+      if (++spins > limit) {
         ok = 0;
         atomicMin(status, kStatusTimeout);
         break;
@@ -1069,17 +1062,18 @@ __device__ __forceinline__ void cursor_advance(const FinalizeShared& sh, uint32_
   c.left -= n;
 }
 
-#ifndef DGS_FINALIZE_REGS
-#define DGS_FINALIZE_REGS 96
-#endif
+// 64 registers a thread: finalize runs beside two CTAs of a push pass on an SM, which leave it that many
 template <int MODE>
-__global__ void __maxnreg__(DGS_FINALIZE_REGS) k_finalize(Workspace ws, SelArgs a) {
+__global__ void __maxnreg__(64) k_finalize(Workspace ws, SelArgs a) {
   __shared__ FinalizeShared sh;
   extern __shared__ __align__(16) unsigned char fin_dyn[];   // finalize_dyn_bytes(S) bytes
 
   constexpr int PM = MODE == kPull ? 1 : 0;
   const uint32_t cta = blockIdx.x, W = gridDim.x, S = ws.num_segs;
   const uint32_t gthread = cta * kThreads + threadIdx.x, nthreads = W * kThreads;
+  // the barrier counts W arrivals; a test can make it wait for CTAs that do not exist, with a short limit,
+  // to see the bounded wait give up (every CTA then leaves with DGS_ETIMEOUT in the status word)
+  const uint32_t Wb = W + a.phantom_workers, spin_limit = a.spin_limit ? a.spin_limit : kSpinLimit;
 
   // pointers are read once, before anything may exchange them
   const float* in = nullptr;
@@ -1115,7 +1109,7 @@ __global__ void __maxnreg__(DGS_FINALIZE_REGS) k_finalize(Workspace ws, SelArgs 
       // the guess was too high for some layer: take the bound that cannot fail from a histogram of
       // the whole input and repeat the stream pass, with the few CTAs this kernel has
       hist_all_tiles<MODE>(ws, a, in, cta, W, sh.stream.hist);
-      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+      if (!worker_barrier(ws.sync, Wb, ws.status, &sh.ok, bar_target, spin_limit)) return;
       for (uint32_t s = cta; s < S; s += W) {
         uint32_t bin, krem;
         uint32_t* h = ws.hist1 + (size_t)s * kBins1;
@@ -1132,9 +1126,9 @@ __global__ void __maxnreg__(DGS_FINALIZE_REGS) k_finalize(Workspace ws, SelArgs 
         for (int b = threadIdx.x; b < kBins1; b += kThreads) h[b] = 0;
       }
       if (cta == 0 && threadIdx.x == 0) ws.sync[kFail] = 0;
-      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+      if (!worker_barrier(ws.sync, Wb, ws.status, &sh.ok, bar_target, spin_limit)) return;
       stream_tiles<MODE>(ws, a, ws.L_safe, in, out, cta, W, sh.stream);
-      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+      if (!worker_barrier(ws.sync, Wb, ws.status, &sh.ok, bar_target, spin_limit)) return;
     }
     // flat numbering of the candidates (the stream pass is complete: an earlier kernel, or the barrier above)
     parts = ld_volatile(ws.sync + kParts);
@@ -1229,13 +1223,13 @@ __global__ void __maxnreg__(DGS_FINALIZE_REGS) k_finalize(Workspace ws, SelArgs 
     if (everyone_picks) {
       if (!failed || redo) break;
       // every CTA has seen the same histogram and comes here: clear it once all have read it, then redo
-      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+      if (!worker_barrier(ws.sync, Wb, ws.status, &sh.ok, bar_target, spin_limit)) return;
       if (cta == 0)
         for (int b = threadIdx.x; b < kBins1; b += kThreads) ws.hist1[b] = 0;
-      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+      if (!worker_barrier(ws.sync, Wb, ws.status, &sh.ok, bar_target, spin_limit)) return;
       redo = true;
     } else {
-      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+      if (!worker_barrier(ws.sync, Wb, ws.status, &sh.ok, bar_target, spin_limit)) return;
       if (redo || ld_volatile(ws.sync + kFail) == 0) break;
       redo = true;
     }
@@ -1289,7 +1283,7 @@ __global__ void __maxnreg__(DGS_FINALIZE_REGS) k_finalize(Workspace ws, SelArgs 
         const uint32_t v = sh.stream.hist[b];
         if (v) atomicAdd(hist + b, v);
       }
-      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+      if (!worker_barrier(ws.sync, Wb, ws.status, &sh.ok, bar_target, spin_limit)) return;
       // the histogram of the level before has been read by everyone
       if (cta == 0) {
         uint32_t* old = level == 2 ? ws.hist1 : ws.hist2;
@@ -1310,7 +1304,7 @@ __global__ void __maxnreg__(DGS_FINALIZE_REGS) k_finalize(Workspace ws, SelArgs 
         const uint32_t prefix = seg_smem ? sm_seg_a[seg] : __ldcg(&ws.sel[seg].prefix);
         if ((key >> SH) == prefix) atomicAdd(hist + (size_t)seg * B + ((key >> (SH - 10)) & 1023u), 1u);
       });
-      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+      if (!worker_barrier(ws.sync, Wb, ws.status, &sh.ok, bar_target, spin_limit)) return;
       for (uint32_t s = cta; s < S; s += W) {
         uint32_t bin, krem;
         uint32_t* h = hist + (size_t)s * B;
@@ -1328,7 +1322,7 @@ __global__ void __maxnreg__(DGS_FINALIZE_REGS) k_finalize(Workspace ws, SelArgs 
         __syncthreads();
         for (int b = threadIdx.x; b < B; b += kThreads) h[b] = 0;
       }
-      if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+      if (!worker_barrier(ws.sync, Wb, ws.status, &sh.ok, bar_target, spin_limit)) return;
     }
   }
 
@@ -1369,7 +1363,7 @@ __global__ void __maxnreg__(DGS_FINALIZE_REGS) k_finalize(Workspace ws, SelArgs 
   unsigned long long cta_total;
   unsigned long long before = block_excl_scan(mine, sh.warp_scan, cta_total);
   if (threadIdx.x == 0) ws.cta_tot[cta] = make_uint2((uint32_t)(cta_total >> 32), (uint32_t)cta_total);
-  if (!worker_barrier(ws.sync, W, ws.status, &sh.ok, bar_target)) return;
+  if (!worker_barrier(ws.sync, Wb, ws.status, &sh.ok, bar_target, spin_limit)) return;
   if (S == 1 && cta == 0)
     for (int b = threadIdx.x; b < kBins3; b += kThreads) ws.hist3[b] = 0;
 
@@ -1548,13 +1542,72 @@ __global__ void __maxnreg__(64) k_stream(Workspace ws, SelArgs a) {
 }
 
 // ---- the pull's stream pass in its ring-less form (contexts with several workers) -----
-#ifndef DGS_LIGHT_REGS
-#define DGS_LIGHT_REGS 64
-#endif
-__global__ void __maxnreg__(DGS_LIGHT_REGS) k_pull_light(Workspace ws, SelArgs a) {
+__global__ void __maxnreg__(64) k_pull_light(Workspace ws, SelArgs a) {
   __shared__ StreamShared sh;
   if (blockIdx.x == 0 && threadIdx.x == 0) ws.sync[kBarCount] = 0;   // for the finalize launch that follows
   pull_tiles_light(ws, a, a.L_in, a.D, blockIdx.x, gridDim.x, sh);
+}
+
+// ---- pull without secondary compression: every nonzero entry of D_w -------------------
+// The stream pass has run with the bound 1 for every layer (key >= 1 <=> the value is not zero),
+// so the candidate buffer lists all nonzero entries of D_w in index order, part after part.
+// This kernel copies the first `capacity` of them into the packet, clears them in D_w (Eq. 4:
+// v_k becomes M), adds them to theta_w if kept (Eq. 5), and writes the count.
+constexpr int kStatusLimit = -6;   // = DGS_ELIMIT
+__global__ void __launch_bounds__(kThreads) k_emit_all(Workspace ws, float* __restrict__ D,
+                                                       float* __restrict__ theta_local,
+                                                       uint32_t* __restrict__ blk_max, uint32_t* __restrict__ out_idx,
+                                                       float* __restrict__ out_val, uint32_t* __restrict__ out_count,
+                                                       uint32_t capacity) {
+  __shared__ uint32_t pre[kMaxGrid + 1], slot0[kMaxGrid];
+  __shared__ unsigned long long warp_scan[kWarps];
+  const uint32_t parts = ld_volatile(ws.sync + kParts);
+  {
+    constexpr int PER = kMaxGrid / kThreads;   // parts <= kMaxGrid
+    unsigned long long carry = 0;
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      if ((uint32_t)(j * kThreads) < parts) {   // CTA-uniform
+        const uint32_t p = j * kThreads + threadIdx.x;
+        const uint32_t cnt = p < parts ? __ldcg(ws.part_cands + p) : 0;
+        if (p < parts) slot0[p] = __ldcg(ws.part_slot0 + p);
+        unsigned long long total;
+        const unsigned long long ex = block_excl_scan(cnt, warp_scan, total) + carry;
+        if (p < parts) pre[p] = (uint32_t)ex;
+        carry += total;
+      }
+    }
+    if (threadIdx.x == 0) pre[parts] = (uint32_t)carry;
+    __syncthreads();
+  }
+  const uint32_t C = pre[parts];
+  const bool all = C <= capacity;          // every nonzero entry is sent: D_w is zero afterwards
+  const uint32_t take = all ? C : capacity;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    *out_count = take;
+    if (!all) atomicMin(ws.status, kStatusLimit);
+    atomicAdd(ws.stats + 2, (unsigned long long)C);
+  }
+  for (uint32_t p = blockIdx.x * kThreads + threadIdx.x; p < take; p += gridDim.x * kThreads) {
+    uint32_t lo = 0, hi = parts - 1;       // last part with pre[part] <= p
+    while (lo < hi) {
+      const uint32_t mid = (lo + hi + 1) >> 1;
+      if (pre[mid] <= p) lo = mid; else hi = mid - 1;
+    }
+    const uint32_t slot = slot0[lo] + (p - pre[lo]);
+    const uint32_t i = __ldcg(ws.cand_idx + slot);
+    const float v = __ldcg(ws.cand_val + slot);
+    out_idx[p] = i;
+    out_val[p] = v;
+    D[i] = 0.f;
+    if (theta_local != nullptr) theta_local[i] = __fadd_rn(theta_local[i], v);
+    // the block's bound was made exact by the pass (a block without a nonzero entry already has bound 0);
+    // with everything sent the whole block is zero now
+    if (all && blk_max != nullptr) blk_max[i / kWarpTile] = 0;
+  }
+  // the pass has added the candidates' top key bits to the layers' histograms: nobody reads them here
+  const size_t words = (size_t)ws.num_segs * kBins1;
+  for (size_t w = (size_t)blockIdx.x * kThreads + threadIdx.x; w < words; w += (size_t)gridDim.x * kThreads) ws.hist1[w] = 0;
 }
 
 // ---- server apply ---------------------------------------------------------------
@@ -1675,29 +1728,44 @@ struct CatchShared {
   uint32_t pre[kCatchMaxPackets + 1];    // exclusive prefix of hi - lo
   uint32_t bmax[kCatchBlocks];           // largest new magnitude per block of kWarpTile elements, from the piece's first block on
   uint32_t dirty[kCatchLines / 4];       // dense: one byte per line, nonzero = the line holds an entry
+  uint32_t ab[2];                        // the range's first element and the element after its last
 };
 static_assert(sizeof(float) * kCatchDense == (sizeof(uint32_t) + sizeof(float)) * kCatchSlots, "the two views share their bytes");
 static_assert(kCatchDense <= 0xFFFF && kCatchDense % kCatchThreads == 0 && kCatchThreads % 32 == 0 &&
               kCatchThreads >= 2 * kCatchMaxPackets, "offsets fit the entry table");
 static_assert(kCatchDense / kWarpTile + 2 <= kCatchBlocks, "a dense piece's blocks fit the table of bounds");
 
-__global__ void __launch_bounds__(kCatchThreads) k_catch_up(PacketLog lg, uint64_t first, uint32_t count,
+__global__ void __maxnreg__(32) k_catch_up(PacketLog lg, uint64_t first, uint32_t count,
                                                        float* __restrict__ D, uint32_t* __restrict__ blk_max,
                                                        uint64_t n) {
   __shared__ CatchShared sh;
   const uint32_t tid = threadIdx.x;
   if (count == 0 || count > (uint32_t)kCatchMaxPackets) return;
   uint8_t* const dirty = reinterpret_cast<uint8_t*>(sh.dirty);
-  // a CTA takes the ranges blockIdx.x, blockIdx.x + gridDim.x, ... one after the other
+  // a CTA takes the ranges blockIdx.x, blockIdx.x + gridDim.x, ... one after the other; where a range lies
+  // in the packets and in the index space is fetched one range ahead
+  // (thread 2p reads where the range begins in packet p, thread 2p+1 where it ends)
+  const uint32_t* const my_pos = lg.pos + ((first + (tid >> 1)) % lg.ring) * (uint64_t)(lg.ranges + 1) + (tid & 1u);
+  uint32_t pos_ahead = 0, bnd_ahead = 0;     // of the range this CTA takes next
+  if (blockIdx.x < lg.ranges) {
+    if (tid < 2 * count) pos_ahead = __ldcg(my_pos + blockIdx.x);
+    if (tid < 2) bnd_ahead = blockIdx.x + tid == 0 ? 0u : (blockIdx.x + tid == lg.ranges ? (uint32_t)n : __ldcg(lg.bnd + blockIdx.x + tid));
+  }
   for (uint32_t c = blockIdx.x; c < lg.ranges; c += gridDim.x) {
   if (tid < 2 * count) {
-    // thread 2p reads where range c begins in packet p, thread 2p+1 where it ends
-    const uint32_t p = tid >> 1;
-    const uint32_t v = __ldcg(lg.pos + ((first + p) % lg.ring) * (uint64_t)(lg.ranges + 1) + c + (tid & 1u));
-    if (tid & 1u) sh.end[p] = v; else sh.lo[p] = v;
+    if (tid & 1u) sh.end[tid >> 1] = pos_ahead; else sh.lo[tid >> 1] = pos_ahead;
   }
-  const uint32_t range_b = c + 1 == lg.ranges ? (uint32_t)n : __ldcg(lg.bnd + c + 1);   // n < 2^32
-  uint32_t a = c == 0 ? 0u : __ldcg(lg.bnd + c);
+  if (tid < 2) sh.ab[tid] = bnd_ahead;
+  {
+    const uint32_t cn = c + gridDim.x;
+    if (cn < lg.ranges) {
+      if (tid < 2 * count) pos_ahead = __ldcg(my_pos + cn);
+      if (tid < 2) bnd_ahead = cn + tid == lg.ranges ? (uint32_t)n : __ldcg(lg.bnd + cn + tid);   // n < 2^32
+    }
+  }
+  __syncthreads();
+  const uint32_t range_b = sh.ab[1];
+  uint32_t a = sh.ab[0];
   for (;;) {   // one round per piece [a, b) of the range; everything here is uniform over the CTA
     for (int s = tid; s < kCatchBlocks; s += kCatchThreads) sh.bmax[s] = 0;
     for (int s = tid; s < kCatchLines / 4; s += kCatchThreads) sh.dirty[s] = 0;
@@ -1826,14 +1894,43 @@ __global__ void __launch_bounds__(kCatchThreads) k_catch_up(PacketLog lg, uint64
           if (k[u] != kFull) sh.tab.vals[tid + u * kCatchThreads] = d[u];
       }
       __syncthreads();
-      // the packets in arrival order; inside one packet every index, and so every place, occurs once
-      for (uint32_t p = 0; p < count; ++p) {
-        for (uint32_t e = sh.pre[p] + tid; e < sh.pre[p + 1]; e += kCatchThreads) {
-          const uint32_t slot = sh.ent_slot[e];
-          if (slot != 0xFFFFu) cur[slot] = __fsub_rn(cur[slot], sh.ent_val[e]);
+      // The packets in arrival order; inside one packet every index, and so every place, occurs once, so a
+      // packet's part is one parallel step.  A part of a piece rarely has more entries than a warp has lanes:
+      // one warp takes the steps one after the other with only its own barrier between them, which costs a
+      // fraction of a barrier of the whole CTA per packet.
+      if (tid < 32) {
+        constexpr int G = 4;   // packets whose entries a lane fetches together, ahead of the steps that use them
+        for (uint32_t p0 = 0; p0 < count; p0 += G) {
+          uint32_t slot[G], e1[G];
+          float val[G];
+          uint32_t ebeg = sh.pre[p0];
+#pragma unroll
+          for (int j = 0; j < G; ++j) {
+            const uint32_t pend = p0 + j < count ? sh.pre[p0 + j + 1] : ebeg;
+            const uint32_t e = ebeg + tid;
+            slot[j] = 0xFFFFu;
+            val[j] = 0.f;
+            if (e < pend) {
+              slot[j] = sh.ent_slot[e];
+              val[j] = sh.ent_val[e];
+            }
+            e1[j] = pend;
+            ebeg = pend;
+          }
+          ebeg = sh.pre[p0];
+#pragma unroll
+          for (int j = 0; j < G; ++j) {
+            if (slot[j] != 0xFFFFu) cur[slot[j]] = __fsub_rn(cur[slot[j]], val[j]);
+            for (uint32_t e = ebeg + 32 + tid; e < e1[j]; e += 32) {   // a part with more entries than lanes
+              const uint32_t sl = sh.ent_slot[e];
+              if (sl != 0xFFFFu) cur[sl] = __fsub_rn(cur[sl], sh.ent_val[e]);
+            }
+            __syncwarp();
+            ebeg = e1[j];
+          }
         }
-        __syncthreads();
       }
+      __syncthreads();
       // Back to memory.  The blocks' bounds must stay upper bounds: the largest new magnitude per block is
       // collected in shared memory, one global atomic per block afterwards.
       if (dense) {
@@ -1853,7 +1950,8 @@ __global__ void __launch_bounds__(kCatchThreads) k_catch_up(PacketLog lg, uint64
           if (__any_sync(kFull, live)) {
             key = __reduce_max_sync(kFull, key);
             // a line lies inside one block (lines and blocks start at multiples of 32 and of kWarpTile)
-            if ((tid & 31u) == 0 && key) atomicMax(sh.bmax + ((a0 + off) / kWarpTile - blk0), key);
+            uint32_t* const bm = sh.bmax + ((a0 + off) / kWarpTile - blk0);
+            if ((tid & 31u) == 0 && key > *bm) atomicMax(bm, key);
           }
         }
       } else {

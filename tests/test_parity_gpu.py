@@ -228,6 +228,83 @@ def test_trajectory_gpt2_small_per_layer_few_workers():
     replay_and_compare(wl)
 
 
+# ---- pull without secondary compression (Algorithm 2 with the switch off; Eq. 3-5) ---------
+def replay_full_pull(wl, *, flags=0, capacity=None, mixed=False, schedule=None):
+    """push / apply / pull-all for every event on both sides; packets bit for bit at every event
+    (count included), all state bit for bit at the end.  mixed: every third event takes the top-k
+    pull instead, so that both kinds of pull work on the same difference vectors."""
+    keep_local = bool(flags & dgs.DGS_KEEP_LOCAL_MODEL)
+    theta0 = wl.theta0()
+    cap = wl.n if capacity is None else capacity
+    orc = oracle.Oracle.from_workload(wl, keep_local=keep_local, theta0=theta0)
+    ctx = dgs.Context.from_workload(wl, theta0=torch.from_numpy(theta0).to(DEV), flags=flags, pull_all_capacity=cap)
+    sched = wl.schedule() if schedule is None else np.asarray(schedule)
+    for e in range(len(sched)):
+        w = int(sched[e])
+        g = wl.gradient(e)
+        pkt = ctx.worker_push(w, torch.from_numpy(g).to(DEV))
+        pi, pv = packet_to_numpy(ctx, pkt)
+        oi, ov = orc.push(w, g)
+        assert np.array_equal(pi, oi) and np.array_equal(bits(pv), bits(ov)), f"event {e}: push packet differs"
+        ctx.server_apply(w, pkt)
+        orc.apply(w, oi, ov)
+        if mixed and e % 3 == 2:
+            gi, gv = packet_to_numpy(ctx, ctx.worker_pull(w))
+            qi, qv = orc.pull(w)
+        else:
+            vi, vv = ctx.var_packet(ctx.worker_pull_all(w))
+            gi, gv = vi.cpu().numpy().view(np.uint32), vv.cpu().numpy()
+            qi, qv, held = orc.pull_all(w, cap)
+            assert held <= cap
+            assert not ctx.state(dgs.DGS_D, w).any()                       # Eq. 4: v_k = M after the pull
+        assert np.array_equal(gi, qi), f"event {e}: pull index set differs"
+        assert np.array_equal(bits(gv), bits(qv)), f"event {e}: pull values differ"
+        assert ctx.status() == 0
+    from _replay import compare_state
+    compare_state(ctx, orc, wl.num_workers, keep_local)
+    for q in range(wl.num_workers):
+        assert dgs.dgs_prev(ctx.handle, q) == orc.prev(q)
+    return ctx, orc
+
+
+@pytest.mark.parametrize("flags,mixed", [(0, False), (dgs.DGS_KEEP_LOCAL_MODEL, False), (dgs.DGS_KEEP_LOCAL_MODEL, True),
+                                         (dgs.DGS_SINGLE_STREAM, True)])
+def test_full_pull_trajectory_small_ragged(flags, mixed):
+    wl = W.custom("ragged", [300, 7, 5000, 64, 1, 2049, 1531], 3, 30, 20_000, grad_kind="normal", grad_scale=1e-2)
+    replay_full_pull(wl, flags=flags, mixed=mixed)
+
+
+def test_full_pull_many_workers_several_tiles():
+    # 8 workers in a cycle over 600 K parameters: every pull sends what the seven others and the worker itself pushed
+    wl = W.custom("full", [262_144, 70_001, 517, 262_144, 5_194], 8, 40, 2_000, grad_kind="laplace", schedule_kind="cyclic")
+    ctx, orc = replay_full_pull(wl, capacity=8 * wl.K_push, flags=dgs.DGS_KEEP_LOCAL_MODEL)
+    # Eq. 5: a worker that has just pulled holds the global model (up to the rounding of summing differences)
+    w = int(wl.schedule()[-1])
+    assert torch.allclose(ctx.state(dgs.DGS_THETA_LOCAL, w), ctx.state(dgs.DGS_THETA), rtol=0, atol=1e-6)
+
+
+def test_full_pull_overflow_sends_the_lowest_indices_and_reports():
+    wl = W.custom("overflow", [40_000, 9_001], 2, 4, 10_000, grad_kind="normal")
+    cap = 300                                  # a push carries 491 entries: the first pull cannot take them all
+    theta0 = wl.theta0()
+    orc = oracle.Oracle.from_workload(wl, theta0=theta0)
+    ctx = dgs.Context.from_workload(wl, theta0=torch.from_numpy(theta0).to(DEV), pull_all_capacity=cap)
+    g = wl.gradient(0)
+    pkt = ctx.worker_push(0, torch.from_numpy(g).to(DEV))
+    oi, ov = orc.push(0, g)
+    ctx.server_apply(0, pkt)
+    orc.apply(0, oi, ov)
+    vi, vv = ctx.var_packet(ctx.worker_pull_all(0))
+    qi, qv, held = orc.pull_all(0, cap)
+    assert held > cap and vi.numel() == cap
+    assert np.array_equal(vi.cpu().numpy().view(np.uint32), qi) and np.array_equal(bits(vv.cpu().numpy()), bits(qv))
+    assert ctx.status() == dgs.DGS_ELIMIT
+    assert np.array_equal(bits(ctx.state(dgs.DGS_D, 0).cpu().numpy()), bits(orc.state(oracle.D, 0)))   # the rest stays
+    # without a capacity the call is refused
+    plain = dgs.Context.from_workload(wl)
+    assert dgs.lib().dgs_worker_pull_all(plain.handle, 0, None) == dgs.DGS_EINVAL
+
+
 @pytest.mark.parametrize("log2n", [16, 18, 20, 22, 24])
 @pytest.mark.parametrize("ppm", W.SWEEP_PPM)
 def test_sweep_selection(log2n, ppm):
@@ -238,6 +315,68 @@ def test_sweep_selection(log2n, ppm):
     idx, val, _, _ = select_on_gpu(x, [n], [k])
     assert np.array_equal(idx, want)
     assert np.array_equal(bits(val), bits(x[want]))
+
+
+@pytest.mark.parametrize("log2n,ppm", [(26, 1000), (28, 100)])
+def test_sweep_selection_at_the_bandwidth_bound_sizes(log2n, ppm):
+    """The two largest vectors of the kernel sweep (2^26 and 2^28 elements), where the selection is
+    bound by memory bandwidth; one density each, compared with the CPU checker's selection."""
+    n = 1 << log2n
+    x = W.sweep_values(n, index=log2n)
+    k = W.k_of(n, ppm)
+    idx, val, _, ctx = select_on_gpu(x, [n], [k])
+    ctx.close()
+    want = expect_select(x, [n], [k])
+    assert np.array_equal(idx, want)
+    assert np.array_equal(bits(val), bits(x[want]))
+
+
+def test_sweep_scatter_into_33_buffers_matches_the_checker():
+    """The sweep's apply: the packet selected from a sweep vector (2^22 values, 1 %), given to
+    dgs_server_apply as a foreign packet, is subtracted from theta and from 32 difference vectors
+    (Algorithm 2, M <- M - decode(g); Eq. 3) -- compared with the CPU checker's apply, twice in a
+    row so that the second subtraction meets nonzero entries."""
+    n, N = 1 << 22, 32
+    k = W.k_of(n, 10_000)
+    x = W.sweep_values(n, index=22)
+    chosen = oracle.topk(x, k).astype(np.uint32)
+    vals = x[chosen]
+    theta0 = W.custom("t", [n], N, 1, 10_000).theta0()
+    orc = oracle.Oracle(n, N, 0.1, 0.9, [0], [n], [k], [k], theta0)
+    ctx = dgs.Context(n, N, 0.1, 0.9, [0], [n], [k], [k], torch.from_numpy(theta0).to(DEV))
+    idx_d = torch.from_numpy(chosen.view(np.int32)).to(DEV)
+    val_d = torch.from_numpy(vals).to(DEV)
+    pkt = dgs.dgs_packet(idx_d.data_ptr(), val_d.data_ptr(), k)
+    for _ in range(2):
+        ctx.server_apply(0, pkt)
+        orc.apply(0, chosen, vals)
+    assert ctx.status() == 0
+    assert np.array_equal(bits(ctx.state(dgs.DGS_THETA).cpu().numpy()), bits(orc.state(oracle.THETA)))
+    for q in range(N):
+        assert np.array_equal(bits(ctx.state(dgs.DGS_D, q).cpu().numpy()), bits(orc.state(oracle.D, q))), f"D[{q}]"
+    # the block bounds the scatter maintains still let a pull find the largest entries (Eq. 6a)
+    gi, gv = packet_to_numpy(ctx, ctx.worker_pull(5))
+    qi, qv = orc.pull(5)
+    assert np.array_equal(gi, qi) and np.array_equal(bits(gv), bits(qv))
+
+
+def test_a_wait_that_cannot_end_gives_up_and_reports():
+    """Every device-side wait of the library is bounded.  With DGS_TEST_STALLED_BARRIER the barrier among
+    the CTAs of the finalize kernel waits for a CTA that does not exist: each CTA must give up after its
+    poll limit, return, and leave DGS_ETIMEOUT in the status word; the device stays usable."""
+    import time
+    wl = W.custom("stall", [70_000, 513], 2, 2, 10_000)
+    ctx = dgs.Context.from_workload(wl, flags=dgs.DGS_TEST_STALLED_BARRIER)
+    g = torch.from_numpy(wl.gradient(0)).to(DEV)
+    t0 = time.perf_counter()
+    ctx.worker_push(0, g)
+    assert ctx.status() == dgs.DGS_ETIMEOUT
+    ctx.worker_pull(1)
+    assert ctx.status() == dgs.DGS_ETIMEOUT            # sticky
+    assert time.perf_counter() - t0 < 10.0
+    ctx.close()
+    # a context made afterwards on the same device runs clean
+    replay_and_compare(W.custom("after", [40_000, 517], 2, 4, 10_000))
 
 
 def test_apply_foreign_packet_and_bad_index_is_reported():
