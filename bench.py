@@ -411,8 +411,8 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
         "effective_hbm": {"algorithmic_bytes_per_event": ab, "GB/s": eff_gbs,
                           "frac_of_nominal_8TBs": eff_gbs / NOMINAL_HBM_GBS, "frac_of_peak": eff_gbs / peak,
                           "peak_GB/s": peak, "peak_kind": peak_kind},
-        "selection_routes": {"single_pass": stats1[0] - stats0[0], "two_pass": stats1[1] - stats0[1],
-                             "candidates_per_selection": (stats1[3] - stats0[3]) / max(1, 2 * K),
+        "selection_routes": {"selections": 2 * K * R, "single_pass": stats1[0] - stats0[0], "two_pass": stats1[1] - stats0[1],
+                             "candidates_per_selection": (stats1[3] - stats0[3]) / max(1, 2 * K * R),
                              "pull_chunks_read_fraction": (reads1[1] - reads0[1]) / max(1, reads1[0] - reads0[0])},
         "kernels": {k: {"ms_total": ms, "launches": c, "us_per_launch": (1e3 * ms / c if c else None),
                         "share": ms / tot_ms,

@@ -254,7 +254,15 @@ struct dgs_ctx {
   Workspace ws[kAllSets];  // push sets, then pull sets
   float inv_m;
   int sms;               // SMs of the device
-  bool light_pull;       // pulls run the ring-less form of their stream pass
+  // Which form of the pull's stream pass to launch.  The ring-less form wins when a pull reads a small part
+  // of D_w (it holds almost no shared memory beside the push passes), the staged form when it reads most of
+  // it.  The kernels count the chunks they cover and read; after every pull those two counters are copied
+  // to pinned host memory on the pull's stream, and the host looks at whatever has arrived so far (never
+  // waiting): a stale figure only means a less suitable form, the results are the same either way.
+  bool multi_worker;
+  unsigned long long* h_chunks;      // pinned: [0] chunks covered, [1] chunks read, as of some recent pull
+  unsigned long long seen_chunks[2]; // the figures at the last decision
+  bool light_now;
   int stream_grid[3];    // CTAs of the stand-alone stream pass, per mode
   int hist_grid[3];      // CTAs of the whole-input histogram pass, per mode
   int finalize_grid[3];  // CTAs of the cooperative finalize kernel, per mode
@@ -491,6 +499,26 @@ int pick_row(const dgs_ctx* c, int kind, uint64_t age) {
   return best_old >= 0 ? best_old : best;
 }
 
+// The form of the next pull's stream pass (see dgs_ctx::h_chunks): ring-less if the pulls counted since the
+// last decision read less than a third of the chunks they covered.
+bool use_light_pull(dgs_ctx* c) {
+  if (!c->multi_worker || !c->h_chunks) return false;
+  const unsigned long long covered = *(volatile unsigned long long*)&c->h_chunks[0];
+  const unsigned long long read = *(volatile unsigned long long*)&c->h_chunks[1];
+  if (covered > c->seen_chunks[0] && read >= c->seen_chunks[1]) {
+    c->light_now = 3 * (read - c->seen_chunks[1]) < covered - c->seen_chunks[0];
+    c->seen_chunks[0] = covered;
+    c->seen_chunks[1] = read;
+  }
+  return c->light_now;
+}
+// After a pull: its counters on their way to the host (on the pull's stream, nobody waits for them).
+int report_chunks(dgs_ctx* c, cudaStream_t st) {
+  if (c->h_chunks)
+    DGS_CUDA(c, cudaMemcpyAsync(c->h_chunks, c->ws[0].stats + 3, 2 * sizeof(unsigned long long), cudaMemcpyDeviceToHost, st));
+  return DGS_OK;
+}
+
 template <int MODE>
 int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age, int stream_id, int set,
                   Task& task) {
@@ -541,7 +569,7 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age
     TimedLaunch t(c, st, MODE == kPull ? DGS_KERNEL_STREAM_PULL : DGS_KERNEL_STREAM_PUSH);
     // A pull in a context with several workers shares the GPU with the push passes of later events and reads
     // only a small part of D_w: it takes the form of the pass that holds no ring of stages.
-    if (MODE == kPull && c->light_pull)
+    if (MODE == kPull && use_light_pull(c))
       k_pull_light<<<c->stream_grid[MODE], kThreads, 0, st>>>(ws, a);
     else
       k_stream<MODE><<<c->stream_grid[MODE], kThreads, StreamRing<MODE>::kBytes, st>>>(ws, a);
@@ -600,6 +628,7 @@ void destroy_ctx(dgs_ctx* c) {
     if (c->st[i] && (i == 0 || c->st[i] != c->st[0])) cudaStreamDestroy(c->st[i]);
     if (c->ev_tail[i]) cudaEventDestroy(c->ev_tail[i]);
   }
+  if (c->h_chunks) cudaFreeHost(c->h_chunks);
   if (c->ev_in) cudaEventDestroy(c->ev_in);
   for (int i = 0; i < kNumStreams; ++i)
     for (cudaEvent_t e : c->ev_ring[i]) cudaEventDestroy(e);
@@ -710,7 +739,14 @@ int dgs_init(const dgs_config* cfg, dgs_ctx** out) {
   INIT_CUDA(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
   if (!coop) return fail(DGS_ECUDA);
   c->sms = sms;
-  c->light_pull = cfg->num_workers > 1;
+  c->multi_worker = cfg->num_workers > 1;
+  c->h_chunks = nullptr;
+  c->seen_chunks[0] = c->seen_chunks[1] = 0;
+  c->light_now = false;
+  if (c->multi_worker) {
+    INIT_CUDA(cudaHostAlloc(reinterpret_cast<void**>(&c->h_chunks), 2 * sizeof(unsigned long long), cudaHostAllocDefault));
+    c->h_chunks[0] = c->h_chunks[1] = 0;
+  }
   if (occupancy_grids<kPushSam>(c, sms) != DGS_OK || occupancy_grids<kPushResidual>(c, sms) != DGS_OK ||
       occupancy_grids<kPull>(c, sms) != DGS_OK)
     return fail(DGS_ECUDA);
@@ -995,6 +1031,8 @@ int pull_impl(dgs_ctx* c, uint32_t worker, dgs_packet* out) {
   const uint64_t age = c->timestamp - (c->prev[worker] < 0 ? 0 : (uint64_t)c->prev[worker]);
   rc = launch_select<kPull>(c, a, worker, age, stream_id, set, task);
   if (rc != DGS_OK) return rc;
+  rc = report_chunks(c, c->st[stream_id]);
+  if (rc != DGS_OK) return rc;
   c->prev[worker] = (int64_t)c->timestamp;
   c->pull_count += 1;
   if (out) {
@@ -1037,7 +1075,7 @@ int pull_all_impl(dgs_ctx* c, uint32_t worker, dgs_var_packet* out) {
   if (rc != DGS_OK) return rc;
   {
     TimedLaunch t(c, st, DGS_KERNEL_STREAM_PULL);
-    if (c->light_pull)
+    if (use_light_pull(c))
       k_pull_light<<<c->stream_grid[kPull], kThreads, 0, st>>>(ws, a);
     else
       k_stream<kPull><<<c->stream_grid[kPull], kThreads, StreamRing<kPull>::kBytes, st>>>(ws, a);
@@ -1054,6 +1092,8 @@ int pull_all_impl(dgs_ctx* c, uint32_t worker, dgs_var_packet* out) {
     c->launches += 1;
   }
   rc = task_end(c, task);
+  if (rc != DGS_OK) return rc;
+  rc = report_chunks(c, st);
   if (rc != DGS_OK) return rc;
   c->prev[worker] = (int64_t)c->timestamp;
   c->pull_count += 1;

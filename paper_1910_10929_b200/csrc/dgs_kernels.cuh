@@ -35,8 +35,7 @@ constexpr int kBins1 = 2048;        // key bits 30..20
 constexpr int kBins2 = 1024;        // key bits 19..10
 constexpr int kBins3 = 1024;        // key bits  9..0
 constexpr uint32_t kFull = 0xFFFFFFFFu;
-constexpr uint32_t kSpecFactor = 2; // aim for max(2k, k+64) candidates next time
-constexpr uint32_t kSpecSlack = 64;
+constexpr uint32_t kSpecSlack = 64; // a carried bound aims at max(1.5 k, k + 64) candidates next time
 constexpr int kMaxGrid = 512;       // upper bound on the grid of a stream pass (= parts of the candidate buffer)
 constexpr int kMaxWorkers = 320;    // upper bound on the grid of finalize
 constexpr uint32_t kSpinLimit = 1u << 22;  // bounded waits: give up and report after this many polls
@@ -91,7 +90,7 @@ struct Workspace {
   uint32_t* hist3;        // [S][kBins3]
   SegSel* sel;            // [S]
   uint32_t* L_safe;       // [S] bound from the whole-input histogram (two-pass route)
-  uint32_t* L_wide;       // [S] from the same histogram: the bound that admits max(3k, k+64) entries
+  uint32_t* L_wide;       // [S] from the same histogram: the bound that admits about max(1.5 k, k+64) entries
   uint32_t* sync;         // [kNumSyncWords]
   int* status;            // sticky device status word
   // [kNumStats] counters: [0] single-pass selections, [1] two-pass selections, [2] candidates seen,
@@ -121,6 +120,21 @@ struct SelArgs {
 };
 
 __device__ __forceinline__ uint32_t key_of(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
+// candidates a carried bound should admit for a selection of k entries
+__device__ __forceinline__ uint32_t spec_want(uint32_t k) { return max(k + k / 2, k + kSpecSlack); }
+// A bound inside a bin of the first-level histogram (key bits 30..20 = bin): `need` of the bin's `pop`
+// entries are wanted, counted from the largest down; the bin's keys are taken as evenly spread over
+// [lo, hi), lo being the bin's lower edge or the bound that was in force if that cut the bin.  A quarter
+// more than needed is admitted.  Only advice for a later selection: results never depend on it.
+__device__ __forceinline__ uint32_t bound_inside_bin(uint32_t bin, uint32_t need, uint32_t pop, uint32_t floor_key) {
+  const uint32_t hi = (bin + 1u) << 20;
+  uint32_t lo = bin << 20;
+  if (floor_key > lo && floor_key < hi) lo = floor_key;
+  const uint32_t width = hi - lo;
+  const float f = fminf(1.f, 1.25f * (float)need / (float)max(pop, 1u) + 0.02f);
+  const uint32_t take = (uint32_t)ceilf(f * (float)width);
+  return hi - min(width, take);
+}
 __device__ __forceinline__ uint32_t lanemask_lt() {
   uint32_t m;
   asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
@@ -1115,12 +1129,13 @@ __global__ void __maxnreg__(64) k_finalize(Workspace ws, SelArgs a) {
         uint32_t* h = ws.hist1 + (size_t)s * kBins1;
         const uint32_t k = ws.segs[s].k[PM];
         const uint32_t total = block_pick<kBins1>(h, k, bin, krem, sh.warp_scan, sh.res);
-        uint32_t wbin = 0, wrem;
-        const uint32_t want = max(k * kSpecFactor, k + kSpecSlack);
+        uint32_t wbin = 0, wrem = 0;
+        const uint32_t want = spec_want(k);
         if (total >= want) block_pick<kBins1>(h, want, wbin, wrem, sh.warp_scan, sh.res);
         if (threadIdx.x == 0) {
           ws.L_safe[s] = bin << 20;
-          ws.L_wide[s] = wbin << 20;   // 0 (everything) when the layer has fewer than `want` entries
+          // 0 (everything) when the layer has fewer than `want` entries
+          ws.L_wide[s] = total >= want ? bound_inside_bin(wbin, wrem, __ldcg(h + wbin), 0u) : 0u;
         }
         __syncthreads();
         for (int b = threadIdx.x; b < kBins1; b += kThreads) h[b] = 0;
@@ -1195,24 +1210,29 @@ __global__ void __maxnreg__(64) k_finalize(Workspace ws, SelArgs a) {
         }
         if (owner && a.speculate) {
           // bound suggested for a later selection on this layer
-          const uint32_t want = max(k * kSpecFactor, k + kSpecSlack);
+          const uint32_t want = spec_want(k);
           uint32_t lbin, lrem;
+          uint32_t lkey;   // the bound itself
           if (total >= want) {
             block_pick<kBins1>(h, want, lbin, lrem, sh.warp_scan, sh.res);
+            const uint32_t in_force = (redo || a.force_two_pass) ? __ldcg(ws.L_safe + s) : a.L_in[s];
+            lkey = bound_inside_bin(lbin, lrem, __ldcg(h + lbin), in_force);
           } else if (redo || a.force_two_pass) {
-            lbin = __ldcg(ws.L_wide + s) >> 20;   // known exactly from the histogram of the whole input
+            lkey = __ldcg(ws.L_wide + s);         // known from the histogram of the whole input
+            lbin = lkey >> 20;
           } else {
             // fewer candidates than wished for and nothing known below the bound: lower it by half an octave
             const uint32_t used = a.L_in[s] >> 20;
             lbin = used > 4 ? used - 4 : 0;
+            lkey = lbin << 20;
           }
           __syncthreads();
           // A bound of zero makes every element of the layer a candidate (zeros included).  That is fine for a
           // layer not much larger than the wished-for number of candidates; for a large one, no bound at all is
           // the better advice: the next selection finds nothing, notices, and takes its bound from a histogram.
           const uint32_t layer_cap = (ws.segs[s].tile_end - ws.segs[s].tile_begin) * (uint32_t)kWarpTile;
-          const bool flood = lbin == 0 && layer_cap / 8 > want;
-          if (threadIdx.x == 0) a.L_next[s] = flood ? 0xFFFFFFFFu : lbin << 20;
+          const bool flood = lkey == 0 && layer_cap / 8 > want;
+          if (threadIdx.x == 0) a.L_next[s] = flood ? 0xFFFFFFFFu : lkey;
         }
       }
       if (!everyone_picks) {   // the histogram has served; with one layer the others may still be reading it
@@ -1498,7 +1518,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_hist_all(Workspace ws, SelArgs 
 }
 
 // one CTA per layer (strided): L_safe = lower edge of the top-11-bit bin holding the k-th largest key,
-// L_wide = the same for the max(3k, k+64)-th largest (the bound suggested for later selections)
+// L_wide = a bound that admits about max(1.5 k, k+64) entries (the bound suggested for later selections)
 template <int MODE>
 __global__ void __launch_bounds__(kThreads) k_pick_lower(Workspace ws) {
   __shared__ unsigned long long s_warp[kWarps];
@@ -1509,12 +1529,12 @@ __global__ void __launch_bounds__(kThreads) k_pick_lower(Workspace ws) {
     uint32_t* h = ws.hist1 + (size_t)s * kBins1;
     const uint32_t k = ws.segs[s].k[PM];
     const uint32_t total = block_pick<kBins1>(h, k, bin, krem, s_warp, s_res);
-    uint32_t wbin = 0, wrem;
-    const uint32_t want = max(k * kSpecFactor, k + kSpecSlack);
+    uint32_t wbin = 0, wrem = 0;
+    const uint32_t want = spec_want(k);
     if (total >= want) block_pick<kBins1>(h, want, wbin, wrem, s_warp, s_res);
     if (threadIdx.x == 0) {
       ws.L_safe[s] = bin << 20;
-      ws.L_wide[s] = wbin << 20;
+      ws.L_wide[s] = total >= want ? bound_inside_bin(wbin, wrem, __ldcg(h + wbin), 0u) : 0u;
     }
     __syncthreads();
     for (int b = threadIdx.x; b < kBins1; b += kThreads) h[b] = 0;
