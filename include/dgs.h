@@ -34,6 +34,13 @@
  *     was made.  Results (packets, state) are complete for that stream after dgs_flush,
  *     and for the host after any call that is documented to wait.  One host thread per
  *     context.
+ *   - The library's streams are eleven (four for pushes, one for the apply, six for pulls).
+ *     The CUDA driver maps streams onto a fixed number of hardware queues, 8 unless the
+ *     environment variable CUDA_DEVICE_MAX_CONNECTIONS says otherwise, and streams that
+ *     share a queue run one after the other.  The variable is read when the process creates
+ *     its CUDA context, so a process that wants the overlap must set it (to 12 or more; 32
+ *     is the most) BEFORE its first CUDA call; the library cannot do it later.  Results do
+ *     not depend on it, only speed does.  dgs_hardware_queues tells what the process has.
  *   - Every function returns DGS_OK (0) or a negative dgs_error.  Nothing aborts,
  *     throws or waits without bound.
  */
@@ -251,6 +258,13 @@ int dgs_timing_read(dgs_ctx* ctx, double ms[DGS_NUM_KERNELS], uint64_t count[DGS
  * of dgs_timing_read do not include these launches). */
 int dgs_timing_trace(dgs_ctx* ctx, uint32_t cap, float* start_ms, float* stop_ms, int32_t* kernel, int32_t* stream,
                      uint32_t* count);
+
+/* How many hardware queues the library's streams want (*needed: its own streams plus the caller's)
+ * and how many the process asked the driver for (*configured: CUDA_DEVICE_MAX_CONNECTIONS as the
+ * process environment has it now, 8 if unset or unreadable).  configured < needed means that some of
+ * the library's streams share a queue and their kernels do not overlap.  No GPU work; either
+ * pointer may be NULL.  (No counterpart in the paper.) */
+int dgs_hardware_queues(int* needed, int* configured);
 
 /* The cudaError_t of the last failed runtime call of this context (0 if none). */
 int dgs_last_cuda_error(dgs_ctx* ctx);

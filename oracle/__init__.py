@@ -52,7 +52,9 @@ def _load():
         u64, u32, f32, vp = C.c_uint64, C.c_uint32, C.c_float, C.c_void_p
         L.dgs_oracle_topk.argtypes = [vp, u64, u64, vp]
         L.dgs_oracle_topk.restype = None
-        L.dgs_oracle_create.argtypes = [u64, u32, f32, f32, u32, vp, vp, vp, vp, vp, C.c_int, C.c_int]
+        L.dgs_oracle_create.argtypes = [u64, u32, f32, f32, u32, vp, vp, vp, vp, vp, C.c_int, C.c_int, C.c_int]
+        L.dgs_oracle_round16.argtypes = [f32, C.c_int]
+        L.dgs_oracle_round16.restype = f32
         L.dgs_oracle_create.restype = vp
         L.dgs_oracle_free.argtypes = [vp]
         L.dgs_oracle_free.restype = None
@@ -86,7 +88,13 @@ def topk(x: np.ndarray, k: int) -> np.ndarray:
     return out
 
 
+def round16(x: float, fmt: int) -> np.float32:
+    """A packet value in the 16-bit format fmt (1: bfloat16, 2: binary16 saturating at 65504), as float32."""
+    return np.float32(_load().dgs_oracle_round16(np.float32(x), int(fmt)))
+
+
 THETA, U, D, THETA_LOCAL = 0, 1, 2, 3
+FP32, BF16, FP16 = 0, 1, 2
 
 
 class Oracle:
@@ -94,7 +102,7 @@ class Oracle:
 
     def __init__(self, n: int, num_workers: int, lr: float, momentum: float,
                  seg_offset, seg_len, k_push, k_pull, theta0: np.ndarray,
-                 keep_local: bool = False, residual_mode: bool = False):
+                 keep_local: bool = False, residual_mode: bool = False, packet_format: int = 0):
         L = _load()
         self.n, self.N = int(n), int(num_workers)
         so = np.ascontiguousarray(seg_offset, dtype=np.uint64)
@@ -106,15 +114,15 @@ class Oracle:
         self.K_push, self.K_pull = int(kp.sum()), int(kl.sum())
         self._h = L.dgs_oracle_create(self.n, self.N, np.float32(lr), np.float32(momentum),
                                       so.shape[0], _p(so), _p(sl), _p(kp), _p(kl), _p(th),
-                                      int(keep_local), int(residual_mode))
+                                      int(keep_local), int(residual_mode), int(packet_format))
         self._L = L
 
     @classmethod
     def from_workload(cls, wl, keep_local: bool = False, residual_mode: bool = False,
-                      theta0: Optional[np.ndarray] = None) -> "Oracle":
+                      theta0: Optional[np.ndarray] = None, packet_format: int = 0) -> "Oracle":
         return cls(wl.n, wl.num_workers, wl.lr, wl.momentum, wl.seg_offset, wl.seg_len,
                    wl.k_push, wl.k_pull, wl.theta0() if theta0 is None else theta0,
-                   keep_local, residual_mode)
+                   keep_local, residual_mode, packet_format)
 
     def push(self, w: int, grad: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
         g = np.ascontiguousarray(grad, dtype=np.float32)

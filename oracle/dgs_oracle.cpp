@@ -26,6 +26,10 @@
 //   * unsent velocity entries are multiplied once by fl(1/m)  (Eq. 12 form).
 //   * a pull without secondary compression sends every entry of D_k that is not zero
 //     (+0 and -0 both count as zero) and clears it.
+//   * with 16-bit packet values (not in the paper's algorithms; its closing section names the
+//     direction): selection by the unrounded magnitudes; the packet carries q = round16(value); a
+//     push leaves the worker's velocity as Eq. 12 says (no residual exists to take t - q); a pull
+//     lowers D_k by q, so that what rounding left behind stays with the server (Eq. 6b).
 //
 // parity pins: see tests/test_oracle_*.py (brute-force sort, hand-worked example,
 // dense limit = serial momentum ASGD, Eq. 13 telescoping, Eq. 12, exact split).
@@ -41,6 +45,47 @@ inline uint32_t key_of(float x) {          // |x| as an unsigned integer, monoto
   uint32_t b;
   std::memcpy(&b, &x, 4);
   return b & 0x7FFFFFFFu;
+}
+
+// Packet values in a 16-bit floating-point format (the paper's closing section proposes combining the
+// method with other compression; here: the VALUES of a packet are rounded, the selection is untouched).
+// fmt 0: none.  fmt 1: bfloat16 (8 exponent bits, 7 fraction bits).  fmt 2: IEEE binary16 (5 exponent
+// bits, 10 fraction bits, gradual underflow); magnitudes that would round beyond the largest finite
+// binary16 number, 65504, are sent as 65504 (no infinities in a packet).  Round to nearest, ties to even.
+// The result is returned as the float32 number with that value.  Inputs are finite.
+float round16(float x, int fmt) {
+  uint32_t b;
+  std::memcpy(&b, &x, 4);
+  const uint32_t sign = b & 0x80000000u;
+  uint32_t m = b & 0x7FFFFFFFu;            // bits of |x|
+  if (fmt == 1) {
+    m += 0x7FFFu + ((m >> 16) & 1u);       // nearest multiple of 2^16 in the bit pattern, ties to even
+    m &= 0xFFFF0000u;
+    if (m >= 0x7F800000u) m = 0x7F7F0000u; // would be infinite: largest finite bfloat16
+  } else if (fmt == 2) {
+    if (m >= 0x477FF000u) {                // |x| >= 65520 = the midpoint above 65504: saturate
+      m = 0x477FE000u;                     // 65504
+    } else if (m >= 0x38800000u) {         // |x| >= 2^-14: a normal binary16, 13 fraction bits are dropped
+      m += 0xFFFu + ((m >> 13) & 1u);
+      m &= 0xFFFFE000u;
+    } else {
+      // below 2^-14 binary16 steps by 2^-24: |x| / 2^-24 rounded to an integer (exact scaling by a power of two)
+      float ax;
+      std::memcpy(&ax, &m, 4);
+      const float scaled = ax * 16777216.0f;               // exact: < 2^10
+      float r = static_cast<float>(static_cast<int>(scaled));
+      const float frac = scaled - r;                         // exact
+      if (frac > 0.5f || (frac == 0.5f && (static_cast<int>(r) & 1))) r += 1.0f;
+      const float back = r * (1.0f / 16777216.0f);           // exact
+      std::memcpy(&m, &back, 4);
+    }
+  } else {
+    return x;
+  }
+  m |= sign;
+  float y;
+  std::memcpy(&y, &m, 4);
+  return y;
 }
 
 // TOPK(x, k): order by (key descending, index ascending), take the first k.
@@ -72,6 +117,7 @@ struct Oracle {
   float lr = 0, m = 0, inv_m = 0;
   int keep_local = 0;
   int residual_mode = 0;                   // 1: Algorithm 1 (plain residual, no momentum)
+  int packet_format = 0;                   // 0: float32 values; 1: bfloat16; 2: binary16 (see round16)
   std::vector<uint64_t> off, len;
   std::vector<uint32_t> k_push, k_pull;
   std::vector<float> theta;
@@ -85,6 +131,9 @@ struct Oracle {
 
 extern "C" {
 
+// The rounding of packet values, on its own (for pinning it).
+float dgs_oracle_round16(float x, int fmt) { return round16(x, fmt); }
+
 // Standalone selection, for pinning TOPK by brute force. out_pos receives k ascending positions.
 void dgs_oracle_topk(const float* x, uint64_t len, uint64_t k, uint64_t* out_pos) {
   std::vector<uint64_t> c;
@@ -95,8 +144,9 @@ void dgs_oracle_topk(const float* x, uint64_t len, uint64_t k, uint64_t* out_pos
 void* dgs_oracle_create(uint64_t n, uint32_t N, float lr, float m, uint32_t S,
                         const uint64_t* seg_off, const uint64_t* seg_len,
                         const uint32_t* k_push, const uint32_t* k_pull,
-                        const float* theta0, int keep_local, int residual_mode) {
+                        const float* theta0, int keep_local, int residual_mode, int packet_format) {
   Oracle* o = new Oracle;
+  o->packet_format = packet_format;
   o->n = n; o->N = N; o->S = S; o->lr = lr; o->m = m;
   o->inv_m = 1.0f / m;                     // one IEEE division, then used as a constant
   o->keep_local = keep_local;
@@ -149,10 +199,14 @@ uint64_t dgs_oracle_push(void* h, uint32_t w, const float* grad, uint32_t* out_i
     }
     for (uint64_t p : chosen) {             // sent entries
       const uint64_t i = base + p;
+      const float q = round16(t[i], o.packet_format);   // what the packet carries
       out_idx[cnt] = static_cast<uint32_t>(i);
-      out_val[cnt] = t[i];
+      out_val[cnt] = q;
       ++cnt;
-      u[i] = o.residual_mode ? 0.0f : t[i]; // Eq. 12 upper branch / Algorithm 1 masks the sent part out
+      // Eq. 12 upper branch: the velocity of a sent entry stays t (SAMomentum keeps no residual, so the
+      // rounding of a packet value is not fed back).  Algorithm 1: the sent part leaves the residual,
+      // which keeps what the packet did not carry (t - q; zero without rounding).
+      u[i] = o.residual_mode ? t[i] - q : t[i];
     }
   }
   return cnt;
@@ -180,11 +234,12 @@ uint64_t dgs_oracle_pull(void* h, uint32_t w, uint32_t* out_idx, float* out_val)
     topk(D.data() + base, o.len[s], o.k_pull[s], chosen);
     for (uint64_t p : chosen) {
       const uint64_t i = base + p;
+      const float q = round16(D[i], o.packet_format);                       // what the packet carries
       out_idx[cnt] = static_cast<uint32_t>(i);
-      out_val[cnt] = D[i];
+      out_val[cnt] = q;
       ++cnt;
-      if (o.keep_local) o.theta_local[w][i] = o.theta_local[w][i] + D[i];   // Eq. 5
-      D[i] = 0.0f;                                                          // v_k <- v_k + G
+      if (o.keep_local) o.theta_local[w][i] = o.theta_local[w][i] + q;      // Eq. 5
+      D[i] = D[i] - q;                            // v_k <- v_k + G (Eq. 6b): zero, or what rounding left behind
     }
   }
   o.prev[w] = static_cast<int64_t>(o.stamp);
@@ -204,10 +259,11 @@ uint64_t dgs_oracle_pull_all(void* h, uint32_t w, uint32_t* out_idx, float* out_
   for (uint64_t i = 0; i < o.n; ++i) {
     if (D[i] != 0.0f) {
       if (cnt < cap) {
+        const float q = round16(D[i], o.packet_format);
         out_idx[cnt] = static_cast<uint32_t>(i);
-        out_val[cnt] = D[i];
-        if (o.keep_local) o.theta_local[w][i] = o.theta_local[w][i] + D[i];   // Eq. 5
-        D[i] = 0.0f;                                                          // v_k <- v_k + G = M (Eq. 4)
+        out_val[cnt] = q;
+        if (o.keep_local) o.theta_local[w][i] = o.theta_local[w][i] + q;      // Eq. 5
+        D[i] = D[i] - q;                          // v_k <- v_k + G = M (Eq. 4), up to what rounding left behind
       }
       ++cnt;
     }

@@ -31,7 +31,7 @@ EXPORTS = (
     "dgs_event", "dgs_flush", "dgs_event_host", "dgs_state_ptr", "dgs_state_load", "dgs_status", "dgs_stats", "dgs_pull_read_stats",
     "dgs_prev", "dgs_launch_count", "dgs_last_cuda_error", "dgs_free", "dgs_error_string",
     "dgs_timing_enable", "dgs_timing_read", "dgs_timing_trace", "dgs_topk_encode_static",
-    "dgs_topk_encode_static_status",
+    "dgs_topk_encode_static_status", "dgs_hardware_queues",
 )
 DGS_ELIMIT = -6
 DGS_STATIC_MAX_N = 1 << 20
@@ -96,6 +96,7 @@ def lib() -> C.CDLL:
         L.dgs_last_cuda_error.argtypes = [vp]
         L.dgs_topk_encode_static.argtypes = [vp, u32, u32, vp, vp, vp]
         L.dgs_topk_encode_static_status.argtypes = [vp, C.POINTER(i32)]
+        L.dgs_hardware_queues.argtypes = [C.POINTER(i32), C.POINTER(i32)]
         L.dgs_timing_enable.argtypes = [vp, i32]
         L.dgs_timing_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
         L.dgs_timing_trace.argtypes = [vp, u32, C.POINTER(C.c_float), C.POINTER(C.c_float), C.POINTER(C.c_int32),
@@ -253,6 +254,13 @@ def dgs_topk_encode_static_status(stream: int = 0) -> int:
     out = C.c_int(0)
     _check(lib().dgs_topk_encode_static_status(stream or None, C.byref(out)), "dgs_topk_encode_static_status")
     return int(out.value)
+
+
+def dgs_hardware_queues() -> Tuple[int, int]:
+    """(hardware queues the library's streams want, queues the process asked the driver for)."""
+    a, b = C.c_int(0), C.c_int(0)
+    _check(lib().dgs_hardware_queues(C.byref(a), C.byref(b)), "dgs_hardware_queues")
+    return int(a.value), int(b.value)
 
 
 def dgs_free(ctx: int) -> None:

@@ -16,6 +16,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstddef>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -1371,6 +1372,20 @@ int dgs_timing_trace(dgs_ctx* c, uint32_t cap, float* start_ms, float* stop_ms, 
   *count = (uint32_t)m;
   c->ev_kernel.clear();
   c->ev_stream.clear();
+  return DGS_OK;
+}
+
+int dgs_hardware_queues(int* needed, int* configured) {
+  if (needed) *needed = kNumStreams + 1;
+  if (configured) {
+    int v = 8;   // the driver's default
+    if (const char* e = std::getenv("CUDA_DEVICE_MAX_CONNECTIONS")) {
+      char* endp = nullptr;
+      const long x = std::strtol(e, &endp, 10);
+      if (endp != e && x >= 1 && x <= 32) v = (int)x;
+    }
+    *configured = v;
+  }
   return DGS_OK;
 }
 

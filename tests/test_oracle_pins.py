@@ -72,15 +72,18 @@ def _read_golden(path):
     return head, events
 
 
-@pytest.mark.parametrize("name", ["hand_example.txt", "hand_example_algorithm1.txt", "hand_example_full_pull.txt"])
+@pytest.mark.parametrize("name", ["hand_example.txt", "hand_example_algorithm1.txt", "hand_example_full_pull.txt",
+                                  "hand_example_bf16_packets.txt"])
 def test_hand_example(name):
     head, events = _read_golden(os.path.join(GOLDEN, name))
     n, N, k = int(head["n"][0]), int(head["workers"][0]), int(head["k"][0])
     theta0 = np.array([float(v) for v in head["theta0"]], np.float32)
     residual = head.get("mode", ["momentum"])[0] == "residual"       # worker rule of Algorithm 1
     full_pull = head.get("mode", ["momentum"])[0] == "full_pull"     # Algorithm 2 without secondary compression
+    fmt = oracle.BF16 if head.get("mode", ["momentum"])[0] == "bf16" else oracle.FP32
     o = oracle.Oracle(n, N, float(head["lr"][0]), float(head["momentum"][0]),
-                      [0], [n], [k], [k], theta0, keep_local=True, residual_mode=residual)
+                      [0], [n], [k], [k], theta0, keep_local=True, residual_mode=residual,
+                      packet_format=fmt)
     assert o.timestamp == 0 and [o.prev(q) for q in range(N)] == [-1] * N
     for ev in events:
         w = ev["worker"]
@@ -223,6 +226,64 @@ def test_piecewise_state_and_exact_split(residual_mode):
             assert np.allclose(o.state(oracle.THETA_LOCAL, q) + o.state(oracle.D, q),
                                o.state(oracle.THETA), rtol=0, atol=1e-6)
     assert o.timestamp == wl.num_events
+
+
+# ---- 16-bit packet values ---------------------------------------------------------------------
+def test_round16_is_the_library_conversion_and_saturates():
+    import torch
+    r = np.random.default_rng(0)
+    x = r.standard_normal(20000).astype(np.float32) * np.float32(10.0) ** r.integers(-9, 5, 20000).astype(np.float32)
+    x = np.concatenate([x, np.array([0, -0.0, 1 + 2 ** -8, 1 + 2 ** -8 + 2 ** -9, 65504, 65519.99, 2 ** -24, 2 ** -25,
+                                     2 ** -25 * 1.0001, 3 * 2 ** -25, 6e-8, 2 ** -14, 2 ** -14 - 2 ** -26], np.float32)])
+    half = np.array([oracle.round16(v, oracle.FP16) for v in x], np.float32)
+    inside = np.abs(x) < 65520
+    want = x[inside].astype(np.float16).astype(np.float32)              # numpy's IEEE binary16 conversion
+    assert np.array_equal(half[inside].view(np.uint32), want.view(np.uint32))
+    assert np.all(np.abs(half[~inside]) == 65504) and np.array_equal(np.sign(half[~inside]), np.sign(x[~inside]))
+    bf = np.array([oracle.round16(v, oracle.BF16) for v in x], np.float32)
+    want = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()   # torch's bfloat16 conversion
+    assert np.array_equal(bf.view(np.uint32), want.view(np.uint32))
+    # by hand: ties go to the even neighbour; beyond the largest finite binary16 the value saturates
+    assert oracle.round16(1 + 2 ** -8, oracle.BF16) == 1.0 and oracle.round16(1 + 3 * 2 ** -8, oracle.BF16) == 1 + 2 ** -6
+    assert oracle.round16(1 + 2 ** -11, oracle.FP16) == 1.0 and oracle.round16(1 + 3 * 2 ** -11, oracle.FP16) == 1 + 2 ** -9
+    assert oracle.round16(65520.0, oracle.FP16) == 65504.0 and oracle.round16(-1e9, oracle.FP16) == -65504.0
+    assert oracle.round16(2 ** -25, oracle.FP16) == 0.0 and oracle.round16(3 * 2 ** -25, oracle.FP16) == 2 ** -23
+    assert oracle.round16(0.1, oracle.FP32) == np.float32(0.1)
+
+
+@pytest.mark.parametrize("fmt", [1, 2])
+@pytest.mark.parametrize("residual_mode", [False, True])
+def test_rounded_packets_keep_the_books(fmt, residual_mode):
+    """With 16-bit packet values: what a packet carries is the rounded selected value; the worker's state
+    follows Eq. 12 (or keeps t - q under Algorithm 1); the server's residual keeps what a pull's rounding
+    left behind, so theta_k + D_k still equals theta (Eq. 3-5) up to float32 rounding."""
+    wl = W.custom("mini", [300, 7, 1000, 64], 3, 12, 20_000, grad_kind="normal", grad_scale=1e-2)
+    o = oracle.Oracle.from_workload(wl, keep_local=True, residual_mode=residual_mode, packet_format=fmt)
+    m, lr = np.float32(wl.momentum), np.float32(wl.lr)
+    for e, w in enumerate(wl.schedule()):
+        w = int(w)
+        g = wl.gradient(e)
+        u_before = o.state(oracle.U, w).copy()
+        t = (u_before + lr * g) if residual_mode else (m * u_before + lr * g)
+        pi, pv = o.push(w, g)
+        q = np.array([oracle.round16(v, fmt) for v in t[pi]], np.float32)
+        assert np.array_equal(pv, q)
+        u_after = o.state(oracle.U, w)
+        assert np.array_equal(u_after[pi], (t[pi] - q) if residual_mode else t[pi])
+        o.apply(w, pi, pv)
+        Dw = o.state(oracle.D, w).copy()
+        gi, gv = o.pull(w)
+        q = np.array([oracle.round16(v, fmt) for v in Dw[gi]], np.float32)
+        assert np.array_equal(gv, q)
+        left = o.state(oracle.D, w)
+        assert np.array_equal(left[gi], Dw[gi] - q)                       # the remainder stays with the server
+        rest = np.ones(wl.n, bool)
+        rest[gi] = False
+        assert np.array_equal(left[rest], Dw[rest])
+        assert np.all(np.abs(left[gi]) <= np.abs(Dw[gi]) * 2.0 ** -8 + 1e-45)   # at most half a step of the format
+        for q_ in range(wl.num_workers):
+            assert np.allclose(o.state(oracle.THETA_LOCAL, q_) + o.state(oracle.D, q_), o.state(oracle.THETA),
+                               rtol=0, atol=1e-6)
 
 
 # ---- pull without secondary compression: v_k = M afterwards (Eq. 4), theta_k = theta (Eq. 5) ----
