@@ -41,6 +41,14 @@
  *     its CUDA context, so a process that wants the overlap must set it (to 12 or more; 32
  *     is the most) BEFORE its first CUDA call; the library cannot do it later.  Results do
  *     not depend on it, only speed does.  dgs_hardware_queues tells what the process has.
+ *   - 16-bit packet values (DGS_PACKET_BF16 / DGS_PACKET_FP16; not part of the paper's algorithms, its
+ *     closing section names the combination with other compression as the next step): the selection is
+ *     made on the unrounded magnitudes; a packet carries q = the selected value rounded to the 16-bit
+ *     format (nearest, ties to even), stored as the float32 number with that value, so that a transport
+ *     may ship 16 bits per value.  A push leaves the worker's velocity as Eq. 12 says (a sent entry keeps
+ *     t; sparsification-aware momentum has no residual that could take t - q); under DGS_RESIDUAL_MODE
+ *     the residual keeps t - q.  A pull lowers D_k by q (Eq. 6b: v_k <- v_k + G with the G that was
+ *     sent), so what rounding left behind stays with the server and goes out with a later pull.
  *   - Every function returns DGS_OK (0) or a negative dgs_error.  Nothing aborts,
  *     throws or waits without bound.
  */
@@ -104,6 +112,8 @@ enum {
   DGS_NO_SPECULATION = 1u << 3,   /* always take the two-pass selection (histogram pass, then stream pass) */
   DGS_SINGLE_STREAM = 1u << 4,    /* enqueue every step on ONE internal stream: kernels run one after the other in
                                      call order (same results; for debugging and for timing a kernel on its own) */
+  DGS_PACKET_BF16 = 1u << 6,      /* packets carry values rounded to bfloat16 (see "16-bit packet values" below)  */
+  DGS_PACKET_FP16 = 1u << 7,      /* ... to IEEE binary16, saturating at 65504; not together with DGS_PACKET_BF16  */
   DGS_TEST_STALLED_BARRIER = 1u << 5 /* testing only: the barrier among the CTAs of the finalize kernels waits for one
                                      CTA that does not exist, with a limit of a few thousand polls.  Every wait then
                                      runs out: the kernels return early, packets and state are NOT valid, and

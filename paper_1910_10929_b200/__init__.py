@@ -24,6 +24,7 @@ LIB_PATH = os.path.join(_HERE, "libdgs.so")
 DGS_OK, DGS_EINVAL, DGS_ENOMEM, DGS_ECUDA, DGS_ETIMEOUT, DGS_ESTATE = 0, -1, -2, -3, -4, -5
 DGS_KEEP_LOCAL_MODEL, DGS_RESIDUAL_MODE, DGS_HOST_IO, DGS_NO_SPECULATION, DGS_SINGLE_STREAM = 1, 2, 4, 8, 16
 DGS_TEST_STALLED_BARRIER = 32
+DGS_PACKET_BF16, DGS_PACKET_FP16 = 64, 128
 DGS_THETA, DGS_U, DGS_D, DGS_THETA_LOCAL = 0, 1, 2, 3
 
 EXPORTS = (

@@ -77,6 +77,7 @@ int check_config(const dgs_config* c) {
   if (c->num_workers == 0 || c->num_workers > 65535) return DGS_EINVAL;
   if (c->num_segments == 0 || c->num_segments >= 65536) return DGS_EINVAL;
   if (c->pull_all_capacity > c->n) return DGS_EINVAL;
+  if ((c->flags & DGS_PACKET_BF16) && (c->flags & DGS_PACKET_FP16)) return DGS_EINVAL;
   if (!std::isfinite(c->lr)) return DGS_EINVAL;
   if (!(c->momentum > 0.0f) || !(c->momentum <= 1.0f)) return DGS_EINVAL;
   uint64_t pos = 0;
@@ -500,6 +501,10 @@ int pick_row(const dgs_ctx* c, int kind, uint64_t age) {
   return best_old >= 0 ? best_old : best;
 }
 
+inline int packet_format_of(const dgs_ctx* c) {
+  return (c->cfg.flags & DGS_PACKET_BF16) ? 1 : (c->cfg.flags & DGS_PACKET_FP16) ? 2 : 0;
+}
+
 // The form of the next pull's stream pass (see dgs_ctx::h_chunks): ring-less if the pulls counted since the
 // last decision read less than a third of the chunks they covered.
 bool use_light_pull(dgs_ctx* c) {
@@ -540,6 +545,7 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age
   if (3ull * a.pkt_count <= 48ull * kThreads * 8) fin_base = std::min(fin_base, 48);
   const int fin_grid = std::min(c->finalize_max[MODE], std::max(fin_base, (int)(a.pkt_count / 4096)));
   a.workers = (uint32_t)fin_grid;
+  a.packet_format = packet_format_of(c);
   if (c->cfg.flags & DGS_TEST_STALLED_BARRIER) {
     a.phantom_workers = 1;
     a.spin_limit = 4096;
@@ -1088,7 +1094,8 @@ int pull_all_impl(dgs_ctx* c, uint32_t worker, dgs_var_packet* out) {
   uint32_t* vc = c->at<uint32_t>(L.var_count[vslot]);
   {
     TimedLaunch t(c, st, DGS_KERNEL_FINALIZE_PULL);
-    k_emit_all<<<2 * c->sms, kThreads, 0, st>>>(ws, a.D, a.theta_local, a.blk_max, vi, vv, vc, c->cfg.pull_all_capacity);
+    k_emit_all<<<2 * c->sms, kThreads, 0, st>>>(ws, a.D, a.theta_local, a.blk_max, vi, vv, vc, c->cfg.pull_all_capacity,
+                                                packet_format_of(c));
     DGS_CUDA(c, cudaGetLastError());
     c->launches += 1;
   }

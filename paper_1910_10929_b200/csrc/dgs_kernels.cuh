@@ -117,9 +117,35 @@ struct SelArgs {
   uint32_t seq;           // launch sequence number (tags the decision word)
   uint32_t phantom_workers;  // testing only: CTAs the finalize barrier waits for beyond those launched (0 in normal use)
   uint32_t spin_limit;    // polls after which a bounded wait gives up (0: kSpinLimit)
+  int packet_format;      // 0: packets carry float32 values; 1: bfloat16; 2: binary16 (see round16)
 };
 
 __device__ __forceinline__ uint32_t key_of(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
+// A packet value in a 16-bit floating-point format, as the float32 number with that value (round to
+// nearest, ties to even).  fmt 1: bfloat16 (8 exponent bits, 7 fraction bits).  fmt 2: IEEE binary16
+// (5 exponent bits, 10 fraction bits, gradual underflow); a magnitude that would round beyond the largest
+// finite binary16 number is sent as that number, 65504.  fmt 0: the value itself.  Inputs are finite.
+__device__ __forceinline__ float round16(float x, int fmt) {
+  if (fmt == 0) return x;
+  const uint32_t b = __float_as_uint(x);
+  uint32_t m = b & 0x7FFFFFFFu;
+  if (fmt == 1) {
+    m = (m + 0x7FFFu + ((m >> 16) & 1u)) & 0xFFFF0000u;
+    if (m >= 0x7F800000u) m = 0x7F7F0000u;
+  } else if (m >= 0x477FF000u) {          // 65520 and above
+    m = 0x477FE000u;                      // 65504
+  } else if (m >= 0x38800000u) {          // 2^-14 and above: 13 fraction bits go
+    m = (m + 0xFFFu + ((m >> 13) & 1u)) & 0xFFFFE000u;
+  } else {
+    // steps of 2^-24 below 2^-14: the multiple nearest to |x| (scaling by powers of two is exact)
+    const float scaled = __fmul_rn(__uint_as_float(m), 16777216.0f);
+    const int whole = (int)scaled;        // truncation; scaled < 1024
+    const float frac = __fsub_rn(scaled, (float)whole);
+    const int up = (frac > 0.5f || (frac == 0.5f && (whole & 1))) ? 1 : 0;
+    m = __float_as_uint(__fmul_rn((float)(whole + up), 1.0f / 16777216.0f));
+  }
+  return __uint_as_float(m | (b & 0x80000000u));
+}
 // candidates a carried bound should admit for a selection of k entries
 __device__ __forceinline__ uint32_t spec_want(uint32_t k) { return max(k + k / 2, k + kSpecSlack); }
 // A bound inside a bin of the first-level histogram (key bits 30..20 = bin): `need` of the bin's `pop`
@@ -1418,16 +1444,19 @@ __global__ void __maxnreg__(64) k_finalize(Workspace ws, SelArgs a) {
       const bool sel = is_gt || (is_eq && eq_in_layer < r);
       if (sel) {
         const uint32_t pos = pkt_off + (gt_before - start.x) + min(eq_in_layer, r);
+        const float q = round16(val, a.packet_format);   // what the packet carries (val itself with float32 packets)
         if (pos < a.pkt_count) {
           a.pkt_idx[pos] = idx;
-          a.pkt_val[pos] = val;
+          a.pkt_val[pos] = q;
         } else {
           atomicMin(ws.status, -1000 - MODE);
         }
-        if (MODE == kPushResidual) out[idx] = 0.f;       // Algorithm 1: the sent part leaves v
+        // Algorithm 1: the sent part leaves v (what a rounded packet did not carry stays: val - q, else zero).
+        // Algorithm 3 keeps the sent entry's velocity t (already stored): no residual exists to take val - q.
+        if (MODE == kPushResidual) out[idx] = __fsub_rn(val, q);
         if (MODE == kPull) {
-          a.D[idx] = 0.f;                                // Eq. 6b: v_k <- v_k + G
-          if (a.theta_local) a.theta_local[idx] = __fadd_rn(a.theta_local[idx], val);  // Eq. 5
+          a.D[idx] = __fsub_rn(val, q);                  // Eq. 6b: v_k <- v_k + G; the rounding remainder stays
+          if (a.theta_local) a.theta_local[idx] = __fadd_rn(a.theta_local[idx], q);  // Eq. 5
         }
       } else {
         if (MODE == kPushSam) out[idx] = __fmul_rn(val, a.inv_m);  // Eq. 12, lower branch
@@ -1578,7 +1607,7 @@ __global__ void __launch_bounds__(kThreads) k_emit_all(Workspace ws, float* __re
                                                        float* __restrict__ theta_local,
                                                        uint32_t* __restrict__ blk_max, uint32_t* __restrict__ out_idx,
                                                        float* __restrict__ out_val, uint32_t* __restrict__ out_count,
-                                                       uint32_t capacity) {
+                                                       uint32_t capacity, int packet_format) {
   __shared__ uint32_t pre[kMaxGrid + 1], slot0[kMaxGrid];
   __shared__ unsigned long long warp_scan[kWarps];
   const uint32_t parts = ld_volatile(ws.sync + kParts);
@@ -1617,13 +1646,14 @@ __global__ void __launch_bounds__(kThreads) k_emit_all(Workspace ws, float* __re
     const uint32_t slot = slot0[lo] + (p - pre[lo]);
     const uint32_t i = __ldcg(ws.cand_idx + slot);
     const float v = __ldcg(ws.cand_val + slot);
+    const float q = round16(v, packet_format);
     out_idx[p] = i;
-    out_val[p] = v;
-    D[i] = 0.f;
-    if (theta_local != nullptr) theta_local[i] = __fadd_rn(theta_local[i], v);
+    out_val[p] = q;
+    D[i] = __fsub_rn(v, q);      // zero with float32 packets; else what rounding left behind stays (Eq. 6b)
+    if (theta_local != nullptr) theta_local[i] = __fadd_rn(theta_local[i], q);
     // the block's bound was made exact by the pass (a block without a nonzero entry already has bound 0);
-    // with everything sent the whole block is zero now
-    if (all && blk_max != nullptr) blk_max[i / kWarpTile] = 0;
+    // with everything sent unrounded the whole block is zero now
+    if (all && packet_format == 0 && blk_max != nullptr) blk_max[i / kWarpTile] = 0;
   }
   // the pass has added the candidates' top key bits to the layers' histograms: nobody reads them here
   const size_t words = (size_t)ws.num_segs * kBins1;

@@ -26,6 +26,11 @@ def max_rel_err(a: np.ndarray, b: np.ndarray) -> float:
     return float(out.max()) if out.size else 0.0
 
 
+def packet_format(flags: int) -> int:
+    """The CPU checker's packet_format for a context's flags."""
+    return oracle.BF16 if flags & dgs.DGS_PACKET_BF16 else (oracle.FP16 if flags & dgs.DGS_PACKET_FP16 else oracle.FP32)
+
+
 def packet_to_numpy(ctx: dgs.Context, pkt):
     idx, val = ctx.packet(pkt)
     return idx.cpu().numpy().view(np.uint32), val.cpu().numpy()
@@ -39,7 +44,8 @@ def replay_and_compare(wl, *, flags: int = 0, num_events=None, schedule=None, co
     keep_local = bool(flags & dgs.DGS_KEEP_LOCAL_MODEL)
     residual = bool(flags & dgs.DGS_RESIDUAL_MODE)
     theta0 = wl.theta0()
-    orc = oracle.Oracle.from_workload(wl, keep_local=keep_local, residual_mode=residual, theta0=theta0)
+    orc = oracle.Oracle.from_workload(wl, keep_local=keep_local, residual_mode=residual, theta0=theta0,
+                                      packet_format=packet_format(flags))
     ctx = dgs.Context.from_workload(wl, theta0=torch.from_numpy(theta0).to(device), flags=flags)
     sched = wl.schedule() if schedule is None else np.asarray(schedule)
     E = len(sched) if num_events is None else num_events
@@ -107,7 +113,8 @@ def replay_async_and_compare(wl, *, flags: int = 0, num_events=None, schedule=No
     pi, pv = packet_to_numpy(ctx, last[0])
     gi, gv = packet_to_numpy(ctx, last[1])
     assert ctx.status() == 0
-    orc = oracle.Oracle.from_workload(wl, keep_local=keep_local, residual_mode=residual, theta0=theta0)
+    orc = oracle.Oracle.from_workload(wl, keep_local=keep_local, residual_mode=residual, theta0=theta0,
+                                      packet_format=packet_format(flags))
     for e in range(E):
         (oi, ov), (qi, qv) = orc.event(int(sched[e]), grads_host[e])
     assert np.array_equal(pi, oi) and np.array_equal(bits(pv), bits(ov)), "last push packet differs"

@@ -88,3 +88,12 @@ def test_init_without_arena_is_rejected_before_any_gpu_work():
     h = C.c_void_p(None)
     assert dgs.lib().dgs_init(C.byref(c), C.byref(h)) == dgs.DGS_EINVAL
     assert h.value is None
+
+
+def test_hardware_queues_reports_what_the_environment_says(monkeypatch):
+    needed, configured = dgs.dgs_hardware_queues()
+    assert needed == 12                      # eleven streams of the library and the caller's
+    monkeypatch.setenv("CUDA_DEVICE_MAX_CONNECTIONS", "5")
+    assert dgs.dgs_hardware_queues() == (12, 5)
+    monkeypatch.delenv("CUDA_DEVICE_MAX_CONNECTIONS")
+    assert dgs.dgs_hardware_queues() == (12, 8)

@@ -236,7 +236,8 @@ def replay_full_pull(wl, *, flags=0, capacity=None, mixed=False, schedule=None):
     keep_local = bool(flags & dgs.DGS_KEEP_LOCAL_MODEL)
     theta0 = wl.theta0()
     cap = wl.n if capacity is None else capacity
-    orc = oracle.Oracle.from_workload(wl, keep_local=keep_local, theta0=theta0)
+    from _replay import packet_format
+    orc = oracle.Oracle.from_workload(wl, keep_local=keep_local, theta0=theta0, packet_format=packet_format(flags))
     ctx = dgs.Context.from_workload(wl, theta0=torch.from_numpy(theta0).to(DEV), flags=flags, pull_all_capacity=cap)
     sched = wl.schedule() if schedule is None else np.asarray(schedule)
     for e in range(len(sched)):
@@ -256,7 +257,8 @@ def replay_full_pull(wl, *, flags=0, capacity=None, mixed=False, schedule=None):
             gi, gv = vi.cpu().numpy().view(np.uint32), vv.cpu().numpy()
             qi, qv, held = orc.pull_all(w, cap)
             assert held <= cap
-            assert not ctx.state(dgs.DGS_D, w).any()                       # Eq. 4: v_k = M after the pull
+            if not flags & (dgs.DGS_PACKET_BF16 | dgs.DGS_PACKET_FP16):
+                assert not ctx.state(dgs.DGS_D, w).any()                   # Eq. 4: v_k = M after the pull
         assert np.array_equal(gi, qi), f"event {e}: pull index set differs"
         assert np.array_equal(bits(gv), bits(qv)), f"event {e}: pull values differ"
         assert ctx.status() == 0
@@ -272,6 +274,35 @@ def replay_full_pull(wl, *, flags=0, capacity=None, mixed=False, schedule=None):
 def test_full_pull_trajectory_small_ragged(flags, mixed):
     wl = W.custom("ragged", [300, 7, 5000, 64, 1, 2049, 1531], 3, 30, 20_000, grad_kind="normal", grad_scale=1e-2)
     replay_full_pull(wl, flags=flags, mixed=mixed)
+
+
+# ---- 16-bit packet values ---------------------------------------------------------------------
+@pytest.mark.parametrize("flags", [dgs.DGS_PACKET_BF16, dgs.DGS_PACKET_FP16,
+                                   dgs.DGS_PACKET_BF16 | dgs.DGS_KEEP_LOCAL_MODEL | dgs.DGS_RESIDUAL_MODE,
+                                   dgs.DGS_PACKET_FP16 | dgs.DGS_KEEP_LOCAL_MODEL | dgs.DGS_NO_SPECULATION])
+def test_trajectory_with_16_bit_packet_values(flags):
+    # Gradients down to 1e-6: binary16 meets its subnormal range and zero, bfloat16 only loses precision.
+    # Packets (rounded values), worker state (Eq. 12 untouched, or t - q under Algorithm 1) and the server's
+    # remainders (Eq. 6b) must agree with the CPU checker bit for bit.
+    wl = W.custom("q16", [300, 7, 5000, 64, 1, 2049, 1531], 3, 30, 20_000, grad_kind="normal", grad_scale=1e-5)
+    replay_and_compare(wl, flags=flags, compare_state_every=7)
+
+
+def test_overlapped_events_with_bfloat16_packets_several_tiles():
+    wl = W.custom("q16-async", [150_000, 517, 90_000, 64, 70_001], 5, 60, 5_000, grad_kind="laplace")
+    replay_async_and_compare(wl, flags=dgs.DGS_PACKET_BF16 | dgs.DGS_KEEP_LOCAL_MODEL)
+
+
+def test_full_pull_with_bfloat16_packets_keeps_the_remainders():
+    wl = W.custom("q16-full", [40_000, 513, 9_001], 3, 15, 10_000, grad_kind="laplace")
+    replay_full_pull(wl, flags=dgs.DGS_PACKET_BF16 | dgs.DGS_KEEP_LOCAL_MODEL, mixed=True)
+
+
+def test_both_16_bit_formats_at_once_are_refused():
+    cfg = dgs.make_config(64, 1, 0.1, 0.9, [0], [64], [1], [1], flags=dgs.DGS_PACKET_BF16 | dgs.DGS_PACKET_FP16)
+    import ctypes as C
+    out = C.c_uint64(0)
+    assert dgs.lib().dgs_arena_bytes(C.byref(cfg), C.byref(out)) == dgs.DGS_EINVAL
 
 
 def test_full_pull_many_workers_several_tiles():
