@@ -543,7 +543,11 @@ int launch_select(dgs_ctx* c, const SelArgs& a_in, uint32_t worker, uint64_t age
   // those 48: finalize runs beside the push passes of later events and should hold few SMs.
   int fin_base = c->finalize_grid[MODE];
   if (3ull * a.pkt_count <= 48ull * kThreads * 8) fin_base = std::min(fin_base, 48);
-  const int fin_grid = std::min(c->finalize_max[MODE], std::max(fin_base, (int)(a.pkt_count / 4096)));
+  // With several layers the threads visit their candidates four times; as many CTAs as keep those candidates
+  // (about twice the entries) in the threads' registers, eight each, save the re-reads.
+  int fin_want = (int)(a.pkt_count / 4096);
+  if (c->cfg.num_segments > 1) fin_want = (int)((2ull * a.pkt_count + kThreads * 8 - 1) / (kThreads * 8));
+  const int fin_grid = std::min(c->finalize_max[MODE], std::max(fin_base, fin_want));
   a.workers = (uint32_t)fin_grid;
   a.packet_format = packet_format_of(c);
   if (c->cfg.flags & DGS_TEST_STALLED_BARRIER) {

@@ -1067,6 +1067,12 @@ __device__ __forceinline__ uint32_t seg_of(const uint32_t* off, uint32_t S, uint
   }
   return lo;
 }
+// The same for a thread that visits candidates in index order: consecutive candidates mostly lie in the
+// same layer, so the layer found last is tried first and the search is only made when it does not hold i.
+__device__ __forceinline__ uint32_t seg_near(const uint32_t* off, uint32_t S, uint32_t i, uint32_t& last) {
+  if (i < off[last] || i >= off[last + 1]) last = seg_of(off, S, i);
+  return last;
+}
 // slot of flat candidate p: last part with pre[part] <= p
 __device__ __forceinline__ uint32_t slot_of(const FinalizeShared& sh, uint32_t parts, uint32_t p, uint32_t* part_out) {
   uint32_t lo = 0, hi = parts - 1;
@@ -1281,6 +1287,7 @@ __global__ void __maxnreg__(64) k_finalize(Workspace ws, SelArgs a) {
     }
   }
 
+  uint32_t near_seg = 0;   // layer of the candidate this thread looked at last (S > 1)
   // visits this thread's candidates in flat order: fn(value, index)
   auto each_own = [&](auto fn) {
     if (per_thread <= (uint32_t)kKeep) {
@@ -1346,7 +1353,7 @@ __global__ void __maxnreg__(64) k_finalize(Workspace ws, SelArgs a) {
       }
       each_own([&](float v, uint32_t idx) {
         const uint32_t key = key_of(v);
-        const uint32_t seg = seg_of(seg_off, S, idx);
+        const uint32_t seg = seg_near(seg_off, S, idx, near_seg);
         const uint32_t prefix = seg_smem ? sm_seg_a[seg] : __ldcg(&ws.sel[seg].prefix);
         if ((key >> SH) == prefix) atomicAdd(hist + (size_t)seg * B + ((key >> (SH - 10)) & 1023u), 1u);
       });
@@ -1400,7 +1407,7 @@ __global__ void __maxnreg__(64) k_finalize(Workspace ws, SelArgs a) {
     const uint32_t key = key_of(v);
     uint32_t T = one_prefix;
     if (S > 1) {
-      const uint32_t seg = seg_of(seg_off, S, idx);
+      const uint32_t seg = seg_near(seg_off, S, idx, near_seg);
       T = seg_smem ? sm_seg_a[seg] : __ldcg(&ws.sel[seg].T);
     }
     if (key > T) mine += 1ull << 32;
@@ -1433,7 +1440,7 @@ __global__ void __maxnreg__(64) k_finalize(Workspace ws, SelArgs a) {
       uint32_t T = one_prefix, r = one_krem, pkt_off = 0;
       uint2 start = make_uint2(0, 0);
       if (S > 1) {
-        const uint32_t seg = seg_of(seg_off, S, idx);
+        const uint32_t seg = seg_near(seg_off, S, idx, near_seg);
         T = seg_smem ? sm_seg_a[seg] : __ldcg(&ws.sel[seg].T);
         r = seg_smem ? sm_seg_b[seg] : __ldcg(&ws.sel[seg].r);
         start = seg_smem ? sm_seg_start[seg] : __ldcg(ws.seg_start + seg);
