@@ -9,7 +9,7 @@ selection, 32 workers.  Prints ONE JSON line (rank 0).
 
 Timed region: K consecutive events with every gradient already resident in HBM,
 CUDA events on the library's stream, barrier + synchronize on both sides, max over
-ranks.  Before the W warm-up events an untimed pre-roll serves every worker once,
+ranks.  Before the W warm-up events an untimed pre-roll serves every worker three times,
 so that the timed events are steady-state ones (a worker's first arrival takes the
 two-pass selection route).  Each event reads a different gradient, velocity and
 difference vector (3 x 102 MB at the default workload, more than the L2), so no
@@ -86,7 +86,9 @@ def make_workload(name: str, seed: int, workers: int = 0):
 
 
 def preroll_events(wl) -> int:
-    return wl.num_workers if wl.schedule_kind == "cyclic" else 2 * wl.num_workers
+    """Untimed events before the warm-up: three rounds of the workers, so that every worker has come back,
+    carried bounds and the pulls' planned ranges exist, and even a short run times steady-state events."""
+    return 3 * wl.num_workers
 
 
 def config_of(wl, args, world: int = 1) -> dict:
