@@ -1920,17 +1920,22 @@ __global__ void __maxnreg__(32) k_catch_up(PacketLog lg, uint64_t first, uint32_
       float* const cur = dense ? sh.dense : sh.tab.vals;    // running values, by place
       constexpr int SPT = kCatchSlots / kCatchThreads;      // sparse: table slots per thread
       constexpr int EPT = kCatchDense / kCatchThreads;      // dense: elements per thread, element tid + j * kCatchThreads
+      constexpr int LB = EPT < 8 ? EPT : 8;                  // loads a thread has in flight together
       if (dense) {
-        // A warp's 32 threads hold one line at every step j: one 128-byte request per line that holds an entry.
-        // The copies go from global to shared memory asynchronously (no registers held while they are under
-        // way), all of them in flight together; elements of lines without an entry are never looked at.
+        // a warp's 32 threads hold one line at every step j: one 128-byte request per line that holds an entry
+#pragma unroll 1
+        for (int j0 = 0; j0 < EPT; j0 += LB) {
+          if ((uint32_t)(j0 * kCatchThreads) >= span) break;
+          float d[LB];
 #pragma unroll
-        for (int j = 0; j < EPT; ++j) {
-          const uint32_t off = tid + j * kCatchThreads;
-          if (off < span && dirty[off >> 5])
-            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_addr(sh.dense + off)), "l"(D + a0 + off) : "memory");
+          for (int j = 0; j < LB; ++j) {
+            const uint32_t off = tid + (j0 + j) * kCatchThreads;
+            d[j] = 0.f;
+            if (off < span && dirty[off >> 5]) d[j] = __ldcg(D + a0 + off);
+          }
+#pragma unroll
+          for (int j = 0; j < LB; ++j) sh.dense[tid + (j0 + j) * kCatchThreads] = d[j];
         }
-        asm volatile("cp.async.wait_all;" ::: "memory");
       } else {
         // one load of D per distinct index, all in flight together
         uint32_t k[SPT];
