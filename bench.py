@@ -384,10 +384,13 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
     dom = "stream_push" if ktimes["stream_push"][1] else max(ktimes, key=lambda k: ktimes[k][0])
     dom_ms, dom_cnt = stimes[dom]          # on its own (single-stream pass)
     ovl_ms, ovl_cnt = ktimes[dom]          # with the other streams' kernels beside it
+    # algorithmic bytes per launch: the streaming passes move whole vectors; the apply reads the packet and
+    # lowers theta (8 K read + 8 K read-modify-write); a catch-up lowers one difference vector by the packets
+    # of one round of the workers (8 bytes per entry, N K entries)
     kernel_bytes = {
         "stream_push": 12 * wl.n, "finalize_push": None, "two_pass_push": 8 * wl.n,
-        "scatter": None, "stream_pull": 4 * wl.n, "finalize_pull": None, "two_pass_pull": 4 * wl.n,
-        "catch_up": None,
+        "scatter": 16 * wl.K_push, "stream_pull": 4 * wl.n, "finalize_pull": None, "two_pass_pull": 4 * wl.n,
+        "catch_up": 8 * wl.K_push * N,
     }
     achieved = kernel_bytes[dom] / (dom_ms * 1e-3 / max(dom_cnt, 1)) / 1e9
     achieved_ovl = kernel_bytes[dom] / (ovl_ms * 1e-3 / max(ovl_cnt, 1)) / 1e9
@@ -423,7 +426,9 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
         "kernels_single_stream": {k: {"launches": c, "us_per_launch": (1e3 * ms / c if c else None),
                                       "share": ms / stot_ms,
                                       "GB/s": (kernel_bytes[k] / (ms * 1e-3 / c) / 1e9
-                                               if c and ms > 0 and kernel_bytes[k] else None)}
+                                               if c and ms > 0 and kernel_bytes[k] else None),
+                                      "frac_of_peak": (kernel_bytes[k] / (ms * 1e-3 / c) / 1e9 / peak
+                                                       if c and ms > 0 and kernel_bytes[k] else None)}
                                   for k, (ms, c) in stimes.items()},
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": peak_kind, "traffic": traffic,
