@@ -448,9 +448,55 @@ def run_ours(args, wl, rank: int, world: int, local_rank: int, dist) -> dict:
     }
     if world == 1 and N > 1 and not args.no_jitter:
         out["jittered_arrivals"] = run_jittered(wl, grads, pool, theta0, min(K, 512), dev)
+    if world == 1 and N > 1 and not args.no_jitter:
+        out["full_pull"] = run_full_pull(wl, sched, grads, pool, theta0, min(K, 512), dev)
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(wl, args.cpu_seconds)
     return out
+
+
+def run_full_pull(wl, sched, grads, pool, theta0, K, dev) -> dict:
+    """The same workload with the pull that has no secondary compression (the paper's normal case): every
+    pull sends all nonzero entries of the worker's difference vector (dgs_worker_pull_all) instead of the
+    k largest.  Same arrival order, same gradients; push, apply and pull are three calls per event."""
+    import torch
+
+    import paper_1910_10929_b200 as dgs
+    N = wl.num_workers
+    # a worker's difference vector holds what arrived since its previous pull: a round of the workers in a
+    # fixed cycle, now and then much more under random arrivals
+    cap = int(min(wl.n, (2 if wl.schedule_kind == "cyclic" else 16) * N * wl.K_push))
+    ctx = dgs.Context.from_workload(wl, theta0=theta0, pull_all_capacity=cap)
+    pre = preroll_events(wl)
+    sched = np.resize(sched, pre + K)
+
+    def event(e):
+        w = int(sched[e])
+        pkt = ctx.worker_push(w, grads[e % pool])
+        ctx.server_apply(w, pkt)
+        return ctx.worker_pull_all(w)
+
+    for e in range(pre):
+        event(e)
+    ctx.flush()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    ev0.record(ctx.stream)
+    last = None
+    for e in range(pre, pre + K):
+        last = event(e)
+    ctx.flush()
+    ev1.record(ctx.stream)
+    torch.cuda.synchronize(dev)
+    idx, _ = ctx.var_packet(last)
+    status = ctx.status()
+    assert status in (0, dgs.DGS_ELIMIT), "device status word is not clean"
+    ctx.close()
+    t = ev0.elapsed_time(ev1) * 1e-3
+    return {"pull": "all nonzero entries of the difference vector (no secondary compression)", "events": K,
+            "value": K / t, "unit": UNIT, "ms_per_step": 1e3 * t / K, "packet_capacity": cap,
+            "entries_in_last_pull_packet": int(idx.numel()),
+            "a_packet_overflowed_its_capacity": status == dgs.DGS_ELIMIT}
 
 
 def run_jittered(wl, grads, pool, theta0, K, dev) -> dict:
