@@ -1795,7 +1795,7 @@ static_assert(kCatchDense / kWarpTile + 2 <= kCatchBlocks, "a dense piece's bloc
 __global__ void __maxnreg__(32) k_catch_up(PacketLog lg, uint64_t first, uint32_t count,
                                                        float* __restrict__ D, uint32_t* __restrict__ blk_max,
                                                        uint64_t n) {
-  __shared__ CatchShared sh;
+  __shared__ __align__(16) CatchShared sh;
   const uint32_t tid = threadIdx.x;
   if (count == 0 || count > (uint32_t)kCatchMaxPackets) return;
   uint8_t* const dirty = reinterpret_cast<uint8_t*>(sh.dirty);
@@ -1827,6 +1827,15 @@ __global__ void __maxnreg__(32) k_catch_up(PacketLog lg, uint64_t first, uint32_
     for (int s = tid; s < kCatchBlocks; s += kCatchThreads) sh.bmax[s] = 0;
     for (int s = tid; s < kCatchLines / 4; s += kCatchThreads) sh.dirty[s] = 0;
     __syncthreads();
+    // If what is left of the range fits a dense piece, its lines of D set out for shared memory now
+    // (asynchronous 16-byte copies past L1), while the entries are being counted and gathered: where
+    // updates crowd nearly every line holds an entry anyway, and a trip to memory leaves the chain.
+    const bool ahead = range_b - (a & ~31u) <= (uint32_t)kCatchDense;
+    if (ahead) {
+      const uint32_t a0 = a & ~31u, floats = (range_b - a0 + 31u) & ~31u;   // whole lines; D is padded beyond n
+      for (uint32_t q = tid * 4; q < floats; q += kCatchThreads * 4)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(sh.dense + q)), "l"(D + a0 + q) : "memory");
+    }
     if (tid < count) sh.hi[tid] = sh.end[tid];
     uint32_t b = range_b;
     uint32_t E;
@@ -1921,7 +1930,9 @@ __global__ void __maxnreg__(32) k_catch_up(PacketLog lg, uint64_t first, uint32_
       constexpr int SPT = kCatchSlots / kCatchThreads;      // sparse: table slots per thread
       constexpr int EPT = kCatchDense / kCatchThreads;      // dense: elements per thread, element tid + j * kCatchThreads
       constexpr int LB = EPT < 8 ? EPT : 8;                  // loads a thread has in flight together
-      if (dense) {
+      if (dense && ahead) {
+        asm volatile("cp.async.wait_all;" ::: "memory");   // the lines that set out at the start of the piece
+      } else if (dense) {
         // a warp's 32 threads hold one line at every step j: one 128-byte request per line that holds an entry
 #pragma unroll 1
         for (int j0 = 0; j0 < EPT; j0 += LB) {
@@ -2030,6 +2041,7 @@ __global__ void __maxnreg__(32) k_catch_up(PacketLog lg, uint64_t first, uint32_
         if (v) atomicMax(blk_max + a / kWarpTile + s, v);
       }
     }
+    asm volatile("cp.async.wait_all;" ::: "memory");   // (copies of a piece that turned out empty: nothing may still land)
     if (b == range_b) break;
     __syncthreads();   // the tables and the pieces are read until here
     if (tid < count) sh.lo[tid] = sh.hi[tid];
