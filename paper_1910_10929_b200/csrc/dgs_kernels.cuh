@@ -1681,7 +1681,7 @@ constexpr int kCatchCap = 1024;          // entries a CTA of k_catch_up can hold
 constexpr int kCatchSlots = 2 * kCatchCap;        // sparse pieces: slots of the table of distinct indices (>= 2 * kCatchCap)
 constexpr int kCatchDense = 2 * kCatchSlots;      // dense pieces: elements of D a piece can mirror (= the bytes of the sparse table)
 constexpr int kCatchLines = kCatchDense / 32;
-constexpr uint32_t kCatchTarget = kCatchCap / 2;  // entries per range of the log the launch aims at
+constexpr uint32_t kCatchTarget = 3 * kCatchCap / 4;  // entries per range of the log the launch aims at (a range that holds more than kCatchCap is halved)
 constexpr int kCatchMaxGrid = 16384;
 constexpr int kCatchBlocks = kCatchCap / 8 < 16 ? 16 : kCatchCap / 8;   // blocks of D whose bounds a CTA of k_catch_up collects in shared memory first
 constexpr int catch_log2(int v) { return v <= 1 ? 0 : 1 + catch_log2(v / 2); }
