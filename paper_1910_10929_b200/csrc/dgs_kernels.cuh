@@ -2002,24 +2002,37 @@ __global__ void __maxnreg__(32) k_catch_up(PacketLog lg, uint64_t first, uint32_
       // Back to memory.  The blocks' bounds must stay upper bounds: the largest new magnitude per block is
       // collected in shared memory, one global atomic per block afterwards.
       if (dense) {
+        // A warp takes four consecutive lines at a time (their dirty flags are one word); the loads of the
+        // four are in flight together, and a block's bound gets one reduction where the four lie in one block.
         const uint32_t lead = a - a0;            // elements of the first line that belong to the range before
-        const uint32_t blk0 = a / kWarpTile;
+        const uint32_t blk0 = a / kWarpTile, line0 = a0 >> 5;
+        const uint32_t lines = (span + 31u) >> 5, lane = tid & 31u;
 #pragma unroll 1
-        for (int j = 0; j < EPT; ++j) {
-          const uint32_t off = tid + j * kCatchThreads;
-          if ((uint32_t)(j * kCatchThreads) >= span) break;
-          const bool live = off < span && dirty[off >> 5] != 0;    // the same for the whole warp but for off < span
-          uint32_t key = 0;
-          if (live && off >= lead) {
-            const float r = sh.dense[off];
-            __stcg(D + a0 + off, r);
-            key = key_of(r);
+        for (uint32_t l0 = (tid >> 5) * 4; l0 < lines; l0 += (kCatchThreads / 32) * 4) {
+          const uint32_t flags = sh.dirty[l0 >> 2];
+          if (flags == 0) continue;
+          uint32_t key[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const uint32_t off = (l0 + u) * 32 + lane;
+            key[u] = 0;
+            if (((flags >> (8 * u)) & 0xFFu) && off < span && off >= lead) {
+              const float r = sh.dense[off];
+              __stcg(D + a0 + off, r);
+              key[u] = key_of(r);
+            }
           }
-          if (__any_sync(kFull, live)) {
-            key = __reduce_max_sync(kFull, key);
-            // a line lies inside one block (lines and blocks start at multiples of 32 and of kWarpTile)
-            uint32_t* const bm = sh.bmax + ((a0 + off) / kWarpTile - blk0);
-            if ((tid & 31u) == 0 && key > *bm) atomicMax(bm, key);
+          // a line lies inside one block (lines and blocks start at multiples of 32 and of kWarpTile)
+          const uint32_t b_first = (line0 + l0) / (kWarpTile / 32) - blk0, b_last = (line0 + l0 + 3) / (kWarpTile / 32) - blk0;
+          if (b_first == b_last) {
+            const uint32_t k4 = __reduce_max_sync(kFull, max(max(key[0], key[1]), max(key[2], key[3])));
+            if (lane == 0 && k4) atomicMax(sh.bmax + b_first, k4);
+          } else {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const uint32_t k1 = __reduce_max_sync(kFull, key[u]);
+              if (lane == 0 && k1) atomicMax(sh.bmax + ((line0 + l0 + u) / (kWarpTile / 32) - blk0), k1);
+            }
           }
         }
       } else {
