@@ -1825,8 +1825,7 @@ __global__ void __maxnreg__(32) k_catch_up(PacketLog lg, uint64_t first, uint32_
   uint32_t a = sh.ab[0];
   for (;;) {   // one round per piece [a, b) of the range; everything here is uniform over the CTA
     for (int s = tid; s < kCatchBlocks; s += kCatchThreads) sh.bmax[s] = 0;
-    for (int s = tid; s < kCatchLines / 4; s += kCatchThreads) sh.dirty[s] = 0;
-    __syncthreads();
+    for (int s = tid; s < kCatchLines / 4; s += kCatchThreads) sh.dirty[s] = 0;   // (first written after the barriers below)
     // If what is left of the range fits a dense piece, its lines of D set out for shared memory now
     // (asynchronous 16-byte copies past L1), while the entries are being counted and gathered: where
     // updates crowd nearly every line holds an entry anyway, and a trip to memory leaves the chain.
@@ -1891,10 +1890,11 @@ __global__ void __maxnreg__(32) k_catch_up(PacketLog lg, uint64_t first, uint32_
         ei[u] = kFull;
         ev[u] = 0.f;
         if (e < E) {
-          uint32_t l = 0, r = count - 1;        // last packet p with pre[p] <= e
-          while (l < r) {
-            const uint32_t mid = (l + r + 1) >> 1;
-            if (sh.pre[mid] <= e) l = mid; else r = mid - 1;
+          uint32_t l = 0;                       // last packet p with pre[p] <= e: the same six probes for every
+#pragma unroll                                  // entry, so that the searches of a thread's entries overlap
+          for (uint32_t step = kCatchMaxPackets / 2; step >= 1; step >>= 1) {
+            const uint32_t t = l + step;
+            if (t < count && sh.pre[t] <= e) l = t;
           }
           const uint64_t at = ((first + l) % lg.ring) * (uint64_t)lg.stride + sh.lo[l] + (e - sh.pre[l]);
           ei[u] = __ldcg(lg.idx + at);
