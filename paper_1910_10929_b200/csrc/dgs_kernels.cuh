@@ -62,6 +62,8 @@ struct SegSel {        // per-layer selection state of the selection in flight
   uint32_t T;          // k-th largest key
   uint32_t r;          // entries with key == T that are taken (lowest indices)
   uint32_t neq;        // candidates with key == T
+  uint32_t wrem;       // bound suggested for a later selection: rank of its entry inside the first-level bin of
+                       // the k-th, when it lies in that bin (the second level then places it), else 0
 };
 
 // word indices in Workspace::sync
@@ -1149,6 +1151,7 @@ __global__ void __maxnreg__(64) k_finalize(Workspace ws, SelArgs a) {
   uint32_t ridx[kKeep];               // valid when per_thread <= kKeep
   uint32_t bar_target = 0;
   uint32_t one_prefix = 0, one_krem = 0;   // S == 1: the layer's selection state, the same in every thread of the grid
+  uint32_t one_wrem = 0;                   // S == 1, CTA 0: SegSel::wrem of the layer
   bool redo = false;
   for (int attempt = 0; attempt < 2; ++attempt) {
     if (redo) {
@@ -1238,8 +1241,10 @@ __global__ void __maxnreg__(64) k_finalize(Workspace ws, SelArgs a) {
         if (owner && threadIdx.x == 0) {
           ws.sel[s].prefix = bin;
           ws.sel[s].krem = krem;
+          ws.sel[s].wrem = 0;
           atomicAdd(ws.stats + 2, (unsigned long long)total);
         }
+        one_wrem = 0;
         if (owner && a.speculate) {
           // bound suggested for a later selection on this layer
           const uint32_t want = spec_want(k);
@@ -1249,14 +1254,37 @@ __global__ void __maxnreg__(64) k_finalize(Workspace ws, SelArgs a) {
             block_pick<kBins1>(h, want, lbin, lrem, sh.warp_scan, sh.res);
             const uint32_t in_force = (redo || a.force_two_pass) ? __ldcg(ws.L_safe + s) : a.L_in[s];
             lkey = bound_inside_bin(lbin, lrem, __ldcg(h + lbin), in_force);
+            // Inside the bin of the k-th the keys are anything but evenly spread where a push has run for a
+            // while: what was never sent piles up right below the k-th, what lies above it is a thin tail, and
+            // a bound interpolated from the top of the bin lands in the tail (the next selection then finds
+            // fewer than k candidates and starts over).  The second level counts that bin in 1024 parts.
+            if (lbin == bin && bin > 0) {
+              const uint32_t roomy = lrem + want / 16;          // a little beyond, if the bin holds that many
+              one_wrem = roomy <= __ldcg(h + bin) ? roomy : lrem;
+              if (threadIdx.x == 0) ws.sel[s].wrem = one_wrem;
+            }
           } else if (redo || a.force_two_pass) {
             lkey = __ldcg(ws.L_wide + s);         // known from the histogram of the whole input
             lbin = lkey >> 20;
           } else {
-            // fewer candidates than wished for and nothing known below the bound: lower it by half an octave
-            const uint32_t used = a.L_in[s] >> 20;
-            lbin = used > 4 ? used - 4 : 0;
-            lkey = lbin << 20;
+            // Fewer candidates than wished for (but at least k) and nothing known below the bound: lower it by
+            // as much as would hold the missing ones at the density seen right above it -- what was never sent
+            // piles up below the k-th, so half an octave down may hold a hundred times the wished-for number --
+            // and by half an octave only where too few keys lie above the bound to tell.
+            const uint32_t L_used = a.L_in[s], used = L_used >> 20;
+            uint32_t pop = __ldcg(h + used), width = ((used + 1u) << 20) - L_used;
+            if (pop < 64u && used + 1u < (uint32_t)kBins1) {
+              pop += __ldcg(h + used + 1u);
+              width += 1u << 20;
+            }
+            const float step = 1.5f * (float)(want + want / 16 - total) / (float)max(pop, 1u) * (float)width;
+            if (pop >= 64u && step < (float)(4u << 20)) {
+              const uint32_t down = (uint32_t)step + 1u;
+              lkey = L_used > down ? L_used - down : 0u;
+            } else {
+              lkey = used > 4 ? (used - 4) << 20 : 0u;
+            }
+            lbin = lkey >> 20;
           }
           __syncthreads();
           // A bound of zero makes every element of the layer a candidate (zeros included).  That is fine for a
@@ -1344,6 +1372,11 @@ __global__ void __maxnreg__(64) k_finalize(Workspace ws, SelArgs a) {
       }
       uint32_t bin, krem;
       block_pick<B>(hist, one_krem, bin, krem, sh.warp_scan, sh.res);
+      if (level == 2 && cta == 0 && one_wrem) {   // (CTA-uniform) the suggested bound: lower edge of the part that holds its entry
+        uint32_t wsub, wleft;
+        block_pick<B>(hist, one_wrem, wsub, wleft, sh.warp_scan, sh.res);
+        if (threadIdx.x == 0) a.L_next[0] = ((one_prefix << 10) | wsub) << 10;
+      }
       one_prefix = (one_prefix << 10) | bin;
       one_krem = krem;
     } else {
@@ -1362,6 +1395,13 @@ __global__ void __maxnreg__(64) k_finalize(Workspace ws, SelArgs a) {
         uint32_t bin, krem;
         uint32_t* h = hist + (size_t)s * B;
         block_pick<B>(h, __ldcg(&ws.sel[s].krem), bin, krem, sh.warp_scan, sh.res);
+        const uint32_t wrem = level == 2 ? __ldcg(&ws.sel[s].wrem) : 0u;   // written by this CTA at the first level
+        if (wrem) {
+          uint32_t wsub, wleft;
+          block_pick<B>(h, wrem, wsub, wleft, sh.warp_scan, sh.res);
+          if (threadIdx.x == 0) a.L_next[s] = ((__ldcg(&ws.sel[s].prefix) << 10) | wsub) << 10;
+          __syncthreads();   // the prefix is read before it is extended below
+        }
         if (threadIdx.x == 0) {
           const uint32_t pre = (__ldcg(&ws.sel[s].prefix) << 10) | bin;
           ws.sel[s].prefix = pre;
