@@ -38,7 +38,7 @@ constexpr int kWorkerStreams = 4, kServerStreams = 6;   // library streams for t
 constexpr int kPushSets = kWorkerStreams;  // scratch sets and spare velocity buffers of the pushes
 constexpr int kPullSets = kServerStreams;  // scratch sets of the pulls
 constexpr int kAllSets = kPushSets + kPullSets;
-constexpr int kLogRingMax = 64;             // most packets the apply log keeps
+constexpr int kLogRingMax = 128;            // most packets the apply log keeps
 constexpr int kLogSlack = 32;               // slots of the log beyond one per worker
 enum StreamId : int { kStW0 = 0, kStApply = kWorkerStreams, kStS0 = kWorkerStreams + 1,
                       kNumStreams = kWorkerStreams + 1 + kServerStreams };
@@ -191,7 +191,10 @@ void make_layout(const dgs_config* c, Layout* L) {
   // A slot of the log is reused `ring` packets later, and the apply that refills it waits for every catch-up that
   // still reads the old packet.  A worker that comes back after N events reads the N newest packets, so ring - N
   // is how many events the server side of an event may lag behind the pushes before the pushes stall.
-  L->log_ring = (uint32_t)std::min<uint64_t>(kLogRingMax, std::max<uint64_t>(N + kLogSlack, 16));
+  // (with irregular arrivals a worker is often away for more than N events -- one gap in eight is longer than 2 N when
+  // every event's worker is drawn at random -- and a worker about to fall off the ring is caught up on the apply
+  // stream, in the way of every later event: four rounds of room where that many packets fit the cap)
+  L->log_ring = (uint32_t)std::min<uint64_t>(kLogRingMax, std::max<uint64_t>(std::max<uint64_t>(N + kLogSlack, 4 * N), 16));
   L->log_stride = (uint32_t)align_up(L->K[0], 64);
   L->log_idx = take((uint64_t)L->log_ring * L->log_stride * 4);
   L->log_val = take((uint64_t)L->log_ring * L->log_stride * 4);

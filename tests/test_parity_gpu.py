@@ -169,8 +169,9 @@ def test_pull_skips_cold_chunks_and_notices_when_they_heat_up():
 
 
 def test_more_workers_than_packets_kept():
-    # 70 workers in a fixed cycle: every difference vector is 70 packets behind when its worker returns
-    wl = W.custom("many", [30_000, 301, 2_048], 70, 180, 10_000, grad_kind="normal", schedule_kind="cyclic")
+    # 140 workers in a fixed cycle: every difference vector is 140 packets behind when its worker returns,
+    # more than the library keeps (128 at most)
+    wl = W.custom("many", [30_000, 301, 2_048], 140, 330, 10_000, grad_kind="normal", schedule_kind="cyclic")
     replay_async_and_compare(wl)
 
 
