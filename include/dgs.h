@@ -218,8 +218,9 @@ int dgs_status(dgs_ctx* ctx, int* device_status);
 
 /* Waits for all work in flight and reports counters: out[0] selections served by the
  * single-pass (speculative) route, out[1] selections that took the two-pass
- * route, out[2] server timestamp t (packets applied), out[3] candidates the finalize
- * steps have examined in total (the k selected ones included). */
+ * route from the start or started over because the carried bound admitted fewer
+ * than k candidates, out[2] server timestamp t (packets applied), out[3] candidates
+ * the finalize steps have examined in total (the k selected ones included). */
 int dgs_stats(dgs_ctx* ctx, uint64_t out[4]);
 
 /* Waits for all work in flight and reports how much of the difference vectors the pulls'
